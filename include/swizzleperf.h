@@ -1,0 +1,151 @@
+/* swizzleperf.h -- C ABI of libswizzleperf.so
+ *
+ * A tiled dense bf16 GEMM for NVIDIA B200 (sm_100a) whose block-to-output-tile mapping
+ * is a programmable "swizzle": a bijective remap of tile ids, as in the GEMM case study
+ * of the SwizzlePerf paper (arXiv 2508.20258, appendix "Case Study: GEMM Swizzling").
+ *
+ * Vocabulary.  C (M x N) = A (M x K) . B (K x N) is cut into Tm x Tn output tiles,
+ * Tm = ceil(M / tileM), Tn = ceil(N / tileN), T = Tm * Tn.  The logical id of tile
+ * (tm, tn) is t = tm * Tn + tn (the row-major decomposition pid_m = pid / Tn,
+ * pid_n = pid % Tn of the paper's hardware-unaware listing).  Blocks are issued in
+ * slot order s = 0 .. T-1; the remap is perm[s] = t, "the block issued at slot s
+ * computes tile t" -- the direction of the paper's  pid = f(pid)  (hardware id in,
+ * logical id out).  A remap must be a bijection on [0, T); the paper counts anything
+ * else as a broken mapping, and every entry point here rejects it before any launch.
+ *
+ * Conventions.  Every function returns an sp_status (0 = success) and never throws,
+ * aborts or prints.  "host" / "device" below says where a pointer must point.  The
+ * caller owns every buffer it passes; the library owns only its internal caches (tile
+ * tables, a status word), released by sp_shutdown().  All device work is enqueued on the
+ * caller's stream; nothing synchronises unless stated.
+ */
+#ifndef SWIZZLEPERF_H_
+#define SWIZZLEPERF_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SP_OK = 0,
+  SP_ERR_INVALID_ARG = 1,   /* NULL pointer, non-positive size, bad parameter value            */
+  SP_ERR_NOT_BIJECTIVE = 2, /* the requested remap does not hit every tile id exactly once     */
+  SP_ERR_UNSUPPORTED = 3,   /* tile shape / dtype / size outside what the kernels implement    */
+  SP_ERR_ALIGNMENT = 4,     /* pointer not 16-byte aligned, or K / N not a multiple of 8       */
+  SP_ERR_CUDA = 5,          /* a CUDA runtime or driver call failed (see sp_last_error)        */
+  SP_ERR_TIMEOUT = 6,       /* a bounded device-side wait expired; output is undefined         */
+  SP_ERR_DEVICE = 7         /* no usable sm_100 device                                         */
+} sp_status;
+
+/* Tile orders.  SP_XCD is the paper's formula; the others are this library's. */
+typedef enum {
+  SP_ROW_MAJOR = 0, /* perm[s] = s (the paper's unswizzled baseline)                                        */
+  SP_COL_MAJOR = 1, /* tile columns outer, tile rows inner                                                  */
+  SP_GROUP_M = 2,   /* supertiles of `group` tile rows: per band walk columns, per column walk band rows    */
+  SP_GROUP_N = 3,   /* supertiles of `group` tile columns (transpose of SP_GROUP_M)                         */
+  SP_MORTON = 4,    /* Z-order on the enclosing 2^k square (k minimal), cells outside the grid skipped;     */
+                    /*   the longer grid side is walked by the curve's y (odd bits)                         */
+  SP_HILBERT = 5,   /* Hilbert order on the same square, same skipping, curve from (0,0) to (2^k-1,0)       */
+  SP_XCD = 6,       /* paper, GEMM listing: within each window of `wave` slots of size n,                   */
+                    /*   p -> (p % X) * ceil(n / X) + p / X, X = num_xcds.  With xcd_balanced = 1 the       */
+                    /*   remainder-aware form p -> (p % X) * (n / X) + min(p % X, n % X) + p / X, which is  */
+                    /*   a bijection for every n and equals the printed form when X divides n.              */
+  SP_DIE_SPLIT = 7, /* tile space cut in two halves along split_axis (half 0 gets the ceil), each half a    */
+                    /*   grid of its own ordered by inner_scheme; perm = half 0 then half 1, or alternating */
+                    /*   (slot parity = half, the paper's formula with two chiplets) when interleave = 1    */
+  SP_CUSTOM = 8     /* caller-supplied table                                                                */
+} sp_scheme;
+
+/* sp_params.flags */
+#define SP_FLAG_TRACE 1u /* reserved for sp_gemm_trace */
+
+typedef struct {
+  uint32_t struct_size;       /* must be sizeof(sp_params)                                                  */
+  int32_t group;              /* G >= 1 for SP_GROUP_M / SP_GROUP_N                                         */
+  int32_t num_xcds;           /* X >= 1 for SP_XCD                                                          */
+  int32_t wave;               /* W for SP_XCD: window length in slots; 0 means W = T                        */
+  int32_t xcd_balanced;       /* SP_XCD: 0 = formula exactly as printed (may be rejected), 1 = balanced     */
+  int32_t split_axis;         /* SP_DIE_SPLIT: 0 = halve the tile rows, 1 = halve the tile columns          */
+  int32_t inner_scheme;       /* SP_DIE_SPLIT: order inside each half: SP_ROW_MAJOR .. SP_HILBERT           */
+  int32_t inner_group;        /* SP_DIE_SPLIT: G of the inner scheme                                        */
+  int32_t interleave;         /* SP_DIE_SPLIT: 0 = concatenated halves, 1 = alternating merge               */
+  const int32_t* custom_perm; /* SP_CUSTOM: HOST array of T tile ids (validated, copied)                    */
+  int32_t tile_m, tile_n;     /* sp_gemm*: 128x128, 128x256 (one CTA per tile) or 256x128, 256x256 (a CTA   */
+                              /*   pair per tile); 0,0 = 256x256.  Ignored by sp_tile_map*.                 */
+  int32_t out_dtype;          /* sp_gemm*: 0 = C is bf16 (round to nearest even), 1 = C is fp32             */
+  int32_t b_layout;           /* sp_gemm*: 0 = B is K x N row-major, 1 = B is N x K row-major               */
+  uint32_t flags;             /* 0                                                                          */
+} sp_params;
+
+/* One record per tile, written by sp_gemm_trace. */
+typedef struct {
+  int32_t slot;      /* issue slot s                                   */
+  int32_t tile;      /* logical tile id executed at that slot          */
+  int32_t smid;      /* %smid of the (leader) CTA that ran it          */
+  int32_t unit;      /* index of the persistent CTA / CTA pair         */
+  uint64_t t_begin;  /* %globaltimer when its first load was issued    */
+  uint64_t t_end;    /* %globaltimer when its last store was issued    */
+} sp_trace_rec;
+
+/* Number of tiles T = ceil(M/tileM) * ceil(N/tileN); -1 on non-positive arguments. */
+int64_t sp_tile_count(int64_t M, int64_t N, int32_t tileM, int32_t tileN);
+
+/* The remap (paper: the recomputed pid of each block).
+ *   out_perm : HOST, caller-owned, T int32 entries; out_perm[s] = tile run at slot s.
+ *   params   : HOST; may be NULL for schemes that need no parameter.
+ * Errors: SP_ERR_INVALID_ARG (sizes <= 0, T > 2^24, G < 1, X < 1, wave < 0, bad axis / inner scheme,
+ * wrong struct_size, NULL out_perm), SP_ERR_NOT_BIJECTIVE (printed SP_XCD form when X does not
+ * divide a window, bad custom table).  On any error out_perm is left untouched.  Pure host code. */
+int sp_tile_map(int64_t M, int64_t N, int32_t tileM, int32_t tileN, int scheme, const sp_params* params,
+                int32_t* out_perm);
+
+/* Same remap, evaluated by the DEVICE code the GEMM scheduler uses, written to
+ *   out_perm_dev : DEVICE, T int32 entries, on `stream` (asynchronous).
+ * Validation (including bijectivity) happens on the host first; same error codes. */
+int sp_tile_map_device(int64_t M, int64_t N, int32_t tileM, int32_t tileN, int scheme, const sp_params* params,
+                       int32_t* out_perm_dev, void* stream);
+
+/* C = A . B under the given tile order (paper: the GEMM whose block ids are remapped).
+ *   A : DEVICE, bf16, M x K row-major, read-only.
+ *   B : DEVICE, bf16, K x N row-major (b_layout 0) or N x K row-major (b_layout 1), read-only.
+ *   C : DEVICE, M x N row-major, bf16 or fp32 per params->out_dtype; fully overwritten; must not alias A or B.
+ *   stream : cudaStream_t (NULL = default stream).  Asynchronous.
+ * Products are accumulated in fp32 on the tensor cores.  M and N need not be tile multiples.
+ * Errors (all detected on the host, nothing launched): as sp_tile_map, plus SP_ERR_ALIGNMENT (A, B or C not
+ * 16-byte aligned; K or N not a multiple of 8), SP_ERR_UNSUPPORTED (tile shape), SP_ERR_DEVICE, SP_ERR_CUDA.
+ * The first call for a given (grid, scheme) may allocate a cached tile table; later calls allocate nothing.
+ * A device-side wait that expires is reported by sp_get_status, not here. */
+int sp_gemm(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t K, int scheme,
+            const sp_params* params, void* stream);
+
+/* sp_gemm that also records, for every tile, where and when it ran.
+ *   trace_dev : DEVICE, T sp_trace_rec entries, indexed by slot. */
+int sp_gemm_trace(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t K, int scheme,
+                  const sp_params* params, void* stream, sp_trace_rec* trace_dev);
+
+/* Number of persistent CTAs (tile 128xN) or CTA pairs (tile 256xN) sp_gemm launches for T tiles;
+ * slot s is run by unit s % units in round s / units.  Returns -1 on error. */
+int sp_gemm_units(int32_t tile_m, int32_t tile_n, int64_t T);
+
+/* Launch-order probe (the counterpart of the paper's "default scheduling policy" context):
+ * launches `n_blocks` trivial blocks in clusters of `cluster` (1 or 2) and records for block b
+ *   smid_host[b] = %smid, start_host[b] = %globaltimer at entry.  HOST arrays of n_blocks. Synchronous. */
+int sp_probe_dispatch(int32_t n_blocks, int32_t cluster, int32_t* smid_host, uint64_t* start_host);
+
+/* Synchronises `stream`, then returns and clears the device status word of the current device:
+ * SP_OK, or SP_ERR_TIMEOUT if a kernel gave up on a bounded wait since the last call.
+ * *detail (HOST, may be NULL) receives the raw word (which wait, which role). */
+int sp_get_status(void* stream, int32_t* detail);
+
+/* Text for the last error on the calling thread; valid until that thread's next call. Never NULL. */
+const char* sp_last_error(void);
+
+/* Frees the library's caches on every device it touched.  No call may be in flight. */
+void sp_shutdown(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SWIZZLEPERF_H_ */

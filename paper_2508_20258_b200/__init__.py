@@ -1,0 +1,13 @@
+"""B200-native swizzled tiled GEMM: Python face of libswizzleperf.so.
+
+``tile_map`` returns the remap of tile ids, ``gemm`` runs the bf16 GEMM under it; both are
+thin wrappers over the C ABI declared in ``include/swizzleperf.h``.  All computation runs
+in hand-written sm_100a kernels; nothing here falls back to another implementation.
+"""
+
+from .binding import (  # noqa: F401
+    COL_MAJOR, CUSTOM, DIE_SPLIT, GROUP_M, GROUP_N, HILBERT, MORTON, ROW_MAJOR, XCD, SCHEME_NAMES,
+    ERR_ALIGNMENT, ERR_CUDA, ERR_DEVICE, ERR_INVALID_ARG, ERR_NOT_BIJECTIVE, ERR_TIMEOUT, ERR_UNSUPPORTED, OK,
+    SpError, SpParams, gemm, gemm_trace, gemm_units, get_status, last_error, lib, make_params, probe_dispatch,
+    shutdown, tile_count, tile_map, tile_map_device,
+)

@@ -1,0 +1,386 @@
+// C ABI of libswizzleperf.so: argument validation, the host remap, caches, status.
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <mutex>
+#include <vector>
+
+#include "internal.h"
+
+namespace sp {
+
+static thread_local char g_err[512] = "";
+
+void set_error(const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof g_err, fmt, ap);
+  va_end(ap);
+}
+
+static bool plain_inner(int s) { return s >= kRow && s <= kHilbert; }
+
+int resolve_sched(int64_t M, int64_t N, int32_t tileM, int32_t tileN, int scheme, const sp_params* p, Sched* out) {
+  if (M <= 0 || N <= 0 || tileM <= 0 || tileN <= 0) {
+    set_error("sizes must be positive (M=%lld N=%lld tileM=%d tileN=%d)", (long long)M, (long long)N, tileM, tileN);
+    return SP_ERR_INVALID_ARG;
+  }
+  if (p && p->struct_size != sizeof(sp_params)) {
+    set_error("sp_params.struct_size is %u, expected %zu", p->struct_size, sizeof(sp_params));
+    return SP_ERR_INVALID_ARG;
+  }
+  const int64_t Tm = (M + tileM - 1) / tileM, Tn = (N + tileN - 1) / tileN;
+  if (Tm > kMaxTiles || Tn > kMaxTiles || Tm * Tn > kMaxTiles) {
+    set_error("too many tiles (%lld x %lld)", (long long)Tm, (long long)Tn);
+    return SP_ERR_INVALID_ARG;
+  }
+  Sched c;
+  memset(&c, 0, sizeof c);
+  c.scheme = scheme;
+  c.Tm = (int)Tm; c.Tn = (int)Tn; c.T = (int)(Tm * Tn);
+  c.group = 1; c.X = 1; c.W = c.T; c.inner_group = 1;
+  switch (scheme) {
+    case kRow: case kCol: case kMorton: case kHilbert: break;
+    case kGroupM: case kGroupN:
+      if (!p || p->group < 1) { set_error("group must be >= 1"); return SP_ERR_INVALID_ARG; }
+      c.group = p->group;
+      break;
+    case kXcd:
+      if (!p || p->num_xcds < 1) { set_error("num_xcds must be >= 1"); return SP_ERR_INVALID_ARG; }
+      if (p->wave < 0) { set_error("wave must be >= 0"); return SP_ERR_INVALID_ARG; }
+      c.X = p->num_xcds;
+      c.W = (p->wave == 0 || p->wave > c.T) ? c.T : p->wave;
+      c.balanced = p->xcd_balanced != 0;
+      break;
+    case kDieSplit:
+      if (!p) { set_error("SP_DIE_SPLIT needs parameters"); return SP_ERR_INVALID_ARG; }
+      if (p->split_axis != 0 && p->split_axis != 1) { set_error("split_axis must be 0 or 1"); return SP_ERR_INVALID_ARG; }
+      if (!plain_inner(p->inner_scheme)) { set_error("inner_scheme must be a plain order"); return SP_ERR_INVALID_ARG; }
+      c.axis = p->split_axis; c.inner = p->inner_scheme; c.interleave = p->interleave != 0;
+      if (c.inner == kGroupM || c.inner == kGroupN) {
+        if (p->inner_group < 1) { set_error("inner_group must be >= 1"); return SP_ERR_INVALID_ARG; }
+        c.inner_group = p->inner_group;
+      }
+      break;
+    case kCustom:
+      if (!p || !p->custom_perm) { set_error("SP_CUSTOM needs custom_perm"); return SP_ERR_INVALID_ARG; }
+      break;
+    default:
+      set_error("unknown scheme %d", scheme);
+      return SP_ERR_INVALID_ARG;
+  }
+  const bool curve = scheme == kMorton || scheme == kHilbert ||
+                     (scheme == kDieSplit && (c.inner == kMorton || c.inner == kHilbert));
+  if (curve && (c.Tm > kMaxCurveSide || c.Tn > kMaxCurveSide)) {
+    set_error("curve orders support grids up to %d tiles per side", kMaxCurveSide);
+    return SP_ERR_UNSUPPORTED;
+  }
+  c.use_table = arithmetic_scheme(c) ? 0 : 1;
+  *out = c;
+  return SP_OK;
+}
+
+static bool bijective(const std::vector<int32_t>& perm, int T) {
+  if ((int)perm.size() != T) return false;
+  std::vector<uint8_t> seen((size_t)T, 0);
+  for (int32_t t : perm) {
+    if (t < 0 || t >= T || seen[(size_t)t]) return false;
+    seen[(size_t)t] = 1;
+  }
+  return true;
+}
+
+// Walks a curve over a (rows x cols) sub-grid and emits grid ids of the whole grid.
+template <typename Emit>
+static void walk_curve(int kind, int rows, int cols, int row0, int col0, int Tn, Emit emit) {
+  const int k = curve_order(rows, cols);
+  const uint64_t cells = 1ull << (2 * k);
+  int idx = 0;
+  for (uint64_t d = 0; d < cells; ++d) {
+    int tm, tn;
+    if (curve_cell(kind, k, rows, cols, (uint32_t)d, tm, tn)) emit(idx++, (row0 + tm) * Tn + col0 + tn);
+  }
+}
+
+int build_perm_host(const Sched& c, const int32_t* custom, std::vector<int32_t>& perm) {
+  perm.assign((size_t)c.T, -1);
+  if (c.scheme == kCustom) {
+    if (!custom) { set_error("SP_CUSTOM needs custom_perm"); return SP_ERR_INVALID_ARG; }
+    for (int s = 0; s < c.T; ++s) perm[(size_t)s] = custom[s];
+  } else if (arithmetic_scheme(c)) {
+    for (int s = 0; s < c.T; ++s) perm[(size_t)s] = slot_to_tile(c, s);
+  } else if (c.scheme == kMorton || c.scheme == kHilbert) {
+    walk_curve(c.scheme, c.Tm, c.Tn, 0, 0, c.Tn, [&](int idx, int t) { perm[(size_t)idx] = t; });
+  } else {  // DIE_SPLIT with a curve inside each half
+    for (int half = 0; half < 2; ++half) {
+      const int cut = c.axis == 0 ? (c.Tm + 1) / 2 : (c.Tn + 1) / 2;
+      const int rows = c.axis == 0 ? (half ? c.Tm - cut : cut) : c.Tm;
+      const int cols = c.axis == 0 ? c.Tn : (half ? c.Tn - cut : cut);
+      if (rows == 0 || cols == 0) continue;
+      walk_curve(c.inner, rows, cols, (c.axis == 0 && half) ? cut : 0, (c.axis == 1 && half) ? cut : 0, c.Tn,
+                 [&](int idx, int t) { perm[(size_t)die_split_slot(c, half, idx)] = t; });
+    }
+  }
+  if (!bijective(perm, c.T)) {
+    set_error("remap (scheme %d) is not a bijection on [0,%d)", c.scheme, c.T);
+    return SP_ERR_NOT_BIJECTIVE;
+  }
+  return SP_OK;
+}
+
+// ------------------------------------------------------------------ per-device caches
+struct TableEntry {
+  Sched key;
+  uint64_t custom_hash;
+  int32_t* dev;
+  uint64_t stamp;
+};
+
+struct DeviceState {
+  int device = -1;
+  int32_t* status = nullptr;
+  std::vector<TableEntry> tables;
+};
+
+static std::mutex g_mu;
+static std::vector<DeviceState> g_devs;
+static uint64_t g_stamp = 0;
+constexpr size_t kMaxTables = 64;
+
+static DeviceState* device_state(int dev) {
+  for (auto& d : g_devs) if (d.device == dev) return &d;
+  g_devs.emplace_back();
+  g_devs.back().device = dev;
+  return &g_devs.back();
+}
+
+static uint64_t fnv(const int32_t* v, int n) {
+  uint64_t h = 1469598103934665603ull;
+  for (int i = 0; i < n; ++i) { h ^= (uint32_t)v[i]; h *= 1099511628211ull; }
+  return h;
+}
+
+#define SP_CUDA(call)                                                             \
+  do {                                                                            \
+    cudaError_t e_ = (call);                                                      \
+    if (e_ != cudaSuccess) {                                                      \
+      set_error("%s failed: %s", #call, cudaGetErrorString(e_));                  \
+      return SP_ERR_CUDA;                                                         \
+    }                                                                             \
+  } while (0)
+
+static int current_device(int* dev) {
+  int n = 0;
+  if (cudaGetDeviceCount(&n) != cudaSuccess || n == 0) {
+    cudaGetLastError();
+    set_error("no CUDA device");
+    return SP_ERR_DEVICE;
+  }
+  SP_CUDA(cudaGetDevice(dev));
+  int major = 0;
+  SP_CUDA(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, *dev));
+  if (major != 10) {
+    set_error("device %d has compute capability %d.x; this library is sm_100a only", *dev, major);
+    return SP_ERR_DEVICE;
+  }
+  return SP_OK;
+}
+
+static int get_status_word(DeviceState* ds) {
+  if (!ds->status) {
+    SP_CUDA(cudaMalloc(&ds->status, sizeof(int32_t)));
+    SP_CUDA(cudaMemset(ds->status, 0, sizeof(int32_t)));
+  }
+  return SP_OK;
+}
+
+// Device table for a table scheme; built by the device builder (or copied for SP_CUSTOM).
+static int get_table(DeviceState* ds, const Sched& c, const std::vector<int32_t>& host_perm, bool is_custom,
+                     cudaStream_t stream, const int32_t** out) {
+  const uint64_t h = is_custom ? fnv(host_perm.data(), c.T) : 0;
+  for (auto& e : ds->tables)
+    if (memcmp(&e.key, &c, sizeof c) == 0 && e.custom_hash == h) { e.stamp = ++g_stamp; *out = e.dev; return SP_OK; }
+  if (ds->tables.size() >= kMaxTables) {
+    size_t lru = 0;
+    for (size_t i = 1; i < ds->tables.size(); ++i) if (ds->tables[i].stamp < ds->tables[lru].stamp) lru = i;
+    cudaFree(ds->tables[lru].dev);  // synchronises: no kernel can still be reading it afterwards
+    ds->tables.erase(ds->tables.begin() + (long)lru);
+  }
+  TableEntry e;
+  e.key = c; e.custom_hash = h; e.stamp = ++g_stamp; e.dev = nullptr;
+  SP_CUDA(cudaMalloc(&e.dev, sizeof(int32_t) * (size_t)c.T));
+  if (is_custom) {
+    // pageable source: the copy has been staged when the call returns, so host_perm may die
+    cudaError_t ce = cudaMemcpyAsync(e.dev, host_perm.data(), sizeof(int32_t) * (size_t)c.T, cudaMemcpyHostToDevice, stream);
+    if (ce == cudaSuccess) ce = cudaStreamSynchronize(stream);
+    if (ce != cudaSuccess) { cudaFree(e.dev); set_error("table upload failed: %s", cudaGetErrorString(ce)); return SP_ERR_CUDA; }
+  } else {
+    cudaError_t ce = launch_build_perm(c, e.dev, stream);
+    if (ce != cudaSuccess) { cudaFree(e.dev); set_error("table build failed: %s", cudaGetErrorString(ce)); return SP_ERR_CUDA; }
+  }
+  ds->tables.push_back(e);
+  *out = e.dev;
+  return SP_OK;
+}
+
+static int gemm_common(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t K, int scheme,
+                       const sp_params* params, void* stream, sp_trace_rec* trace, bool want_trace) {
+  if (!A || !B || !C) { set_error("A, B and C must not be NULL"); return SP_ERR_INVALID_ARG; }
+  if (want_trace && !trace) { set_error("trace buffer must not be NULL"); return SP_ERR_INVALID_ARG; }
+  if (M <= 0 || N <= 0 || K <= 0) { set_error("M, N, K must be positive"); return SP_ERR_INVALID_ARG; }
+  if (M >= (1ll << 31) || N >= (1ll << 31) || K >= (1ll << 31)) { set_error("dimension too large"); return SP_ERR_UNSUPPORTED; }
+  if (params && params->struct_size != sizeof(sp_params)) {
+    set_error("sp_params.struct_size is %u, expected %zu", params->struct_size, sizeof(sp_params));
+    return SP_ERR_INVALID_ARG;
+  }
+  int tile_m = params ? params->tile_m : 0, tile_n = params ? params->tile_n : 0;
+  if (tile_m == 0 && tile_n == 0) { tile_m = 256; tile_n = 256; }
+  if (!((tile_m == 128 || tile_m == 256) && (tile_n == 128 || tile_n == 256))) {
+    set_error("unsupported tile %dx%d (supported: 128x128, 128x256, 256x128, 256x256)", tile_m, tile_n);
+    return SP_ERR_UNSUPPORTED;
+  }
+  const int out_f32 = params ? params->out_dtype : 0;
+  const int b_nk = params ? params->b_layout : 0;
+  if ((out_f32 != 0 && out_f32 != 1) || (b_nk != 0 && b_nk != 1)) { set_error("bad out_dtype / b_layout"); return SP_ERR_INVALID_ARG; }
+  if (((uintptr_t)A | (uintptr_t)B | (uintptr_t)C) & 15u) { set_error("A, B, C must be 16-byte aligned"); return SP_ERR_ALIGNMENT; }
+  if ((K % 8) != 0 || (N % 8) != 0) { set_error("K and N must be multiples of 8 (16-byte row pitch)"); return SP_ERR_ALIGNMENT; }
+
+  GemmCall call;
+  memset(&call, 0, sizeof call);
+  int rc = resolve_sched(M, N, tile_m, tile_n, scheme, params, &call.sched);
+  if (rc != SP_OK) return rc;
+  std::vector<int32_t> host_perm;
+  rc = build_perm_host(call.sched, params ? params->custom_perm : nullptr, host_perm);  // bijectivity gate
+  if (rc != SP_OK) return rc;
+
+  int dev = 0;
+  rc = current_device(&dev);
+  if (rc != SP_OK) return rc;
+  std::lock_guard<std::mutex> lock(g_mu);
+  DeviceState* ds = device_state(dev);
+  rc = get_status_word(ds);
+  if (rc != SP_OK) return rc;
+  call.A = A; call.B = B; call.C = C; call.M = M; call.N = N; call.K = K;
+  call.tile_m = tile_m; call.tile_n = tile_n; call.out_f32 = out_f32; call.b_nk = b_nk;
+  call.status_dev = ds->status;
+  call.trace_dev = want_trace ? trace : nullptr;
+  call.stream = (cudaStream_t)stream;
+  call.perm_dev = nullptr;
+  if (call.sched.use_table) {
+    rc = get_table(ds, call.sched, host_perm, scheme == kCustom, call.stream, &call.perm_dev);
+    if (rc != SP_OK) return rc;
+  }
+  return launch_gemm(call);
+}
+
+}  // namespace sp
+
+using namespace sp;
+
+extern "C" {
+
+int64_t sp_tile_count(int64_t M, int64_t N, int32_t tileM, int32_t tileN) {
+  if (M <= 0 || N <= 0 || tileM <= 0 || tileN <= 0) return -1;
+  return ((M + tileM - 1) / tileM) * ((N + tileN - 1) / tileN);
+}
+
+int sp_tile_map(int64_t M, int64_t N, int32_t tileM, int32_t tileN, int scheme, const sp_params* params,
+                int32_t* out_perm) {
+  if (!out_perm) { set_error("out_perm must not be NULL"); return SP_ERR_INVALID_ARG; }
+  Sched c;
+  int rc = resolve_sched(M, N, tileM, tileN, scheme, params, &c);
+  if (rc != SP_OK) return rc;
+  std::vector<int32_t> perm;
+  rc = build_perm_host(c, params ? params->custom_perm : nullptr, perm);
+  if (rc != SP_OK) return rc;
+  memcpy(out_perm, perm.data(), sizeof(int32_t) * perm.size());
+  return SP_OK;
+}
+
+int sp_tile_map_device(int64_t M, int64_t N, int32_t tileM, int32_t tileN, int scheme, const sp_params* params,
+                       int32_t* out_perm_dev, void* stream) {
+  if (!out_perm_dev) { set_error("out_perm_dev must not be NULL"); return SP_ERR_INVALID_ARG; }
+  Sched c;
+  int rc = resolve_sched(M, N, tileM, tileN, scheme, params, &c);
+  if (rc != SP_OK) return rc;
+  std::vector<int32_t> perm;
+  rc = build_perm_host(c, params ? params->custom_perm : nullptr, perm);
+  if (rc != SP_OK) return rc;
+  int dev = 0;
+  rc = current_device(&dev);
+  if (rc != SP_OK) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (scheme == kCustom) {
+    SP_CUDA(cudaMemcpyAsync(out_perm_dev, perm.data(), sizeof(int32_t) * perm.size(), cudaMemcpyHostToDevice, st));
+    SP_CUDA(cudaStreamSynchronize(st));
+    return SP_OK;
+  }
+  SP_CUDA(launch_build_perm(c, out_perm_dev, st));
+  return SP_OK;
+}
+
+int sp_gemm(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t K, int scheme,
+            const sp_params* params, void* stream) {
+  return gemm_common(A, B, C, M, N, K, scheme, params, stream, nullptr, false);
+}
+
+int sp_gemm_trace(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t K, int scheme,
+                  const sp_params* params, void* stream, sp_trace_rec* trace_dev) {
+  return gemm_common(A, B, C, M, N, K, scheme, params, stream, trace_dev, true);
+}
+
+int sp_gemm_units(int32_t tile_m, int32_t tile_n, int64_t T) {
+  int dev = 0;
+  if (current_device(&dev) != SP_OK) return -1;
+  return gemm_units(tile_m, tile_n, T);
+}
+
+int sp_probe_dispatch(int32_t n_blocks, int32_t cluster, int32_t* smid_host, uint64_t* start_host) {
+  if (n_blocks <= 0 || n_blocks > (1 << 20) || (cluster != 1 && cluster != 2) || (n_blocks % cluster) != 0 ||
+      !smid_host || !start_host) {
+    set_error("bad probe arguments");
+    return SP_ERR_INVALID_ARG;
+  }
+  int dev = 0;
+  int rc = current_device(&dev);
+  if (rc != SP_OK) return rc;
+  return probe_dispatch(n_blocks, cluster, smid_host, start_host);
+}
+
+int sp_get_status(void* stream, int32_t* detail) {
+  int dev = 0;
+  int rc = current_device(&dev);
+  if (rc != SP_OK) return rc;
+  SP_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+  std::lock_guard<std::mutex> lock(g_mu);
+  DeviceState* ds = device_state(dev);
+  int32_t word = 0;
+  if (ds->status) {
+    SP_CUDA(cudaMemcpy(&word, ds->status, sizeof word, cudaMemcpyDeviceToHost));
+    if (word != 0) SP_CUDA(cudaMemset(ds->status, 0, sizeof word));
+  }
+  if (detail) *detail = word;
+  if (word != 0) { set_error("a device-side wait expired (status word 0x%x)", word); return SP_ERR_TIMEOUT; }
+  return SP_OK;
+}
+
+const char* sp_last_error(void) { return g_err; }
+
+void sp_shutdown(void) {
+  std::lock_guard<std::mutex> lock(g_mu);
+  int prev = 0;
+  const bool have = cudaGetDevice(&prev) == cudaSuccess;
+  for (auto& d : g_devs) {
+    if (cudaSetDevice(d.device) != cudaSuccess) continue;
+    for (auto& e : d.tables) cudaFree(e.dev);
+    d.tables.clear();
+    if (d.status) cudaFree(d.status);
+    d.status = nullptr;
+  }
+  g_devs.clear();
+  if (have) cudaSetDevice(prev);
+  cudaGetLastError();
+}
+
+}  // extern "C"

@@ -1,0 +1,573 @@
+// Persistent, warp-specialised bf16 GEMM for sm_100a whose tile order is a remap of slot ids
+// (the paper's swizzle: each block recomputes which output tile it works on).
+//
+// One persistent unit = one CTA (tile 128 x BN) or a CTA pair (tile 256 x BN, cta_group::2).
+// Unit u runs slots u, u + units, u + 2*units, ...; slot s computes tile slot_to_tile(s).
+//
+// Warp roles (192 threads):
+//   warp 0  lane 0 : TMA producer   -- A and B k-blocks into a ring of 128B-swizzled smem stages
+//   warp 1  lane 0 : MMA issuer     -- tcgen05.mma, fp32 accumulators in TMEM (two buffers);
+//                                      the warp also owns TMEM alloc / dealloc
+//   warps 2..5     : epilogue       -- tcgen05.ld, convert, 16-byte global stores, ragged-edge predication
+//
+// Synchronisation: mbarriers only.  full[s]/empty[s] per smem stage, tmem_full[b]/tmem_empty[b]
+// per accumulator buffer.  In pair mode the barriers that feed the MMA issuer live in the
+// leader CTA (cluster rank 0); tcgen05.commit multicasts its arrivals to both CTAs.
+// Every wait is bounded: after kTimeoutNs, or once another role has given up, the role
+// records a code in the status word and leaves; teardown always runs and frees TMEM.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdio.h>
+#include <stdlib.h>
+
+#include <mutex>
+
+#include "internal.h"
+
+namespace sp {
+
+constexpr int kBK = 64;          // k extent of one stage: 64 bf16 = one 128-byte swizzle row
+constexpr int kUmmaK = 16;       // k extent of one tcgen05.mma with 16-bit inputs
+constexpr int kThreads = 192;
+constexpr uint32_t kSmemLimit = 232448;  // 227 KiB opt-in maximum per CTA
+constexpr uint32_t kBarrierBytes = 1024;
+constexpr unsigned long long kTimeoutNs = 2000000000ull;
+constexpr int kTmemCols = 512;
+
+template <int CG, int BN>
+struct Cfg {
+  static constexpr int kBCols = BN / CG;                        // columns of B held by one CTA
+  static constexpr uint32_t kABytes = 128 * kBK * 2;            // 128 rows of A
+  static constexpr uint32_t kBBytes = kBCols * kBK * 2;
+  static constexpr uint32_t kStageBytes = kABytes + kBBytes;
+  static constexpr int kFit = (kSmemLimit - kBarrierBytes - 1024) / kStageBytes;
+  static constexpr int kStages = kFit > 8 ? 8 : kFit;
+  static constexpr uint32_t kSmemBytes = kStages * kStageBytes + kBarrierBytes + 1024;  // + alignment slack
+};
+
+struct GemmArgs {
+  void* C;
+  const int32_t* perm;
+  int32_t* status;
+  sp_trace_rec* trace;
+  int M, N, K;
+  int kblocks;
+  int units;
+  uint32_t b_lbo, b_sbo, b_kstep;  // B operand descriptor strides in bytes
+  Sched sched;
+};
+
+// status word: (role << 8) | which wait
+enum : int { kRoleProducer = 1, kRoleMma = 2, kRoleEpilogue = 3 };
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ unsigned long long globaltimer() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+
+// Arrive on a barrier given by its cluster-window address (own or peer CTA).
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+
+__device__ __forceinline__ uint32_t mapa(uint32_t addr, uint32_t rank) {
+  uint32_t out;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(out) : "r"(addr), "r"(rank));
+  return out;
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+// Bounded wait.  Returns false after kTimeoutNs or once the status word is set by anyone.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, int32_t* status, int code) {
+  const unsigned long long t0 = globaltimer();
+  for (uint32_t i = 1;; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 63u) == 0) {
+      if (*(volatile int32_t*)status != 0) return false;
+      if (globaltimer() - t0 > kTimeoutNs) {
+        atomicCAS(status, 0, code);
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t* status, int code) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, status, code);
+}
+
+template <int CG>
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  if constexpr (CG == 1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+  } else {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.cta_group::2 "
+        "[%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+  }
+}
+
+__device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+template <int CG>
+__device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t cols) {
+  if constexpr (CG == 1)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(cols) : "memory");
+  else
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(cols) : "memory");
+}
+
+template <int CG>
+__device__ __forceinline__ void tmem_relinquish() {
+  if constexpr (CG == 1) asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  else asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+
+template <int CG>
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  if constexpr (CG == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+  else asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+
+template <int CG>
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  if constexpr (CG == 1) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  }
+}
+
+// Arrive on `bar` (same smem offset in every CTA of the group) once all MMAs issued so far by this thread are done.
+template <int CG>
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  if constexpr (CG == 1) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+  } else {
+    const uint16_t mask = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(mask)
+                 : "memory");
+  }
+}
+
+__device__ __forceinline__ void tmem_ld_32x32b_x32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+template <int CG>
+__device__ __forceinline__ void unit_sync() {
+  if constexpr (CG == 1) {
+    __syncthreads();
+  } else {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+  }
+}
+
+// Shared-memory operand descriptor (tcgen05): start address, leading / stride byte offsets
+// (all in 16-byte units), descriptor version 1, 128-byte swizzle.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
+         ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
+}
+
+// Instruction descriptor, kind::f16: D fp32, A and B bf16, A K-major, B K- or MN-major.
+__host__ __device__ constexpr uint32_t make_idesc(int m, int n, bool b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) |
+         ((uint32_t)(m >> 4) << 24);
+}
+
+__device__ __forceinline__ int tile_of_slot(const GemmArgs& a, int s) {
+  return a.sched.use_table ? __ldg(a.perm + s) : slot_to_tile(a.sched, s);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(uint32_t lo_bits, uint32_t hi_bits) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(lo_bits), __uint_as_float(hi_bits));
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+// ------------------------------------------------------------------ the kernel
+template <int CG, int BN, bool B_NK, bool OUT_F32>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmArgs args) {
+  using C = Cfg<CG, BN>;
+  constexpr int S = C::kStages;
+  constexpr int TILE_M = 128 * CG;
+
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t bar_base = smem_base + S * C::kStageBytes;
+  const uint32_t bar_full = bar_base;              // S barriers
+  const uint32_t bar_empty = bar_base + 8 * S;     // S barriers
+  const uint32_t bar_tfull = bar_base + 16 * S;    // 2 barriers
+  const uint32_t bar_tempty = bar_tfull + 16;      // 2 barriers
+  const uint32_t tmem_slot = bar_tempty + 16;      // 4 bytes
+  volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = CG == 1 ? 0u : cluster_ctarank();
+  const int unit = blockIdx.x / CG;
+  const int T = args.sched.T, Tn = args.sched.Tn;
+  const int KB = args.kblocks;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < S; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_empty + 8 * i, 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_tfull + 8 * i, 1); mbar_init(bar_tempty + 8 * i, 4 * CG); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    tmem_alloc<CG>(tmem_slot, kTmemCols);
+    tmem_relinquish<CG>();
+  }
+  tcgen05_fence_before();
+  unit_sync<CG>();
+  tcgen05_fence_after();
+  const uint32_t tmem_base = *tmem_slot_ptr;
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int s = unit; s < T && ok; s += args.units) {
+        const int t = tile_of_slot(args, s);
+        const int tm = t / Tn, tn = t - tm * Tn;
+        const int row0 = tm * TILE_M + (int)rank * 128;
+        const int col0 = tn * BN + (int)rank * C::kBCols;
+        if (args.trace && rank == 0) {
+          sp_trace_rec* rec = args.trace + s;
+          uint32_t smid;
+          asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+          rec->slot = s; rec->tile = t; rec->smid = (int)smid; rec->unit = unit; rec->t_begin = globaltimer();
+        }
+        for (int kb = 0; kb < KB; ++kb) {
+          ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, args.status, (kRoleProducer << 8) | 1);
+          if (!ok) break;
+          const uint32_t full_local = bar_full + 8 * stage;
+          const uint32_t full_leader = CG == 1 ? full_local : mapa(full_local, 0);
+          if (rank == 0) mbar_arrive_expect_tx(full_local, CG * C::kStageBytes);
+          const uint32_t sa = smem_base + stage * C::kStageBytes;
+          const uint32_t sb = sa + C::kABytes;
+          tma_load_2d<CG>(sa, &tmA, kb * kBK, row0, full_leader);
+          if constexpr (B_NK) {
+            tma_load_2d<CG>(sb, &tmB, kb * kBK, col0, full_leader);
+          } else {
+#pragma unroll
+            for (int j = 0; j < C::kBCols / 64; ++j)
+              tma_load_2d<CG>(sb + j * (64 * kBK * 2), &tmB, col0 + j * 64, kb * kBK, full_leader);
+          }
+          if (++stage == S) { stage = 0; phase ^= 1u; }
+        }
+      }
+      // tail: every stage handed out must have been released, so that no commit arrival
+      // (or, after a failure, no copy) is still in flight towards this CTA when it exits
+      for (int i = 0; i < S && ok; ++i) {
+        ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, args.status, (kRoleProducer << 8) | 2);
+        if (++stage == S) { stage = 0; phase ^= 1u; }
+      }
+      if (!ok) {
+        const unsigned long long t0 = globaltimer();
+        while (globaltimer() - t0 < 1000000ull) __nanosleep(1000);  // let copies in flight land
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer (leader CTA only)
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = make_idesc(TILE_M, BN, !B_NK);
+      int stage = 0;
+      uint32_t phase = 0;
+      int it = 0;
+      bool ok = true;
+      for (int s = unit; s < T && ok; s += args.units, ++it) {
+        const int buf = it & 1;
+        const uint32_t use = (uint32_t)(it >> 1) & 1u;
+        ok = mbar_wait(bar_tempty + 8 * buf, use ^ 1u, args.status, (kRoleMma << 8) | 1);
+        if (!ok) break;
+        tcgen05_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+        for (int kb = 0; kb < KB; ++kb) {
+          ok = mbar_wait(bar_full + 8 * stage, phase, args.status, (kRoleMma << 8) | 2);
+          if (!ok) break;
+          tcgen05_fence_after();
+          const uint32_t sa = smem_base + stage * C::kStageBytes;
+          const uint32_t sb = sa + C::kABytes;
+#pragma unroll
+          for (int k = 0; k < kBK / kUmmaK; ++k) {
+            const uint64_t da = smem_desc(sa + k * (kUmmaK * 2), 16, 1024);
+            const uint64_t db = smem_desc(sb + k * args.b_kstep, args.b_lbo, args.b_sbo);
+            umma_bf16<CG>(d_tmem, da, db, idesc, (uint32_t)((kb | k) != 0));
+          }
+          umma_commit<CG>(bar_empty + 8 * stage);
+          if (++stage == S) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) umma_commit<CG>(bar_tfull + 8 * buf);
+      }
+    }
+    __syncwarp();
+  } else {
+    // ---------------------------------------------------------------- epilogue
+    const int quarter = warp & 3;  // TMEM lanes [32*quarter, 32*quarter + 32) are this warp's
+    int it = 0;
+    bool ok = true;
+    for (int s = unit; s < T && ok; s += args.units, ++it) {
+      const int t = tile_of_slot(args, s);
+      const int tm = t / Tn, tn = t - tm * Tn;
+      const int buf = it & 1;
+      const uint32_t use = (uint32_t)(it >> 1) & 1u;
+      ok = mbar_wait(bar_tfull + 8 * buf, use, args.status, (kRoleEpilogue << 8) | 1);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tcgen05_fence_after();
+      const int row = tm * TILE_M + (int)rank * 128 + quarter * 32 + lane;
+      const int col_base = tn * BN;
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN);
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        uint32_t v[32];
+        tmem_ld_32x32b_x32(taddr + (uint32_t)(c * 32), v);
+        tmem_ld_wait();
+        const int col = col_base + c * 32;
+        if (row < args.M && col < args.N) {
+          if constexpr (OUT_F32) {
+            float* dst = reinterpret_cast<float*>(args.C) + (size_t)row * (size_t)args.N + col;
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              if (col + 4 * j < args.N)
+                *reinterpret_cast<uint4*>(dst + 4 * j) = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+          } else {
+            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(args.C) + (size_t)row * (size_t)args.N + col;
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              if (col + 8 * j < args.N)
+                *reinterpret_cast<uint4*>(dst + 8 * j) =
+                    make_uint4(pack_bf16(v[8 * j], v[8 * j + 1]), pack_bf16(v[8 * j + 2], v[8 * j + 3]),
+                               pack_bf16(v[8 * j + 4], v[8 * j + 5]), pack_bf16(v[8 * j + 6], v[8 * j + 7]));
+          }
+        }
+      }
+      tcgen05_fence_before();
+      __syncwarp();
+      if (lane == 0) {
+        const uint32_t te = bar_tempty + 8 * buf;
+        mbar_arrive_cluster(CG == 1 ? te : mapa(te, 0));
+        if (args.trace && rank == 0 && warp == 2) args.trace[s].t_end = globaltimer();
+      }
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tcgen05_fence_before();
+  unit_sync<CG>();
+  if (warp == 1) tmem_dealloc<CG>(tmem_base, kTmemCols);
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+  });
+  return fn;
+}
+
+// bf16 row-major [rows, cols] matrix, box = box_rows x 64 elements, 128-byte swizzle.
+static int make_map(CUtensorMap* m, const void* base, int64_t rows, int64_t cols, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) { set_error("cuTensorMapEncodeTiled is not available from the driver"); return SP_ERR_CUDA; }
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled failed (CUresult %d)", (int)r); return SP_ERR_CUDA; }
+  return SP_OK;
+}
+
+// Co-resident persistent units for one tile shape: one CTA per SM, or as many CTA pairs as the
+// device can hold at once (asked of the occupancy calculator, cached per shape).
+template <int CG, int BN>
+static int max_units() {
+  static int cached = 0;
+  if (cached > 0) return cached;
+  using C = Cfg<CG, BN>;
+  auto kern = gemm_kernel<CG, BN, false, false>;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return -1;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return -1;
+  int units = sms / CG;
+  if (CG == 2) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemBytes) != cudaSuccess) return -1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(sms / CG * CG));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = C::kSmemBytes;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CG; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) == cudaSuccess && n > 0 && n < units) units = n;
+    cudaGetLastError();
+  }
+  cached = units;
+  return units;
+}
+
+int gemm_units(int tile_m, int tile_n, int64_t T) {
+  int64_t units = tile_m == 256 ? (tile_n == 128 ? max_units<2, 128>() : max_units<2, 256>())
+                                : (tile_n == 128 ? max_units<1, 128>() : max_units<1, 256>());
+  if (units <= 0) return -1;
+  if (const char* e = getenv("SP_MAX_UNITS")) {  // experiments only: cap the number of persistent units
+    const int64_t cap = atoll(e);
+    if (cap > 0 && cap < units) units = cap;
+  }
+  if (units > T) units = T;
+  return (int)units;
+}
+
+template <int CG, int BN, bool B_NK, bool OUT_F32>
+static int launch_variant(const GemmCall& call, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArgs& args) {
+  using C = Cfg<CG, BN>;
+  auto kern = gemm_kernel<CG, BN, B_NK, OUT_F32>;
+  static bool configured = false;  // per instantiation; attribute is per device but identical everywhere
+  cudaError_t e = cudaSuccess;
+  if (!configured) {
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemBytes);
+    if (e != cudaSuccess) { set_error("cudaFuncSetAttribute(smem=%u) failed: %s", C::kSmemBytes, cudaGetErrorString(e)); return SP_ERR_CUDA; }
+    configured = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(args.units * CG));
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = C::kSmemBytes;
+  cfg.stream = call.stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = CG;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  e = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, args);
+  if (e != cudaSuccess) { set_error("kernel launch failed: %s", cudaGetErrorString(e)); return SP_ERR_CUDA; }
+  return SP_OK;
+}
+
+template <int CG, int BN>
+static int launch_shape(const GemmCall& call, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArgs& args) {
+  if (call.b_nk) {
+    return call.out_f32 ? launch_variant<CG, BN, true, true>(call, tmA, tmB, args)
+                        : launch_variant<CG, BN, true, false>(call, tmA, tmB, args);
+  }
+  return call.out_f32 ? launch_variant<CG, BN, false, true>(call, tmA, tmB, args)
+                      : launch_variant<CG, BN, false, false>(call, tmA, tmB, args);
+}
+
+int launch_gemm(const GemmCall& call) {
+  const int cg = call.tile_m / 128;
+  const int bcols = call.tile_n / cg;  // B columns per CTA
+  CUtensorMap tmA, tmB;
+  int rc = make_map(&tmA, call.A, call.M, call.K, 128);
+  if (rc != SP_OK) return rc;
+  if (call.b_nk) rc = make_map(&tmB, call.B, call.N, call.K, bcols);   // N x K, K contiguous: one box of bcols rows
+  else rc = make_map(&tmB, call.B, call.K, call.N, 64);                // K x N, N contiguous: boxes of 64 k x 64 n
+  if (rc != SP_OK) return rc;
+
+  GemmArgs args;
+  args.C = call.C;
+  args.perm = call.perm_dev;
+  args.status = call.status_dev;
+  args.trace = call.trace_dev;
+  args.M = (int)call.M; args.N = (int)call.N; args.K = (int)call.K;
+  args.kblocks = (int)((call.K + kBK - 1) / kBK);
+  args.units = gemm_units(call.tile_m, call.tile_n, call.sched.T);
+  if (args.units <= 0) { set_error("could not size the grid"); return SP_ERR_CUDA; }
+  if (call.b_nk) {
+    // K-major B: rows of 128 bytes, 8-row groups 1024 bytes apart; k advances inside the swizzle row
+    args.b_lbo = 16; args.b_sbo = 1024; args.b_kstep = kUmmaK * 2;
+  } else {
+    // MN-major B: a box is 64 k-rows of 128 bytes (64 n); groups of 8 k-rows are 1024 bytes apart
+    // (stride offset); the next 64 n live in the next box, 8192 bytes on (leading offset)
+    args.b_lbo = 64 * kBK * 2; args.b_sbo = 1024; args.b_kstep = kUmmaK * 128;
+  }
+  if (const char* e = getenv("SP_DEBUG_BDESC")) {  // bring-up only: "lbo,sbo,kstep" in bytes
+    unsigned l = 0, s = 0, k = 0;
+    if (sscanf(e, "%u,%u,%u", &l, &s, &k) == 3) { args.b_lbo = l; args.b_sbo = s; args.b_kstep = k; }
+  }
+  args.sched = call.sched;
+
+  if (cg == 1) return call.tile_n == 128 ? launch_shape<1, 128>(call, tmA, tmB, args) : launch_shape<1, 256>(call, tmA, tmB, args);
+  return call.tile_n == 128 ? launch_shape<2, 128>(call, tmA, tmB, args) : launch_shape<2, 256>(call, tmA, tmB, args);
+}
+
+}  // namespace sp

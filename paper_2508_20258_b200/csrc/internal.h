@@ -1,0 +1,52 @@
+// Internal declarations shared by the translation units of libswizzleperf.so.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "../../include/swizzleperf.h"
+#include "remap.cuh"
+
+namespace sp {
+
+// Largest tile count any entry point accepts, and largest grid side for curve orders
+// (their enclosing square has 4^k cells, all of which are visited once).
+constexpr int64_t kMaxTiles = 1 << 24;
+constexpr int kMaxCurveSide = 4096;
+
+void set_error(const char* fmt, ...);
+
+// Validates sizes and parameters and fills `out`.  Returns an sp_status.
+int resolve_sched(int64_t M, int64_t N, int32_t tileM, int32_t tileN, int scheme, const sp_params* params, Sched* out);
+
+// Evaluates the remap on the host (closed forms, curve walks, caller table) and checks
+// that it is a bijection.  Returns SP_OK or SP_ERR_NOT_BIJECTIVE / SP_ERR_INVALID_ARG.
+int build_perm_host(const Sched& sched, const int32_t* custom, std::vector<int32_t>& perm);
+
+// Device evaluation of the same remap into out_dev (T entries).  Not valid for kCustom.
+cudaError_t launch_build_perm(const Sched& sched, int32_t* out_dev, cudaStream_t stream);
+
+struct GemmCall {
+  const void* A;
+  const void* B;
+  void* C;
+  int64_t M, N, K;
+  int tile_m, tile_n;
+  int out_f32;
+  int b_nk;
+  Sched sched;
+  const int32_t* perm_dev;  // table for non-arithmetic schemes, else nullptr
+  int32_t* status_dev;
+  sp_trace_rec* trace_dev;  // nullptr unless tracing
+  cudaStream_t stream;
+};
+
+// Number of persistent units (CTAs or CTA pairs) for this tile shape on the current device.
+int gemm_units(int tile_m, int tile_n, int64_t T);
+// Encodes tensor maps and launches the kernel.  Returns an sp_status.
+int launch_gemm(const GemmCall& call);
+
+int probe_dispatch(int n_blocks, int cluster, int32_t* smid_host, uint64_t* start_host);
+
+}  // namespace sp

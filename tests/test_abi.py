@@ -1,0 +1,55 @@
+"""The shared library loads without a GPU and exports every symbol the header declares."""
+
+import ctypes
+import os
+import re
+
+import numpy as np
+
+import paper_2508_20258_b200 as sp
+from paper_2508_20258_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "swizzleperf.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(sp_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported():
+    names = _declared()
+    assert set(names) == set(binding.EXPORTS)
+    L = ctypes.CDLL(binding.LIB_PATH)
+    for n in names:
+        assert getattr(L, n) is not None
+
+
+def test_struct_layout_matches_header():
+    assert ctypes.sizeof(binding.SpParams) == 72
+    assert ctypes.sizeof(binding.SpTraceRec) == 32 and binding.TRACE_DTYPE.itemsize == 32
+    assert binding.SpParams.custom_perm.offset == 40 and binding.SpParams.tile_m.offset == 48
+
+
+def test_gemm_rejects_bad_arguments_before_touching_a_device():
+    L = sp.lib()
+    p = sp.make_params(tile_m=128, tile_n=128)
+    a = 0x1000  # never dereferenced: every check below fails on the host first
+    assert L.sp_gemm(None, a, a, 128, 128, 128, sp.ROW_MAJOR, ctypes.byref(p), None) == sp.ERR_INVALID_ARG
+    assert L.sp_gemm(a, a, a, 0, 128, 128, sp.ROW_MAJOR, ctypes.byref(p), None) == sp.ERR_INVALID_ARG
+    assert L.sp_gemm(a + 8, a, a, 128, 128, 128, sp.ROW_MAJOR, ctypes.byref(p), None) == sp.ERR_ALIGNMENT
+    assert L.sp_gemm(a, a, a, 128, 128, 100, sp.ROW_MAJOR, ctypes.byref(p), None) == sp.ERR_ALIGNMENT
+    assert L.sp_gemm(a, a, a, 128, 124, 128, sp.ROW_MAJOR, ctypes.byref(p), None) == sp.ERR_ALIGNMENT
+    q = sp.make_params(tile_m=64, tile_n=128)
+    assert L.sp_gemm(a, a, a, 128, 128, 128, sp.ROW_MAJOR, ctypes.byref(q), None) == sp.ERR_UNSUPPORTED
+    q = sp.make_params(tile_m=128, tile_n=128, custom_perm=[0, 0])
+    assert L.sp_gemm(a, a, a, 128, 256, 128, sp.CUSTOM, ctypes.byref(q), None) == sp.ERR_NOT_BIJECTIVE
+    q = sp.make_params(tile_m=128, tile_n=128, num_xcds=4)
+    assert L.sp_gemm(a, a, a, 256, 640, 128, sp.XCD, ctypes.byref(q), None) == sp.ERR_NOT_BIJECTIVE
+    q = sp.make_params(tile_m=128, tile_n=128, group=0)
+    assert L.sp_gemm(a, a, a, 256, 640, 128, sp.GROUP_M, ctypes.byref(q), None) == sp.ERR_INVALID_ARG
+    assert L.sp_gemm_trace(a, a, a, 128, 128, 128, sp.ROW_MAJOR, ctypes.byref(p), None, None) == sp.ERR_INVALID_ARG
+    assert sp.last_error() != ""
+    smid = np.zeros(4, dtype=np.int32)
+    assert L.sp_probe_dispatch(3, 2, smid.ctypes.data, smid.ctypes.data) == sp.ERR_INVALID_ARG

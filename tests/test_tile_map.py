@@ -1,0 +1,125 @@
+"""Host remap (closed forms in the library) against the enumerating oracle: bit-exact."""
+
+import ctypes
+
+import numpy as np
+import pytest
+from hypothesis import given, settings, strategies as st
+
+import paper_2508_20258_b200 as sp
+from oracle import remap as R
+
+
+def _lib_map(Tm, Tn, scheme, **kw):
+    return sp.tile_map(Tm * 128, Tn * 64, 128, 64, scheme, sp.make_params(**kw)).tolist()
+
+
+@given(Tm=st.integers(1, 150), Tn=st.integers(1, 150), G=st.integers(1, 200))
+@settings(max_examples=120, deadline=None)
+def test_plain_and_grouped_orders(Tm, Tn, G):
+    assert _lib_map(Tm, Tn, sp.ROW_MAJOR) == R.row_major(Tm, Tn)
+    assert _lib_map(Tm, Tn, sp.COL_MAJOR) == R.col_major(Tm, Tn)
+    assert _lib_map(Tm, Tn, sp.GROUP_M, group=G) == R.group_m(Tm, Tn, G)
+    assert _lib_map(Tm, Tn, sp.GROUP_N, group=G) == R.group_n(Tm, Tn, G)
+
+
+@given(Tm=st.integers(1, 70), Tn=st.integers(1, 70))
+@settings(max_examples=60, deadline=None)
+def test_curves(Tm, Tn):
+    assert _lib_map(Tm, Tn, sp.MORTON) == R.morton(Tm, Tn)
+    assert _lib_map(Tm, Tn, sp.HILBERT) == R.hilbert(Tm, Tn)
+
+
+@pytest.mark.parametrize("Tm,Tn", [(1, 1), (32, 32), (32, 16), (64, 8), (64, 64), (128, 8), (5, 100)])
+def test_curves_on_config_grids(Tm, Tn):
+    assert _lib_map(Tm, Tn, sp.MORTON) == R.morton(Tm, Tn)
+    assert _lib_map(Tm, Tn, sp.HILBERT) == R.hilbert(Tm, Tn)
+
+
+@given(T=st.integers(1, 3000), X=st.integers(1, 200), W=st.integers(0, 400), bal=st.booleans())
+@settings(max_examples=200, deadline=None)
+def test_xcd(T, X, W, bal):
+    try:
+        want = R.xcd(T, X, W, bal)
+    except R.NotBijective:
+        want = None
+    out = np.full(T, -7, dtype=np.int32)
+    p = sp.make_params(num_xcds=X, wave=W, xcd_balanced=int(bal))
+    rc = sp.lib().sp_tile_map(128, T * 128, 128, 128, sp.XCD, ctypes.byref(p), out.ctypes.data)
+    if want is None:
+        assert rc == sp.ERR_NOT_BIJECTIVE
+        assert (out == -7).all()          # untouched on rejection
+    else:
+        assert rc == sp.OK and out.tolist() == want
+
+
+@given(Tm=st.integers(1, 40), Tn=st.integers(1, 40), axis=st.integers(0, 1),
+       inner=st.sampled_from([R.ROW_MAJOR, R.COL_MAJOR, R.GROUP_M, R.GROUP_N, R.MORTON, R.HILBERT]),
+       G=st.integers(1, 9), inter=st.booleans())
+@settings(max_examples=200, deadline=None)
+def test_die_split(Tm, Tn, axis, inner, G, inter):
+    got = _lib_map(Tm, Tn, sp.DIE_SPLIT, split_axis=axis, inner_scheme=inner, inner_group=G, interleave=int(inter))
+    assert got == R.die_split(Tm, Tn, axis, inner, G, inter)
+
+
+def test_front_door_matches_oracle_on_the_five_workload_grids():
+    cases = [(512, 512, 128, 128), (4096, 4096, 128, 256), (8192, 8192, 256, 256), (16384, 2048, 256, 256),
+             (16384, 2048, 128, 256), (16384, 16384, 256, 256), (1000, 520, 128, 128)]
+    for (M, N, tm, tn) in cases:
+        for scheme, kw in [(sp.ROW_MAJOR, {}), (sp.COL_MAJOR, {}), (sp.GROUP_M, dict(group=8)),
+                           (sp.GROUP_N, dict(group=4)), (sp.MORTON, {}), (sp.HILBERT, {}),
+                           (sp.XCD, dict(num_xcds=2, wave=74, xcd_balanced=1)),
+                           (sp.DIE_SPLIT, dict(split_axis=0, inner_scheme=sp.HILBERT)),
+                           (sp.DIE_SPLIT, dict(split_axis=1, inner_scheme=sp.GROUP_M, inner_group=8, interleave=1))]:
+            got = sp.tile_map(M, N, tm, tn, scheme, sp.make_params(**kw)).tolist()
+            want = R.tile_map(M, N, tm, tn, scheme, R.Params(**kw))
+            assert got == want, (M, N, tm, tn, scheme, kw)
+
+
+def test_custom_tables():
+    good = [3, 1, 2, 0]
+    assert sp.tile_map(256, 256, 128, 128, sp.CUSTOM, sp.make_params(custom_perm=good)).tolist() == good
+    for bad in ([0, 0, 1, 2], [0, 1, 2, 4], [0, 1, 2, -1]):
+        with pytest.raises(sp.SpError) as e:
+            sp.tile_map(256, 256, 128, 128, sp.CUSTOM, sp.make_params(custom_perm=bad))
+        assert e.value.status == sp.ERR_NOT_BIJECTIVE
+
+
+def test_argument_errors():
+    L = sp.lib()
+    out = np.zeros(16, dtype=np.int32)
+    ok = sp.make_params(group=2)
+    assert L.sp_tile_map(0, 512, 128, 128, sp.ROW_MAJOR, None, out.ctypes.data) == sp.ERR_INVALID_ARG
+    assert L.sp_tile_map(512, 512, 128, 0, sp.ROW_MAJOR, None, out.ctypes.data) == sp.ERR_INVALID_ARG
+    assert L.sp_tile_map(512, 512, 128, 128, 99, None, out.ctypes.data) == sp.ERR_INVALID_ARG
+    assert L.sp_tile_map(512, 512, 128, 128, sp.GROUP_M, None, out.ctypes.data) == sp.ERR_INVALID_ARG
+    assert L.sp_tile_map(512, 512, 128, 128, sp.GROUP_M, ctypes.byref(ok), None) == sp.ERR_INVALID_ARG
+    for kw in (dict(group=0), ):
+        p = sp.make_params(**kw)
+        assert L.sp_tile_map(512, 512, 128, 128, sp.GROUP_M, ctypes.byref(p), out.ctypes.data) == sp.ERR_INVALID_ARG
+    p = sp.make_params(num_xcds=0)
+    assert L.sp_tile_map(512, 512, 128, 128, sp.XCD, ctypes.byref(p), out.ctypes.data) == sp.ERR_INVALID_ARG
+    p = sp.make_params(num_xcds=2, wave=-1)
+    assert L.sp_tile_map(512, 512, 128, 128, sp.XCD, ctypes.byref(p), out.ctypes.data) == sp.ERR_INVALID_ARG
+    p = sp.make_params(split_axis=2)
+    assert L.sp_tile_map(512, 512, 128, 128, sp.DIE_SPLIT, ctypes.byref(p), out.ctypes.data) == sp.ERR_INVALID_ARG
+    p = sp.make_params(inner_scheme=sp.XCD)
+    assert L.sp_tile_map(512, 512, 128, 128, sp.DIE_SPLIT, ctypes.byref(p), out.ctypes.data) == sp.ERR_INVALID_ARG
+    p = sp.make_params(group=2)
+    p.struct_size = 12
+    assert L.sp_tile_map(512, 512, 128, 128, sp.GROUP_M, ctypes.byref(p), out.ctypes.data) == sp.ERR_INVALID_ARG
+    assert "struct_size" in sp.last_error()
+    # more than 2^24 tiles
+    assert L.sp_tile_map(1 << 20, 1 << 20, 128, 128, sp.ROW_MAJOR, None, out.ctypes.data) == sp.ERR_INVALID_ARG
+    # curve on a grid too elongated for its enclosing square
+    assert L.sp_tile_map(128 * 5000, 128, 128, 128, sp.HILBERT, None, out.ctypes.data) == sp.ERR_UNSUPPORTED
+    assert sp.tile_count(512, 640, 128, 128) == 20 and sp.tile_count(1, 1, 128, 128) == 1
+    assert sp.tile_count(0, 5, 1, 1) == -1
+
+
+def test_paper_example_through_the_library():
+    got = sp.tile_map(4 * 128, 5 * 128, 128, 128, sp.XCD, sp.make_params(num_xcds=4)).tolist()
+    assert got == [0, 5, 10, 15, 1, 6, 11, 16, 2, 7, 12, 17, 3, 8, 13, 18, 4, 9, 14, 19]
+    with pytest.raises(sp.SpError) as e:      # 148 blocks over 8 chiplets: printed form leaves the range
+        sp.tile_map(128, 148 * 128, 128, 128, sp.XCD, sp.make_params(num_xcds=8))
+    assert e.value.status == sp.ERR_NOT_BIJECTIVE
