@@ -1,0 +1,331 @@
+#!/usr/bin/env python
+"""Benchmark of the swizzled tiled GEMM on B200.
+
+A step is one pass of the whole hot path (remap -> TMA producer -> tcgen05 mainloop ->
+epilogue, one kernel launch) over one synthetic GEMM.  The default workload is the
+8192^3 bf16 GEMM with 256x256 CTA-pair tiles, the configuration the throughput target is
+quoted on.  One JSON line is printed by rank 0.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+                  [--workload cfg1..cfg5] [--scheme SPEC] [--tile MxN] [--kernel-only] [--sweep]
+
+With N > 1 (under torchrun) every rank runs an independent replica of the same GEMM on
+its own GPU: the path has no exchange step, so no collective touches the data.
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2508_20258_b200 import benchutil, synth  # noqa: E402
+
+L2_BYTES = 126 * 2 ** 20
+
+# DRAM bytes per launch of the GEMM kernel from the ncu captures summarised under profiles/
+# (dram__bytes_read.sum + dram__bytes_write.sum), keyed by (workload, tile, scheme spec); None = not captured.
+NCU_DRAM_BYTES = {}
+
+
+def parse_scheme(spec: str):
+    """'group_m:8' -> (scheme id, keyword dict for make_params)."""
+    import paper_2508_20258_b200 as sp
+    a = spec.split(":")
+    name = a[0]
+    if name == "row_major":
+        return sp.ROW_MAJOR, {}
+    if name == "col_major":
+        return sp.COL_MAJOR, {}
+    if name == "group_m":
+        return sp.GROUP_M, dict(group=int(a[1]))
+    if name == "group_n":
+        return sp.GROUP_N, dict(group=int(a[1]))
+    if name == "morton":
+        return sp.MORTON, {}
+    if name == "hilbert":
+        return sp.HILBERT, {}
+    if name == "xcd":      # xcd:X[:W]  (balanced form)
+        return sp.XCD, dict(num_xcds=int(a[1]), wave=int(a[2]) if len(a) > 2 else 0, xcd_balanced=1)
+    if name == "die_split":  # die_split:{m|n}:inner[:G][:i]
+        inner = {"row_major": sp.ROW_MAJOR, "col_major": sp.COL_MAJOR, "group_m": sp.GROUP_M, "group_n": sp.GROUP_N,
+                 "morton": sp.MORTON, "hilbert": sp.HILBERT}[a[2]]
+        rest = a[3:]
+        inter = int("i" in rest)
+        g = [int(v) for v in rest if v.isdigit()]
+        return sp.DIE_SPLIT, dict(split_axis=int(a[1] == "n"), inner_scheme=inner, inner_group=g[0] if g else 1,
+                                  interleave=inter)
+    raise ValueError(f"unknown scheme spec {spec!r}")
+
+
+SWEEPS = {
+    "cfg1": ["row_major", "group_m:2"],
+    "cfg2": ["row_major", "group_m:4", "group_m:8", "group_m:16", "hilbert"],
+    "cfg3": ["row_major", "col_major", "group_m:2", "group_m:4", "group_m:8", "group_m:16", "group_n:2", "group_n:4",
+             "group_n:8", "group_n:16", "morton", "hilbert", "xcd:2:74", "xcd:2", "die_split:m:group_m:8",
+             "die_split:n:group_m:8", "die_split:m:hilbert", "die_split:n:hilbert", "die_split:m:group_m:8:i"],
+    "cfg4": [f"group_m:{g}" for g in (1, 2, 4, 8, 16, 32, 64)] + [f"group_n:{g}" for g in (1, 2, 4, 8)],
+    "cfg5": [f"group_m:{g}" for g in (1, 2, 4, 8, 16, 32)] + [f"group_n:{g}" for g in (2, 4, 8, 16, 32)] +
+            ["hilbert", "die_split:m:group_m:8", "die_split:m:hilbert", "die_split:m:group_m:8:i"],
+}
+DEFAULT_SCHEME = {"cfg1": "group_m:2", "cfg2": "group_m:8", "cfg3": "group_m:8", "cfg4": "group_n:2", "cfg5": "group_m:8"}
+
+
+def dist_env():
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+
+
+# ---------------------------------------------------------------------------------- reference arm
+def run_reference(args) -> int:
+    """Times the CPU oracle, as it stands, on a bounded sample of the same workload."""
+    rank, _, world = dist_env()
+    if rank != 0:
+        return 0
+    from oracle import gemm as G
+    w = synth.WORKLOADS[args.workload]
+    _, A, B = synth.make_workload(args.workload)
+    cores = G.threads()
+    t0 = time.perf_counter()
+    G.gemm_rows(A, B, np.arange(8))                                   # calibration, also builds the object
+    rate = 8 / max(time.perf_counter() - t0, 1e-6)                    # rows per second (includes panel widening)
+    budget = 150.0 / (args.steps + args.warmup)
+    rows = int(max(1, min(w.M // 16, rate * budget)))
+    band = np.arange(rows)
+    for _ in range(args.warmup):
+        G.gemm_rows(A, B, band)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        G.gemm_rows(A, B, band)
+    dt = time.perf_counter() - t0
+    tflops = 2.0 * rows * w.N * w.K * args.steps / dt / 1e12
+    sample = f"{rows} contiguous rows of C ({rows}x{w.N}x{w.K}) per step, of the {w.M}-row product"
+    line = {
+        "impl": "reference", "metric": "bf16 GEMM TFLOP/s", "value": tflops, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{w.name}: M={w.M} N={w.N} K={w.K} bf16 inputs, fp64 CPU oracle", "sample": sample},
+        "cpu_baseline": {"value": tflops, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": tflops, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+# ---------------------------------------------------------------------------------- our arm
+def time_steps(sp, dA, dB, dC, scheme, p, steps, stream):
+    import torch
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        sp.gemm(dA, dB, dC, scheme, p, stream)
+    e1.record(stream)
+    e1.synchronize()
+    return e0.elapsed_time(e1)
+
+
+def run_ours(args) -> int:
+    import torch
+    import paper_2508_20258_b200 as sp
+
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    sp.lib()  # fail loudly if the extension is missing
+
+    w = synth.WORKLOADS[args.workload]
+    tile_m, tile_n = (int(v) for v in args.tile.split("x")) if args.tile else (w.tile_m, w.tile_n)
+    out_f32 = int(w.out_dtype == "fp32")
+    _, A, B = synth.make_workload(args.workload)
+    dA = torch.from_numpy(A.view(np.int16)).cuda().view(torch.bfloat16)
+    dB = torch.from_numpy(B.view(np.int16)).cuda().view(torch.bfloat16)
+    dC = torch.empty((w.M, w.N), dtype=torch.float32 if out_f32 else torch.bfloat16, device="cuda")
+    stream = torch.cuda.current_stream()
+    flops = 2.0 * w.M * w.N * w.K
+    resident = A.nbytes + B.nbytes + dC.numel() * dC.element_size()
+
+    def params_for(spec):
+        scheme, kw = parse_scheme(spec)
+        return scheme, sp.make_params(tile_m=tile_m, tile_n=tile_n, out_dtype=out_f32, **kw)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    if args.sweep:
+        return run_sweep(args, sp, w, dA, dB, dC, params_for, flops, stream)
+
+    spec = args.scheme or DEFAULT_SCHEME[args.workload]
+    scheme, p = params_for(spec)
+    for _ in range(max(args.warmup, 3)):
+        sp.gemm(dA, dB, dC, scheme, p, stream)
+    torch.cuda.synchronize()
+    if args.kernel_only:                       # the command profilers wrap: nothing but the kernel
+        ms = time_steps(sp, dA, dB, dC, scheme, p, args.steps, stream)
+        sp.get_status()
+        print(json.dumps({"kernel_only": True, "workload": w.name, "scheme": spec, "tile": f"{tile_m}x{tile_n}",
+                          "ms_per_step": ms / args.steps, "tflops": flops * args.steps / ms / 1e9}), flush=True)
+        return 0
+
+    sampler = benchutil.ClockSampler(local_rank).start()
+    barrier()
+    t_host0 = time.perf_counter()
+    ms_total = time_steps(sp, dA, dB, dC, scheme, p, args.steps, stream)
+    torch.cuda.synchronize()
+    t_host1 = time.perf_counter()
+    barrier()
+    sampler.stop()
+    assert sp.get_status() == 0
+    agg = benchutil.aggregate(ms_total, flops * args.steps, world)
+    value = agg["units"] / agg["ms"] / 1e9                      # TFLOP/s, whole job
+    clocks = sampler.summary(t_host0, t_host1)
+
+    # burst protocol: isolated launches, best of 10 (how the pool's peak itself was measured)
+    burst_ms = min(time_steps(sp, dA, dB, dC, scheme, p, 1, stream) for _ in range(10))
+    row_scheme, row_p = params_for("row_major")
+    for _ in range(3):
+        sp.gemm(dA, dB, dC, row_scheme, row_p, stream)
+    row_ms = time_steps(sp, dA, dB, dC, row_scheme, row_p, args.steps, stream) / args.steps
+
+    # end to end through the C ABI with host buffers (pinned): H2D of A and B, kernel, D2H of C, every step
+    e2e = None
+    if not args.no_e2e:
+        hA = torch.from_numpy(A.view(np.int16)).pin_memory()
+        hB = torch.from_numpy(B.view(np.int16)).pin_memory()
+        hC = torch.empty((w.M, w.N), dtype=torch.float32 if out_f32 else torch.int16).pin_memory()
+        e2e_steps = max(1, min(args.steps, 5))
+        sp.gemm_host(hA, hB, hC, scheme, p, stream)
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            sp.gemm_host(hA, hB, hC, scheme, p, stream)        # synchronises before returning
+        e2e_ms = (time.perf_counter() - t0) * 1e3
+        barrier()
+        eagg = benchutil.aggregate(e2e_ms, flops * e2e_steps, world)
+        e2e = {"value": eagg["units"] / eagg["ms"] / 1e9, "unit": "TFLOP/s", "h2d_bytes_per_step": int(A.nbytes + B.nbytes),
+               "d2h_bytes_per_step": int(hC.numel() * hC.element_size()), "steps": e2e_steps,
+               "ms_per_step": eagg["ms"] / e2e_steps, "api": "sp_gemm_host (pinned host buffers)"}
+        del hA, hB, hC
+
+    peaks = benchutil.measured_peaks(ROOT)
+    launch_ms = ms_total / args.steps
+    achieved = flops / launch_ms / 1e9
+    roofline = {
+        "bound": "tensor", "kernel": f"gemm_kernel<CG={tile_m // 128},BN={tile_n}>", "achieved": achieved,
+        "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops_sustained"],
+        "peak_kind": f"cuBLAS bf16 sustained, {peaks['source']}; launches are timed back to back inside the step loop",
+        "traffic": NCU_DRAM_BYTES.get((w.name, f"{tile_m}x{tile_n}", spec)),
+        "algorithmic_flops_per_launch": flops,
+        "burst": {"achieved": flops / burst_ms / 1e9, "peak": peaks["bf16_tflops"],
+                  "frac": flops / burst_ms / 1e9 / peaks["bf16_tflops"], "protocol": "best of 10 isolated launches"},
+        "frac_of_nominal_2250": achieved / 2250.0,
+    }
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import gemm as G
+        t0 = time.perf_counter()
+        G.gemm_rows(A, B, np.arange(8))
+        rate = 8 / max(time.perf_counter() - t0, 1e-6)
+        rows = int(max(8, min(w.M, rate * 15.0)))
+        t0 = time.perf_counter()
+        G.gemm_rows(A, B, np.arange(rows))
+        dt = time.perf_counter() - t0
+        cpu_baseline = {"value": 2.0 * rows * w.N * w.K / dt / 1e12, "unit": "TFLOP/s", "cores": G.threads(),
+                        "kind": "oracle", "seconds": dt,
+                        "sample": f"first {rows} rows of C ({rows}x{w.N}x{w.K}) of the {w.M}-row product"}
+
+    if rank == 0:
+        line = {
+            "metric": "bf16 GEMM TFLOP/s", "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": agg["ms"] / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"{w.name}: C=A.B M={w.M} N={w.N} K={w.K}, bf16 in ({w.dist}, seed {w.seed}), fp32 "
+                                   f"accumulate, {w.out_dtype} out", "tile": f"{tile_m}x{tile_n}", "scheme": spec,
+                       "units": sp.gemm_units(tile_m, tile_n, sp.tile_count(w.M, w.N, tile_m, tile_n)),
+                       "l2": f"no flush: {resident / 1e6:.0f} MB resident per step vs {L2_BYTES / 1e6:.0f} MB L2",
+                       "parallelism": "replicas only" if world > 1 else "1 GPU"},
+            "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": args.steps,
+            "clocks": clocks,
+            "row_major": {"ms_per_step": row_ms, "tflops": flops / row_ms / 1e9, "speedup_of_scheme": row_ms / launch_ms},
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+    return 0
+
+
+def run_sweep(args, sp, w, dA, dB, dC, params_for, flops, stream) -> int:
+    """Every scheme of the workload, interleaved (ABAB) to share thermal state; JSON lines to stdout."""
+    import torch
+    specs = SWEEPS[args.workload]
+    for spec in specs:
+        s, p = params_for(spec)
+        for _ in range(3):
+            sp.gemm(dA, dB, dC, s, p, stream)
+    torch.cuda.synchronize()
+    best = {spec: 1e30 for spec in specs}
+    total = {spec: 0.0 for spec in specs}
+    rounds = max(args.steps, 1)
+    for _ in range(rounds):
+        for spec in specs:
+            s, p = params_for(spec)
+            ms = time_steps(sp, dA, dB, dC, s, p, 1, stream)
+            best[spec] = min(best[spec], ms)
+            total[spec] += ms
+    assert sp.get_status() == 0
+    ref = torch.empty_like(dC)
+    tb = 1e30
+    if dC.dtype == torch.bfloat16:
+        for _ in range(3):
+            torch.matmul(dA, dB, out=ref)
+        for _ in range(rounds):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); torch.matmul(dA, dB, out=ref); e1.record(); e1.synchronize()
+            tb = min(tb, e0.elapsed_time(e1))
+    for spec in specs:
+        print(json.dumps({"sweep": w.name, "scheme": spec, "best_ms": best[spec], "mean_ms": total[spec] / rounds,
+                          "best_tflops": flops / best[spec] / 1e9, "mean_tflops": flops * rounds / total[spec] / 1e9}),
+              flush=True)
+    if tb < 1e30:
+        print(json.dumps({"sweep": w.name, "scheme": "torch.matmul (cuBLAS, context only)", "best_ms": tb,
+                          "best_tflops": flops / tb / 1e9}), flush=True)
+    return 0
+
+
+def main() -> int:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg3", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--scheme", default=None)
+    ap.add_argument("--tile", default=None, help="MxN override, e.g. 128x256")
+    ap.add_argument("--kernel-only", action="store_true", help="time the kernel only (the command profilers wrap)")
+    ap.add_argument("--sweep", action="store_true", help="time every scheme of the workload")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -125,6 +125,13 @@ int sp_gemm(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t
 int sp_gemm_trace(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t K, int scheme,
                   const sp_params* params, void* stream, sp_trace_rec* trace_dev);
 
+/* sp_gemm for callers whose matrices live in HOST memory (pinned or pageable), same layouts and dtypes:
+ * copies A and B to a device staging area owned by the library (grown on demand, kept until sp_shutdown),
+ * runs sp_gemm, copies C back, and synchronises `stream`; C_host is valid on return.  One call at a time per
+ * device (the staging area is shared).  Adds SP_ERR_TIMEOUT to sp_gemm's errors. */
+int sp_gemm_host(const void* A_host, const void* B_host, void* C_host, int64_t M, int64_t N, int64_t K, int scheme,
+                 const sp_params* params, void* stream);
+
 /* Number of persistent CTAs (tile 128xN) or CTA pairs (tile 256xN) sp_gemm launches for T tiles;
  * slot s is run by unit s % units in round s / units.  Returns -1 on error. */
 int sp_gemm_units(int32_t tile_m, int32_t tile_n, int64_t T);

@@ -53,7 +53,8 @@ class SpTraceRec(ctypes.Structure):
 TRACE_DTYPE = np.dtype([("slot", "<i4"), ("tile", "<i4"), ("smid", "<i4"), ("unit", "<i4"), ("t_begin", "<u8"),
                         ("t_end", "<u8")])
 
-EXPORTS = ["sp_tile_count", "sp_tile_map", "sp_tile_map_device", "sp_gemm", "sp_gemm_trace", "sp_gemm_units",
+EXPORTS = ["sp_tile_count", "sp_tile_map", "sp_tile_map_device", "sp_gemm", "sp_gemm_trace", "sp_gemm_host",
+           "sp_gemm_units",
            "sp_probe_dispatch", "sp_get_status", "sp_last_error", "sp_shutdown"]
 
 
@@ -85,6 +86,8 @@ def lib() -> ctypes.CDLL:
         L.sp_gemm.argtypes = [vp, vp, vp, i64, i64, i64, ctypes.c_int, pp, vp]
         L.sp_gemm_trace.restype = ctypes.c_int
         L.sp_gemm_trace.argtypes = [vp, vp, vp, i64, i64, i64, ctypes.c_int, pp, vp, vp]
+        L.sp_gemm_host.restype = ctypes.c_int
+        L.sp_gemm_host.argtypes = [vp, vp, vp, i64, i64, i64, ctypes.c_int, pp, vp]
         L.sp_gemm_units.restype = ctypes.c_int
         L.sp_gemm_units.argtypes = [i32, i32, i64]
         L.sp_probe_dispatch.restype = ctypes.c_int
@@ -194,6 +197,29 @@ def gemm_trace(A, B, C, scheme: int = ROW_MAJOR, params: Optional[SpParams] = No
                                _stream_handle(stream), buf.data_ptr()))
     torch.cuda.synchronize()
     return np.frombuffer(buf.cpu().numpy().tobytes(), dtype=TRACE_DTYPE)
+
+
+def _host_ptr(x) -> int:
+    """Address of a host buffer: numpy array or CPU torch tensor (pinned or not)."""
+    if isinstance(x, np.ndarray):
+        if not x.flags["C_CONTIGUOUS"]:
+            raise ValueError("host arrays must be C-contiguous")
+        return int(x.ctypes.data)
+    if x.is_cuda or not x.is_contiguous():
+        raise ValueError("host tensors must be contiguous CPU tensors")
+    return int(x.data_ptr())
+
+
+def gemm_host(A, B, C, scheme: int = ROW_MAJOR, params: Optional[SpParams] = None, stream=None) -> None:
+    """C = A . B for HOST matrices (bf16 bit patterns as uint16/bfloat16; C bf16 or fp32 per params).
+    Copies in, computes on the GPU, copies out; C is valid on return."""
+    M, K = A.shape
+    b_nk = bool(params.b_layout) if params is not None else False
+    N = B.shape[0] if b_nk else B.shape[1]
+    if (B.shape[1] if b_nk else B.shape[0]) != K or tuple(C.shape) != (M, N):
+        raise ValueError("shape mismatch")
+    _check(lib().sp_gemm_host(_host_ptr(A), _host_ptr(B), _host_ptr(C), M, N, K, scheme, _pp(params),
+                              _stream_handle(stream)))
 
 
 def gemm_units(tile_m: int, tile_n: int, T: int) -> int:

@@ -141,6 +141,8 @@ struct DeviceState {
   int device = -1;
   int32_t* status = nullptr;
   std::vector<TableEntry> tables;
+  void* staging = nullptr;      // device copies of A, B, C for sp_gemm_host (grow-only)
+  size_t staging_bytes = 0;
 };
 
 static std::mutex g_mu;
@@ -330,6 +332,43 @@ int sp_gemm_trace(const void* A, const void* B, void* C, int64_t M, int64_t N, i
   return gemm_common(A, B, C, M, N, K, scheme, params, stream, trace_dev, true);
 }
 
+int sp_gemm_host(const void* A_host, const void* B_host, void* C_host, int64_t M, int64_t N, int64_t K, int scheme,
+                 const sp_params* params, void* stream) {
+  if (!A_host || !B_host || !C_host) { set_error("A, B and C must not be NULL"); return SP_ERR_INVALID_ARG; }
+  if (M <= 0 || N <= 0 || K <= 0) { set_error("M, N, K must be positive"); return SP_ERR_INVALID_ARG; }
+  if (M >= (1ll << 31) || N >= (1ll << 31) || K >= (1ll << 31)) { set_error("dimension too large"); return SP_ERR_UNSUPPORTED; }
+  if (params && params->struct_size != sizeof(sp_params)) {
+    set_error("sp_params.struct_size is %u, expected %zu", params->struct_size, sizeof(sp_params));
+    return SP_ERR_INVALID_ARG;
+  }
+  const size_t out_elt = (params && params->out_dtype == 1) ? 4 : 2;
+  auto pad = [](size_t b) { return (b + 255) & ~(size_t)255; };
+  const size_t a_bytes = (size_t)M * (size_t)K * 2, b_bytes = (size_t)K * (size_t)N * 2, c_bytes = (size_t)M * (size_t)N * out_elt;
+  const size_t need = pad(a_bytes) + pad(b_bytes) + pad(c_bytes);
+  int dev = 0;
+  int rc = current_device(&dev);
+  if (rc != SP_OK) return rc;
+  char *dA, *dB, *dC;
+  {
+    std::lock_guard<std::mutex> lock(g_mu);
+    DeviceState* ds = device_state(dev);
+    if (ds->staging_bytes < need) {
+      if (ds->staging) cudaFree(ds->staging);
+      ds->staging = nullptr; ds->staging_bytes = 0;
+      SP_CUDA(cudaMalloc(&ds->staging, need));
+      ds->staging_bytes = need;
+    }
+    dA = (char*)ds->staging; dB = dA + pad(a_bytes); dC = dB + pad(b_bytes);
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  SP_CUDA(cudaMemcpyAsync(dA, A_host, a_bytes, cudaMemcpyHostToDevice, st));
+  SP_CUDA(cudaMemcpyAsync(dB, B_host, b_bytes, cudaMemcpyHostToDevice, st));
+  rc = gemm_common(dA, dB, dC, M, N, K, scheme, params, stream, nullptr, false);
+  if (rc != SP_OK) return rc;
+  SP_CUDA(cudaMemcpyAsync(C_host, dC, c_bytes, cudaMemcpyDeviceToHost, st));
+  return sp_get_status(stream, nullptr);
+}
+
 int sp_gemm_units(int32_t tile_m, int32_t tile_n, int64_t T) {
   int dev = 0;
   if (current_device(&dev) != SP_OK) return -1;
@@ -377,6 +416,8 @@ void sp_shutdown(void) {
     d.tables.clear();
     if (d.status) cudaFree(d.status);
     d.status = nullptr;
+    if (d.staging) cudaFree(d.staging);
+    d.staging = nullptr; d.staging_bytes = 0;
   }
   g_devs.clear();
   if (have) cudaSetDevice(prev);

@@ -1,0 +1,56 @@
+"""The multi-rank bookkeeping of the benchmark (max of times, sum of work) under gloo, world size 2."""
+
+import os
+import socket
+import sys
+
+import pytest
+
+torch = pytest.importorskip("torch")
+import torch.multiprocessing as mp  # noqa: E402
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _worker(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    import torch.distributed as dist
+    from paper_2508_20258_b200 import benchutil
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    agg = benchutil.aggregate(10.0 + 5.0 * rank, 100.0 * (rank + 1), world)
+    out[rank] = (agg["ms"], agg["units"])
+    dist.destroy_process_group()
+
+
+def test_aggregate_two_ranks():
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    with mp.Manager() as m:
+        out = m.dict()
+        mp.spawn(_worker, args=(2, port, out), nprocs=2, join=True)
+        assert out[0] == out[1] == (15.0, 300.0)
+
+
+def test_aggregate_single_rank_is_identity():
+    sys.path.insert(0, ROOT)
+    from paper_2508_20258_b200 import benchutil
+    assert benchutil.aggregate(3.0, 7.0, 1) == {"ms": 3.0, "units": 7.0}
+    p = benchutil.measured_peaks(ROOT)
+    assert p["bf16_tflops"] > 0 and p["source"] in ("measured", "fallback")
+
+
+def test_scheme_specs_parse():
+    sys.path.insert(0, ROOT)
+    import bench
+    import paper_2508_20258_b200 as sp
+    assert bench.parse_scheme("group_m:8") == (sp.GROUP_M, dict(group=8))
+    assert bench.parse_scheme("xcd:2:74") == (sp.XCD, dict(num_xcds=2, wave=74, xcd_balanced=1))
+    assert bench.parse_scheme("die_split:n:group_m:8:i") == (
+        sp.DIE_SPLIT, dict(split_axis=1, inner_scheme=sp.GROUP_M, inner_group=8, interleave=1))
+    for name, specs in bench.SWEEPS.items():
+        for s in specs:
+            bench.parse_scheme(s)

@@ -1,0 +1,203 @@
+"""Parity of the CUDA path (through the C ABI) against the CPU oracle, element by element.
+
+Bars: remaps bit-exact; GEMM max floored relative error <= 1e-2 for bf16 inputs with fp32
+accumulation (the stated tolerance); integer-valued inputs and stamp matrices bit-exact,
+because every fp32 partial sum is then exact in any accumulation order.
+"""
+
+import numpy as np
+import pytest
+
+import paper_2508_20258_b200 as sp
+from oracle import gemm as G
+from oracle import remap as R
+from paper_2508_20258_b200 import synth
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-2
+
+torch = pytest.importorskip("torch")
+
+
+def dev_bf16(bits):
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def run_gemm(A, B, scheme=sp.ROW_MAJOR, tile=(256, 256), out="bf16", b_is_nk=False, **kw):
+    """A, B: uint16 bit patterns on the host (B as K x N).  Returns C as float64 on the host."""
+    M, K = A.shape
+    N = B.shape[1]
+    Bd = np.ascontiguousarray(B.T) if b_is_nk else B
+    dA, dB = dev_bf16(A), dev_bf16(Bd)
+    dC = torch.full((M, N), float("nan"), dtype=torch.float32 if out == "fp32" else torch.bfloat16, device="cuda")
+    p = sp.make_params(tile_m=tile[0], tile_n=tile[1], out_dtype=int(out == "fp32"), b_layout=int(b_is_nk), **kw)
+    sp.gemm(dA, dB, dC, scheme, p)
+    assert sp.get_status() == 0
+    if out == "fp32":
+        return dC.cpu().numpy().astype(np.float64), dC
+    return G.bf16_bits_to_f64(dC.view(torch.int16).cpu().numpy().view(np.uint16)), dC
+
+
+# ------------------------------------------------------------------ remap: device code == oracle
+@pytest.mark.parametrize("M,N,tm,tn", [(512, 512, 128, 128), (4096, 4096, 128, 256), (8192, 8192, 256, 256),
+                                        (16384, 2048, 256, 256), (16384, 16384, 256, 256), (1000, 520, 128, 128),
+                                        (128 * 37, 128 * 5, 128, 128), (128, 128 * 300, 128, 128)])
+def test_device_remap_matches_oracle(M, N, tm, tn):
+    cases = [(sp.ROW_MAJOR, {}), (sp.COL_MAJOR, {}), (sp.GROUP_M, dict(group=8)), (sp.GROUP_M, dict(group=3)),
+             (sp.GROUP_N, dict(group=4)), (sp.MORTON, {}), (sp.HILBERT, {}),
+             (sp.XCD, dict(num_xcds=2, wave=74, xcd_balanced=1)), (sp.XCD, dict(num_xcds=8, xcd_balanced=1)),
+             (sp.DIE_SPLIT, dict(split_axis=0, inner_scheme=sp.HILBERT)),
+             (sp.DIE_SPLIT, dict(split_axis=1, inner_scheme=sp.GROUP_M, inner_group=8, interleave=1)),
+             (sp.DIE_SPLIT, dict(split_axis=1, inner_scheme=sp.MORTON, interleave=1))]
+    for scheme, kw in cases:
+        want = R.tile_map(M, N, tm, tn, scheme, R.Params(**kw))
+        got = sp.tile_map_device(M, N, tm, tn, scheme, sp.make_params(**kw)).cpu().numpy().tolist()
+        assert got == want, (scheme, kw)
+    table = np.random.default_rng(0).permutation(sp.tile_count(M, N, tm, tn)).astype(np.int32)
+    got = sp.tile_map_device(M, N, tm, tn, sp.CUSTOM, sp.make_params(custom_perm=table)).cpu().numpy()
+    assert np.array_equal(got, table)
+
+
+# ------------------------------------------------------------------ exact cases
+SHAPES = [(128, 128), (128, 256), (256, 128), (256, 256)]
+
+
+@pytest.mark.parametrize("tile", SHAPES)
+@pytest.mark.parametrize("b_is_nk", [False, True])
+@pytest.mark.parametrize("M,N,K", [(128, 128, 64), (300, 328, 200), (1000, 520, 264), (768, 1024, 8192)])
+def test_integer_inputs_are_bit_exact(tile, b_is_nk, M, N, K):
+    A, B = synth.make_int_inputs(M, N, K, seed=M + K)
+    ref, _ = G.gemm_full(A, B)
+    got, _ = run_gemm(A, B, sp.GROUP_M, tile, "fp32", b_is_nk, group=2)
+    assert np.array_equal(got, ref)
+
+
+@pytest.mark.parametrize("tile", SHAPES)
+@pytest.mark.parametrize("b_is_nk", [False, True])
+@pytest.mark.parametrize("kk", [0, 17, 63, 100])
+def test_stamp_matrices_pin_addressing(tile, b_is_nk, kk):
+    """One non-zero k: C[i,j] = 2^(i mod 8) * 2^-(j mod 16) names its own position, so a
+    misplaced row, column, k-slice or a transposed operand cannot pass."""
+    M, N, K = 520, 776, 128
+    Af = np.zeros((M, K), np.float32)
+    Bf = np.zeros((K, N), np.float32)
+    Af[:, kk] = 2.0 ** (np.arange(M) % 8) * (1 + (np.arange(M) // 8) % 2)
+    Bf[kk, :] = 2.0 ** -(np.arange(N) % 16) * (1 + 2 * ((np.arange(N) // 16) % 2))
+    A, B = synth.f32_to_bf16_bits(Af), synth.f32_to_bf16_bits(Bf)
+    ref, _ = G.gemm_full(A, B)
+    got, _ = run_gemm(A, B, sp.COL_MAJOR, tile, "fp32", b_is_nk)
+    assert np.array_equal(got, ref)
+
+
+@pytest.mark.parametrize("tile", [(128, 256), (256, 256)])
+def test_bf16_output_is_rne_of_the_fp32_result(tile):
+    A, B = synth.make_inputs(512, 768, 1024, "normal", 1.0, 9)
+    f32, _ = run_gemm(A, B, sp.ROW_MAJOR, tile, "fp32")
+    b16, _ = run_gemm(A, B, sp.ROW_MAJOR, tile, "bf16")
+    want = G.bf16_bits_to_f64(synth.f32_to_bf16_bits(f32.astype(np.float32)))
+    assert np.array_equal(b16, want)
+
+
+# ------------------------------------------------------------------ small workloads, every element
+@pytest.mark.parametrize("scheme,kw", [(sp.ROW_MAJOR, {}), (sp.GROUP_M, dict(group=2))])
+def test_cfg1_full(scheme, kw):
+    w, A, B = synth.make_workload("cfg1")
+    ref, S = G.gemm_full(A, B)
+    got, _ = run_gemm(A, B, scheme, (w.tile_m, w.tile_n), w.out_dtype, **kw)
+    r = G.compare(got, ref, S)
+    assert r["max_err"] <= TOL, r
+    assert r["fro_rel"] <= 1e-5, r          # fp32 output: only accumulation rounding remains
+
+
+@pytest.mark.parametrize("M,N,K,tile,out", [(640, 896, 1000, (128, 128), "bf16"), (1160, 600, 520, (128, 256), "fp32"),
+                                             (1160, 1100, 776, (256, 256), "bf16"), (904, 648, 1288, (256, 128), "bf16")])
+@pytest.mark.parametrize("b_is_nk", [False, True])
+def test_ragged_sizes_full(M, N, K, tile, out, b_is_nk):
+    """Several tiles, ragged M / N tails, K not a multiple of the 64-wide k-block."""
+    A, B = synth.make_inputs(M, N, K, "normal", 1.0, seed=M)
+    ref, S = G.gemm_full(A, B)
+    for scheme, kw in [(sp.HILBERT, {}), (sp.XCD, dict(num_xcds=2, xcd_balanced=1))]:
+        got, _ = run_gemm(A, B, scheme, tile, out, b_is_nk, **kw)
+        r = G.compare(got, ref, S)
+        assert r["max_err"] <= TOL, (scheme, r)
+
+
+def test_tiny_and_degenerate_sizes():
+    for (M, N, K) in [(1, 8, 8), (8, 8, 8), (129, 264, 72), (256, 8, 64)]:
+        A, B = synth.make_int_inputs(M, N, K, seed=3)
+        ref, _ = G.gemm_full(A, B)
+        for tile in SHAPES:
+            got, _ = run_gemm(A, B, sp.ROW_MAJOR, tile, "fp32")
+            assert np.array_equal(got, ref), (M, N, K, tile)
+
+
+def test_cfg2_full():
+    w, A, B = synth.make_workload("cfg2")
+    ref, S = G.gemm_full(A, B)
+    first = None
+    for scheme, kw in [(sp.ROW_MAJOR, {}), (sp.GROUP_M, dict(group=4)), (sp.GROUP_M, dict(group=8)),
+                       (sp.GROUP_M, dict(group=16)), (sp.HILBERT, {})]:
+        got, dC = run_gemm(A, B, scheme, (w.tile_m, w.tile_n), w.out_dtype, **kw)
+        r = G.compare(got, ref, S)
+        assert r["max_err"] <= TOL, (scheme, kw, r)
+        assert r["fro_rel"] <= 3e-3, r
+        bits = dC.view(torch.int16).cpu().numpy()
+        if first is None:
+            first = bits
+        else:
+            assert np.array_equal(bits, first)      # a swizzle only reorders tiles: same bits
+
+
+# ------------------------------------------------------------------ schedule evidence
+@pytest.mark.parametrize("tile", [(128, 256), (256, 256)])
+def test_trace_runs_every_tile_once_under_the_remap(tile):
+    M, N, K = 4096, 4096, 256
+    A, B = synth.make_int_inputs(M, N, K, seed=5)
+    dA, dB = dev_bf16(A), dev_bf16(B)
+    dC = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    for scheme, kw in [(sp.ROW_MAJOR, {}), (sp.HILBERT, {}), (sp.GROUP_M, dict(group=4)),
+                       (sp.DIE_SPLIT, dict(split_axis=0, inner_scheme=sp.GROUP_N, inner_group=2, interleave=1))]:
+        p = sp.make_params(tile_m=tile[0], tile_n=tile[1], **kw)
+        tr = sp.gemm_trace(dA, dB, dC, scheme, p)
+        assert sp.get_status() == 0
+        want = R.tile_map(M, N, tile[0], tile[1], scheme, R.Params(**kw))
+        T = len(want)
+        assert tr["slot"].tolist() == list(range(T))
+        assert tr["tile"].tolist() == want
+        assert sorted(tr["tile"].tolist()) == list(range(T))
+        units = sp.gemm_units(tile[0], tile[1], T)
+        assert tr["unit"].tolist() == [s % units for s in range(T)]
+        assert (tr["t_end"] > tr["t_begin"]).all()
+        # a unit runs its slots in increasing order
+        for u in range(min(units, 4)):
+            mine = tr[tr["unit"] == u]
+            assert (np.diff(mine["t_begin"].astype(np.int64)) > 0).all()
+            assert len(set(mine["smid"].tolist())) == 1
+
+
+def test_output_bits_do_not_depend_on_the_scheme():
+    A, B = synth.make_inputs(2048, 2304, 1024, "normal", 1.0, 12)
+    ref = None
+    table = np.random.default_rng(1).permutation(8 * 9).astype(np.int32)
+    for scheme, kw in [(sp.ROW_MAJOR, {}), (sp.COL_MAJOR, {}), (sp.GROUP_N, dict(group=3)), (sp.MORTON, {}),
+                       (sp.XCD, dict(num_xcds=4, wave=16, xcd_balanced=1)), (sp.CUSTOM, dict(custom_perm=table)),
+                       (sp.DIE_SPLIT, dict(split_axis=1, inner_scheme=sp.HILBERT))]:
+        _, dC = run_gemm(A, B, scheme, (256, 256), "bf16", **kw)
+        bits = dC.view(torch.int16).cpu().numpy()
+        if ref is None:
+            ref = bits
+        assert np.array_equal(bits, ref), scheme
+
+
+def test_runtime_rejections_launch_nothing():
+    A = torch.zeros((256, 256), dtype=torch.bfloat16, device="cuda")
+    C = torch.full((256, 256), 7.0, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(sp.SpError) as e:
+        sp.gemm(A, A, C, sp.XCD, sp.make_params(tile_m=128, tile_n=128, num_xcds=3))   # 4 tiles, X = 3
+    assert e.value.status == sp.ERR_NOT_BIJECTIVE
+    with pytest.raises(sp.SpError) as e:
+        sp.gemm(A, A, C, sp.CUSTOM, sp.make_params(tile_m=128, tile_n=128, custom_perm=[0, 1, 1, 3]))
+    assert e.value.status == sp.ERR_NOT_BIJECTIVE
+    torch.cuda.synchronize()
+    assert (C == 7.0).all()
+    assert sp.get_status() == 0

@@ -1,0 +1,98 @@
+"""Parity at the full sizes of the three large workloads, in the launch configuration the
+benchmark times: sampled rows and whole tiles computed one by one by the oracle, plus a
+whole-matrix randomised identity that holds at any size.
+
+Sampling: for every tile row, 4 complete rows of C (they cross every tile and every
+column) at in-tile offsets that land in each 32-lane quarter of the accumulator and in
+both CTAs of a pair and walk through all residues mod 8 as the tile row varies; the first
+and last row of the matrix; and 12 complete tiles (corners, both sides of the half-way
+boundary, seeded random).
+"""
+
+import numpy as np
+import pytest
+
+import paper_2508_20258_b200 as sp
+from oracle import gemm as G
+from paper_2508_20258_b200 import synth
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-2
+torch = pytest.importorskip("torch")
+
+
+def dev_bf16(bits):
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def sample_rows(M, tile_m):
+    Tm = -(-M // tile_m)
+    rows = {0, M - 1}
+    for tm in range(Tm):
+        for j in range(4):
+            r = tm * tile_m + (37 * tm + (tile_m // 4) * j + 11) % tile_m
+            if r < M:
+                rows.add(r)
+    return sorted(rows)
+
+
+def sample_tiles(Tm, Tn, seed):
+    rng = np.random.default_rng(seed)
+    tiles = {(0, 0), (0, Tn - 1), (Tm - 1, 0), (Tm - 1, Tn - 1),
+             ((Tm + 1) // 2 - 1, Tn // 3), ((Tm + 1) // 2, Tn // 3)}
+    while len(tiles) < min(12, Tm * Tn):
+        tiles.add((int(rng.integers(Tm)), int(rng.integers(Tn))))
+    return sorted(tiles)
+
+
+CASES = [
+    ("cfg3", [(sp.ROW_MAJOR, {}), (sp.GROUP_M, dict(group=8)), (sp.HILBERT, {}),
+              (sp.DIE_SPLIT, dict(split_axis=0, inner_scheme=sp.GROUP_M, inner_group=8))]),
+    ("cfg4", [(sp.GROUP_M, dict(group=4)), (sp.GROUP_N, dict(group=2))]),
+    ("cfg5", [(sp.GROUP_M, dict(group=16)), (sp.HILBERT, {})]),
+]
+
+
+@pytest.mark.parametrize("name,schemes", CASES)
+def test_large_workload_sampled(name, schemes):
+    w, A, B = synth.make_workload(name)
+    dA, dB = dev_bf16(A), dev_bf16(B)
+    dC = torch.empty((w.M, w.N), dtype=torch.bfloat16, device="cuda")
+    rows = sample_rows(w.M, w.tile_m)
+    ref_rows, S_rows = G.gemm_rows(A, B, rows)
+    Tm, Tn = -(-w.M // w.tile_m), -(-w.N // w.tile_n)
+    tiles = sample_tiles(Tm, Tn, w.seed)
+    tile_refs = [G.gemm_block(A, B, tm * w.tile_m, min((tm + 1) * w.tile_m, w.M), tn * w.tile_n,
+                              min((tn + 1) * w.tile_n, w.N)) for (tm, tn) in tiles]
+    # randomised identity: C x = A (B x) for x in {+-1}^N, in fp64
+    Af = synth.bf16_bits_to_f32(A).astype(np.float64)
+    Bf = synth.bf16_bits_to_f32(B).astype(np.float64)
+    xs = [np.random.default_rng(100 + i).choice([-1.0, 1.0], size=w.N) for i in range(2)]
+    want_cx = [Af @ (Bf @ x) for x in xs]
+    del Af, Bf
+    first_bits = None
+    for scheme, kw in schemes:
+        dC.fill_(float("nan"))
+        p = sp.make_params(tile_m=w.tile_m, tile_n=w.tile_n, out_dtype=0, **kw)
+        sp.gemm(dA, dB, dC, scheme, p)
+        assert sp.get_status() == 0
+        bits = dC.view(torch.int16).cpu().numpy().view(np.uint16)
+        got_rows = G.bf16_bits_to_f64(bits[rows, :])
+        r = G.compare(got_rows, ref_rows, S_rows)
+        assert r["max_err"] <= TOL, (name, scheme, kw, r)
+        assert r["fro_rel"] <= 3e-3, r
+        for (tm, tn), (ref, S) in zip(tiles, tile_refs):
+            blk = bits[tm * w.tile_m:(tm + 1) * w.tile_m, tn * w.tile_n:(tn + 1) * w.tile_n]
+            rt = G.compare(G.bf16_bits_to_f64(blk), ref, S)
+            assert rt["max_err"] <= TOL, (name, scheme, kw, tm, tn, rt)
+        if first_bits is None:
+            first_bits = bits
+            Cf = G.bf16_bits_to_f64(bits)
+            norms = np.sqrt((Cf ** 2).sum(axis=1))
+            for x, want in zip(xs, want_cx):
+                # bf16 rounding: |e_ij| <= 2^-9 |C_ij|, independent signs -> sigma <= 2^-9/sqrt(3) * ||C_i||; gate 6 sigma
+                assert (np.abs(Cf @ x - want) <= 6 * 2.0 ** -9 / np.sqrt(3) * norms + 1e-9).all()
+            assert not np.isnan(Cf).any()
+            del Cf
+        else:
+            assert np.array_equal(bits, first_bits)      # same bits under every order
