@@ -82,6 +82,20 @@ def dist_env():
     return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
 
 
+def _rows_for_seconds(G, A, B, M, seconds):
+    """How many rows of C the oracle computes in about `seconds` (two probes separate the fixed
+    cost of widening the B panel from the per-row cost)."""
+    t0 = time.perf_counter()
+    G.gemm_rows(A, B, np.arange(4))
+    t4 = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    G.gemm_rows(A, B, np.arange(36))
+    t36 = time.perf_counter() - t0
+    per_row = max((t36 - t4) / 32.0, 1e-6)
+    fixed = max(t4 - 4 * per_row, 0.0)
+    return int(max(1, min(M, (seconds - fixed) / per_row)))
+
+
 # ---------------------------------------------------------------------------------- reference arm
 def run_reference(args) -> int:
     """Times the CPU oracle, as it stands, on a bounded sample of the same workload."""
@@ -92,11 +106,7 @@ def run_reference(args) -> int:
     w = synth.WORKLOADS[args.workload]
     _, A, B = synth.make_workload(args.workload)
     cores = G.threads()
-    t0 = time.perf_counter()
-    G.gemm_rows(A, B, np.arange(8))                                   # calibration, also builds the object
-    rate = 8 / max(time.perf_counter() - t0, 1e-6)                    # rows per second (includes panel widening)
-    budget = 150.0 / (args.steps + args.warmup)
-    rows = int(max(1, min(w.M // 16, rate * budget)))
+    rows = min(_rows_for_seconds(G, A, B, w.M, 150.0 / (args.steps + args.warmup)), max(1, w.M // 16))
     band = np.arange(rows)
     for _ in range(args.warmup):
         G.gemm_rows(A, B, band)
@@ -238,10 +248,7 @@ def run_ours(args) -> int:
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         from oracle import gemm as G
-        t0 = time.perf_counter()
-        G.gemm_rows(A, B, np.arange(8))
-        rate = 8 / max(time.perf_counter() - t0, 1e-6)
-        rows = int(max(8, min(w.M, rate * 15.0)))
+        rows = _rows_for_seconds(G, A, B, w.M, 15.0)
         t0 = time.perf_counter()
         G.gemm_rows(A, B, np.arange(rows))
         dt = time.perf_counter() - t0
