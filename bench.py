@@ -178,6 +178,14 @@ def run_ours(args) -> int:
 
     if args.sweep:
         return run_sweep(args, sp, w, dA, dB, dC, params_for, flops, stream)
+    if args.profile_sweep:                     # one launch per scheme, in SWEEPS order: the command ncu wraps
+        specs = args.scheme.split(",") if args.scheme else SWEEPS[args.workload]
+        for spec in specs:
+            s_, p_ = params_for(spec)
+            sp.gemm(dA, dB, dC, s_, p_, stream)
+        assert sp.get_status() == 0
+        print(json.dumps({"profile_sweep": w.name, "tile": f"{tile_m}x{tile_n}", "launch_order": specs}), flush=True)
+        return 0
 
     spec = args.scheme or DEFAULT_SCHEME[args.workload]
     scheme, p = params_for(spec)
@@ -326,6 +334,7 @@ def main() -> int:
     ap.add_argument("--tile", default=None, help="MxN override, e.g. 128x256")
     ap.add_argument("--kernel-only", action="store_true", help="time the kernel only (the command profilers wrap)")
     ap.add_argument("--sweep", action="store_true", help="time every scheme of the workload")
+    ap.add_argument("--profile-sweep", action="store_true", help="launch each scheme once (for ncu counters)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -90,8 +90,10 @@ def test_large_workload_sampled(name, schemes):
             Cf = G.bf16_bits_to_f64(bits)
             norms = np.sqrt((Cf ** 2).sum(axis=1))
             for x, want in zip(xs, want_cx):
-                # bf16 rounding: |e_ij| <= 2^-9 |C_ij|, independent signs -> sigma <= 2^-9/sqrt(3) * ||C_i||; gate 6 sigma
-                assert (np.abs(Cf @ x - want) <= 6 * 2.0 ** -9 / np.sqrt(3) * norms + 1e-9).all()
+                # bf16 keeps 8 significand bits: round-to-nearest errs by at most half an ulp, |e_ij| <= 2^-8 |C_ij|
+                # (uniform within that), signs independent of x -> sigma_i <= 2^-8/sqrt(3) * ||C_i||; gate 6 sigma.
+                # A dropped 256-wide tile segment moves a row sum by ~16 * sigma_C, about 13x this gate.
+                assert (np.abs(Cf @ x - want) <= 6 * 2.0 ** -8 / np.sqrt(3) * norms + 1e-9).all()
             assert not np.isnan(Cf).any()
             del Cf
         else:
