@@ -158,7 +158,8 @@ def run_ours(args) -> int:
     w = synth.WORKLOADS[args.workload]
     tile_m, tile_n = (int(v) for v in args.tile.split("x")) if args.tile else (w.tile_m, w.tile_n)
     out_f32 = int(w.out_dtype == "fp32")
-    _, A, B = synth.make_workload(args.workload)
+    b_nk = int(args.b_layout == "nk")
+    _, A, B = synth.make_workload(args.workload, b_is_nk=bool(b_nk))
     dA = torch.from_numpy(A.view(np.int16)).cuda().view(torch.bfloat16)
     dB = torch.from_numpy(B.view(np.int16)).cuda().view(torch.bfloat16)
     dC = torch.empty((w.M, w.N), dtype=torch.float32 if out_f32 else torch.bfloat16, device="cuda")
@@ -168,7 +169,7 @@ def run_ours(args) -> int:
 
     def params_for(spec):
         scheme, kw = parse_scheme(spec)
-        return scheme, sp.make_params(tile_m=tile_m, tile_n=tile_n, out_dtype=out_f32, **kw)
+        return scheme, sp.make_params(tile_m=tile_m, tile_n=tile_n, out_dtype=out_f32, b_layout=b_nk, **kw)
 
     def barrier():
         if world > 1:
@@ -335,6 +336,7 @@ def main() -> int:
     ap.add_argument("--kernel-only", action="store_true", help="time the kernel only (the command profilers wrap)")
     ap.add_argument("--sweep", action="store_true", help="time every scheme of the workload")
     ap.add_argument("--profile-sweep", action="store_true", help="launch each scheme once (for ncu counters)")
+    ap.add_argument("--b-layout", default="kn", choices=["kn", "nk"], help="B stored K x N (default) or N x K")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

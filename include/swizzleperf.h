@@ -85,8 +85,14 @@ typedef struct {
   int32_t tile;      /* logical tile id executed at that slot          */
   int32_t smid;      /* %smid of the (leader) CTA that ran it          */
   int32_t unit;      /* index of the persistent CTA / CTA pair         */
-  uint64_t t_begin;  /* %globaltimer when its first load was issued    */
-  uint64_t t_end;    /* %globaltimer when its last store was issued    */
+  uint64_t t_begin;  /* %globaltimer (ns) when its first load was issued                      */
+  uint64_t t_end;    /* %globaltimer when its last store was issued                            */
+  uint64_t t_mma_begin;   /* %globaltimer when the MMA issuer started on the tile               */
+  uint64_t t_mma_issued;  /* %globaltimer when it had issued the tile's last MMA                */
+  uint32_t mma_wait_data; /* SM cycles the MMA issuer waited for operand stages of this tile    */
+  uint32_t mma_wait_acc;  /* SM cycles it waited for a free accumulator buffer                  */
+  uint32_t load_wait_stage; /* SM cycles the producer waited for a free stage                   */
+  uint32_t epi_wait_acc;  /* SM cycles the first epilogue warp waited for the accumulator       */
 } sp_trace_rec;
 
 /* Number of tiles T = ceil(M/tileM) * ceil(N/tileN); -1 on non-positive arguments. */

@@ -47,11 +47,14 @@ class SpParams(ctypes.Structure):
 
 class SpTraceRec(ctypes.Structure):
     _fields_ = [("slot", ctypes.c_int32), ("tile", ctypes.c_int32), ("smid", ctypes.c_int32), ("unit", ctypes.c_int32),
-                ("t_begin", ctypes.c_uint64), ("t_end", ctypes.c_uint64)]
+                ("t_begin", ctypes.c_uint64), ("t_end", ctypes.c_uint64), ("t_mma_begin", ctypes.c_uint64),
+                ("t_mma_issued", ctypes.c_uint64), ("mma_wait_data", ctypes.c_uint32), ("mma_wait_acc", ctypes.c_uint32),
+                ("load_wait_stage", ctypes.c_uint32), ("epi_wait_acc", ctypes.c_uint32)]
 
 
 TRACE_DTYPE = np.dtype([("slot", "<i4"), ("tile", "<i4"), ("smid", "<i4"), ("unit", "<i4"), ("t_begin", "<u8"),
-                        ("t_end", "<u8")])
+                        ("t_end", "<u8"), ("t_mma_begin", "<u8"), ("t_mma_issued", "<u8"), ("mma_wait_data", "<u4"),
+                        ("mma_wait_acc", "<u4"), ("load_wait_stage", "<u4"), ("epi_wait_acc", "<u4")])
 
 EXPORTS = ["sp_tile_count", "sp_tile_map", "sp_tile_map_device", "sp_gemm", "sp_gemm_trace", "sp_gemm_host",
            "sp_gemm_units",

@@ -150,6 +150,21 @@ static std::vector<DeviceState> g_devs;
 static uint64_t g_stamp = 0;
 constexpr size_t kMaxTables = 64;
 
+static std::mutex g_valid_mu;
+static std::vector<Sched> g_validated;
+
+static bool already_validated(const Sched& c) {
+  std::lock_guard<std::mutex> lock(g_valid_mu);
+  for (const Sched& v : g_validated) if (memcmp(&v, &c, sizeof c) == 0) return true;
+  return false;
+}
+
+static void remember_validated(const Sched& c) {
+  std::lock_guard<std::mutex> lock(g_valid_mu);
+  if (g_validated.size() >= 256) g_validated.erase(g_validated.begin());
+  g_validated.push_back(c);
+}
+
 static DeviceState* device_state(int dev) {
   for (auto& d : g_devs) if (d.device == dev) return &d;
   g_devs.emplace_back();
@@ -252,9 +267,14 @@ static int gemm_common(const void* A, const void* B, void* C, int64_t M, int64_t
   memset(&call, 0, sizeof call);
   int rc = resolve_sched(M, N, tile_m, tile_n, scheme, params, &call.sched);
   if (rc != SP_OK) return rc;
+  // Bijectivity gate.  A (grid, scheme, parameters) that passed once is remembered, so the hot
+  // path does no O(T) host work; caller tables are re-checked on every call (their contents may change).
   std::vector<int32_t> host_perm;
-  rc = build_perm_host(call.sched, params ? params->custom_perm : nullptr, host_perm);  // bijectivity gate
-  if (rc != SP_OK) return rc;
+  if (scheme == kCustom || !already_validated(call.sched)) {
+    rc = build_perm_host(call.sched, params ? params->custom_perm : nullptr, host_perm);
+    if (rc != SP_OK) return rc;
+    if (scheme != kCustom) remember_validated(call.sched);
+  }
 
   int dev = 0;
   rc = current_device(&dev);

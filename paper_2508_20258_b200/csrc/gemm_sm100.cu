@@ -55,7 +55,17 @@ struct GemmArgs {
   int kblocks;
   int units;
   uint32_t b_lbo, b_sbo, b_kstep;  // B operand descriptor strides in bytes
+  uint32_t debug;                  // experiment switches (SP_DEBUG_FLAGS); 0 in normal use
   Sched sched;
+};
+
+// Experiment switches: results are wrong by design when any of these is set.
+enum : uint32_t {
+  kDbgSameOperands = 1u,   // every load fetches the first k-block of the first tile (all L2 hits)
+  kDbgNoStores = 2u,       // epilogue reads TMEM but stores nothing
+  kDbgNoLoads = 4u,        // producer issues no copies; stages are handed over empty
+  kDbgFreeRunMma = 8u,     // no producer at all; the MMA issuer ignores the stage barriers (pure issue rate)
+  kDbgSplitN = 16u,        // with kDbgFreeRunMma: two N/2 MMAs into two accumulators instead of one N-wide MMA
 };
 
 // status word: (role << 8) | which wait
@@ -74,6 +84,17 @@ __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
   return r;
+}
+
+// True in exactly one lane of a fully converged warp.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
 }
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -125,6 +146,17 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, int32
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t* status, int code) {
   if (mbar_try_wait(bar, parity)) return true;
   return mbar_wait_slow(bar, parity, status, code);
+}
+
+// mbar_wait that also adds the cycles spent waiting to *acc when tracing.
+__device__ __forceinline__ bool mbar_wait_timed(uint32_t bar, uint32_t parity, int32_t* status, int code, bool timed,
+                                                uint32_t* acc) {
+  if (mbar_try_wait(bar, parity)) return true;
+  if (!timed) return mbar_wait_slow(bar, parity, status, code);
+  const long long c0 = clock64();
+  const bool ok = mbar_wait_slow(bar, parity, status, code);
+  *acc += (uint32_t)(clock64() - c0);
+  return ok;
 }
 
 template <int CG>
@@ -283,7 +315,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer
-    if (lane == 0) {
+    // The whole warp walks the loop (uniform control flow, uniform operands); one elected
+    // lane issues the copies.
+    if (!(args.debug & kDbgFreeRunMma)) {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
@@ -292,35 +326,49 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const int tm = t / Tn, tn = t - tm * Tn;
         const int row0 = tm * TILE_M + (int)rank * 128;
         const int col0 = tn * BN + (int)rank * C::kBCols;
-        if (args.trace && rank == 0) {
+        const bool tracing = args.trace != nullptr && rank == 0;
+        uint32_t waited = 0;
+        if (tracing && lane == 0) {
           sp_trace_rec* rec = args.trace + s;
           uint32_t smid;
           asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
           rec->slot = s; rec->tile = t; rec->smid = (int)smid; rec->unit = unit; rec->t_begin = globaltimer();
         }
         for (int kb = 0; kb < KB; ++kb) {
-          ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, args.status, (kRoleProducer << 8) | 1);
+          ok = mbar_wait_timed(bar_empty + 8 * stage, phase ^ 1u, args.status, (kRoleProducer << 8) | 1, tracing, &waited);
+          ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           const uint32_t full_local = bar_full + 8 * stage;
           const uint32_t full_leader = CG == 1 ? full_local : mapa(full_local, 0);
-          if (rank == 0) mbar_arrive_expect_tx(full_local, CG * C::kStageBytes);
           const uint32_t sa = smem_base + stage * C::kStageBytes;
           const uint32_t sb = sa + C::kABytes;
-          tma_load_2d<CG>(sa, &tmA, kb * kBK, row0, full_leader);
-          if constexpr (B_NK) {
-            tma_load_2d<CG>(sb, &tmB, kb * kBK, col0, full_leader);
-          } else {
+          const bool same = (args.debug & kDbgSameOperands) != 0;
+          const int kx = same ? 0 : kb * kBK, ry = same ? (int)rank * 128 : row0, cx = same ? (int)rank * C::kBCols : col0;
+          if (elect_one()) {
+            if (args.debug & kDbgNoLoads) {
+              if (rank == 0) mbar_arrive_expect_tx(full_local, 0);
+            } else {
+              if (rank == 0) mbar_arrive_expect_tx(full_local, CG * C::kStageBytes);
+              tma_load_2d<CG>(sa, &tmA, kx, ry, full_leader);
+              if constexpr (B_NK) {
+                tma_load_2d<CG>(sb, &tmB, kx, cx, full_leader);
+              } else {
 #pragma unroll
-            for (int j = 0; j < C::kBCols / 64; ++j)
-              tma_load_2d<CG>(sb + j * (64 * kBK * 2), &tmB, col0 + j * 64, kb * kBK, full_leader);
+                for (int j = 0; j < C::kBCols / 64; ++j)
+                  tma_load_2d<CG>(sb + j * (64 * kBK * 2), &tmB, cx + j * 64, kx, full_leader);
+              }
+            }
           }
+          __syncwarp();
           if (++stage == S) { stage = 0; phase ^= 1u; }
         }
+        if (tracing && lane == 0) args.trace[s].load_wait_stage = waited;
       }
       // tail: every stage handed out must have been released, so that no commit arrival
       // (or, after a failure, no copy) is still in flight towards this CTA when it exits
       for (int i = 0; i < S && ok; ++i) {
         ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, args.status, (kRoleProducer << 8) | 2);
+        ok = __all_sync(0xffffffffu, ok);
         if (++stage == S) { stage = 0; phase ^= 1u; }
       }
       if (!ok) {
@@ -331,7 +379,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     __syncwarp();
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issuer (leader CTA only)
-    if (lane == 0 && rank == 0) {
+    // Whole warp in the loop, one elected lane issues: descriptors stay warp-uniform values.
+    if (rank == 0) {
       constexpr uint32_t idesc = make_idesc(TILE_M, BN, !B_NK);
       int stage = 0;
       uint32_t phase = 0;
@@ -340,26 +389,63 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       for (int s = unit; s < T && ok; s += args.units, ++it) {
         const int buf = it & 1;
         const uint32_t use = (uint32_t)(it >> 1) & 1u;
-        ok = mbar_wait(bar_tempty + 8 * buf, use ^ 1u, args.status, (kRoleMma << 8) | 1);
+        const bool tracing = args.trace != nullptr;
+        uint32_t wait_acc = 0, wait_data = 0;
+        ok = mbar_wait_timed(bar_tempty + 8 * buf, use ^ 1u, args.status, (kRoleMma << 8) | 1, tracing, &wait_acc);
+        ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tcgen05_fence_after();
+        if (tracing && lane == 0) args.trace[s].t_mma_begin = globaltimer();
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+        if (args.debug & kDbgFreeRunMma) {
+          constexpr uint32_t idesc_half = make_idesc(TILE_M, BN / 2, !B_NK);
+          for (int kb = 0; kb < KB; ++kb) {
+            const uint32_t sa = smem_base + (kb % S) * C::kStageBytes;
+            const uint32_t sb = sa + C::kABytes;
+            if (elect_one()) {
+#pragma unroll
+              for (int k = 0; k < kBK / kUmmaK; ++k) {
+                const uint64_t da = smem_desc(sa + k * (kUmmaK * 2), 16, 1024);
+                const uint64_t db = smem_desc(sb + k * args.b_kstep, args.b_lbo, args.b_sbo);
+                if (args.debug & kDbgSplitN) {
+                  umma_bf16<CG>(d_tmem, da, db, idesc_half, (uint32_t)((kb | k) != 0));
+                  umma_bf16<CG>(d_tmem + BN / 2, da, db, idesc_half, (uint32_t)((kb | k) != 0));
+                } else {
+                  umma_bf16<CG>(d_tmem, da, db, idesc, (uint32_t)((kb | k) != 0));
+                }
+              }
+            }
+            __syncwarp();
+          }
+          if (elect_one()) umma_commit<CG>(bar_tfull + 8 * buf);
+          __syncwarp();
+          continue;
+        }
         for (int kb = 0; kb < KB; ++kb) {
-          ok = mbar_wait(bar_full + 8 * stage, phase, args.status, (kRoleMma << 8) | 2);
+          ok = mbar_wait_timed(bar_full + 8 * stage, phase, args.status, (kRoleMma << 8) | 2, tracing, &wait_data);
+          ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tcgen05_fence_after();
           const uint32_t sa = smem_base + stage * C::kStageBytes;
           const uint32_t sb = sa + C::kABytes;
+          if (elect_one()) {
 #pragma unroll
-          for (int k = 0; k < kBK / kUmmaK; ++k) {
-            const uint64_t da = smem_desc(sa + k * (kUmmaK * 2), 16, 1024);
-            const uint64_t db = smem_desc(sb + k * args.b_kstep, args.b_lbo, args.b_sbo);
-            umma_bf16<CG>(d_tmem, da, db, idesc, (uint32_t)((kb | k) != 0));
+            for (int k = 0; k < kBK / kUmmaK; ++k) {
+              const uint64_t da = smem_desc(sa + k * (kUmmaK * 2), 16, 1024);
+              const uint64_t db = smem_desc(sb + k * args.b_kstep, args.b_lbo, args.b_sbo);
+              umma_bf16<CG>(d_tmem, da, db, idesc, (uint32_t)((kb | k) != 0));
+            }
+            umma_commit<CG>(bar_empty + 8 * stage);
           }
-          umma_commit<CG>(bar_empty + 8 * stage);
+          __syncwarp();
           if (++stage == S) { stage = 0; phase ^= 1u; }
         }
-        if (ok) umma_commit<CG>(bar_tfull + 8 * buf);
+        if (ok && elect_one()) umma_commit<CG>(bar_tfull + 8 * buf);
+        __syncwarp();
+        if (tracing && lane == 0) {
+          sp_trace_rec* rec = args.trace + s;
+          rec->mma_wait_data = wait_data; rec->mma_wait_acc = wait_acc; rec->t_mma_issued = globaltimer();
+        }
       }
     }
     __syncwarp();
@@ -373,7 +459,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       const int tm = t / Tn, tn = t - tm * Tn;
       const int buf = it & 1;
       const uint32_t use = (uint32_t)(it >> 1) & 1u;
-      ok = mbar_wait(bar_tfull + 8 * buf, use, args.status, (kRoleEpilogue << 8) | 1);
+      uint32_t wait_epi = 0;
+      ok = mbar_wait_timed(bar_tfull + 8 * buf, use, args.status, (kRoleEpilogue << 8) | 1, args.trace != nullptr, &wait_epi);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tcgen05_fence_after();
@@ -386,7 +473,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         tmem_ld_32x32b_x32(taddr + (uint32_t)(c * 32), v);
         tmem_ld_wait();
         const int col = col_base + c * 32;
-        if (row < args.M && col < args.N) {
+        if (row < args.M && col < args.N && !(args.debug & kDbgNoStores)) {
           if constexpr (OUT_F32) {
             float* dst = reinterpret_cast<float*>(args.C) + (size_t)row * (size_t)args.N + col;
 #pragma unroll
@@ -409,7 +496,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       if (lane == 0) {
         const uint32_t te = bar_tempty + 8 * buf;
         mbar_arrive_cluster(CG == 1 ? te : mapa(te, 0));
-        if (args.trace && rank == 0 && warp == 2) args.trace[s].t_end = globaltimer();
+        if (args.trace && rank == 0 && warp == 2) {
+          args.trace[s].t_end = globaltimer();
+          args.trace[s].epi_wait_acc = wait_epi;
+        }
       }
     }
   }
@@ -564,6 +654,8 @@ int launch_gemm(const GemmCall& call) {
     unsigned l = 0, s = 0, k = 0;
     if (sscanf(e, "%u,%u,%u", &l, &s, &k) == 3) { args.b_lbo = l; args.b_sbo = s; args.b_kstep = k; }
   }
+  args.debug = 0;
+  if (const char* e = getenv("SP_DEBUG_FLAGS")) args.debug = (uint32_t)atoi(e);  // experiments only; wrong results
   args.sched = call.sched;
 
   if (cg == 1) return call.tile_n == 128 ? launch_shape<1, 128>(call, tmA, tmB, args) : launch_shape<1, 256>(call, tmA, tmB, args);

@@ -28,7 +28,7 @@ def test_every_declared_symbol_is_exported():
 
 def test_struct_layout_matches_header():
     assert ctypes.sizeof(binding.SpParams) == 72
-    assert ctypes.sizeof(binding.SpTraceRec) == 32 and binding.TRACE_DTYPE.itemsize == 32
+    assert ctypes.sizeof(binding.SpTraceRec) == 64 and binding.TRACE_DTYPE.itemsize == 64
     assert binding.SpParams.custom_perm.offset == 40 and binding.SpParams.tile_m.offset == 48
 
 
