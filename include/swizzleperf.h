@@ -138,6 +138,31 @@ int sp_gemm_trace(const void* A, const void* B, void* C, int64_t M, int64_t N, i
 int sp_gemm_host(const void* A_host, const void* B_host, void* C_host, int64_t M, int64_t N, int64_t K, int scheme,
                  const sp_params* params, void* stream);
 
+/* sp_gemm for callers that must not allocate device memory.  (The paper has no counterpart: this is a
+ * deployment variant of sp_gemm, same arguments, same result.)
+ *
+ * Who needs it: a process that has given the whole GPU to its own memory pool, where a cudaMalloc made by a
+ * library fails or is charged to a budget nobody planned for; and latency-critical loops, where the
+ * device-wide synchronisation hidden in cudaMalloc / cudaFree is unacceptable.  sp_gemm allocates (once, cached)
+ * a tile table for non-arithmetic orders and a status word; here both live in a fixed array inside the
+ * library image, so this call performs no cudaMalloc, cudaFree or other allocating call.
+ *
+ *   A, B, C, M, N, K, scheme, params, stream : exactly as sp_gemm (DEVICE buffers owned by the caller).
+ *   status_host : HOST, may be NULL.  NULL: the call is asynchronous and an expired device-side wait goes
+ *                 unreported.  Non-NULL: the call synchronises `stream`, stores the raw status word there and
+ *                 returns SP_ERR_TIMEOUT if it is non-zero.
+ * Limits and sharing:
+ *   - at most 65536 tiles (ceil(M/tile_m) * ceil(N/tile_n)); more returns SP_ERR_UNSUPPORTED.  The array
+ *     (about 257 KiB) is held by every GPU context that loads the library until the process exits.
+ *   - every call on a device uses the same array, and the array keeps the previous call's contents: each call
+ *     clears the status word and rewrites the table it needs, on `stream`, before its kernel.  Two calls that
+ *     overlap on the GPU (different streams, or several host threads) race on it; serialise them.
+ *   - the first call on each device looks up the array's device address (with that device current);
+ *     make that first call outside any stream capture.
+ * Errors: as sp_gemm, plus SP_ERR_UNSUPPORTED for too many tiles. */
+int sp_gemm_noalloc(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t K, int scheme,
+                    const sp_params* params, void* stream, int32_t* status_host);
+
 /* Number of persistent CTAs (tile 128xN) or CTA pairs (tile 256xN) sp_gemm launches for T tiles;
  * slot s is run by unit s % units in round s / units.  Returns -1 on error. */
 int sp_gemm_units(int32_t tile_m, int32_t tile_n, int64_t T);

@@ -57,7 +57,7 @@ TRACE_DTYPE = np.dtype([("slot", "<i4"), ("tile", "<i4"), ("smid", "<i4"), ("uni
                         ("mma_wait_acc", "<u4"), ("load_wait_stage", "<u4"), ("epi_wait_acc", "<u4")])
 
 EXPORTS = ["sp_tile_count", "sp_tile_map", "sp_tile_map_device", "sp_gemm", "sp_gemm_trace", "sp_gemm_host",
-           "sp_gemm_units",
+           "sp_gemm_noalloc", "sp_gemm_units",
            "sp_probe_dispatch", "sp_get_status", "sp_last_error", "sp_shutdown"]
 
 
@@ -91,6 +91,8 @@ def lib() -> ctypes.CDLL:
         L.sp_gemm_trace.argtypes = [vp, vp, vp, i64, i64, i64, ctypes.c_int, pp, vp, vp]
         L.sp_gemm_host.restype = ctypes.c_int
         L.sp_gemm_host.argtypes = [vp, vp, vp, i64, i64, i64, ctypes.c_int, pp, vp]
+        L.sp_gemm_noalloc.restype = ctypes.c_int
+        L.sp_gemm_noalloc.argtypes = [vp, vp, vp, i64, i64, i64, ctypes.c_int, pp, vp, ctypes.POINTER(ctypes.c_int32)]
         L.sp_gemm_units.restype = ctypes.c_int
         L.sp_gemm_units.argtypes = [i32, i32, i64]
         L.sp_probe_dispatch.restype = ctypes.c_int
@@ -186,6 +188,18 @@ def gemm(A, B, C, scheme: int = ROW_MAJOR, params: Optional[SpParams] = None, st
     """C = A . B on the current CUDA device under the given tile order (asynchronous)."""
     M, N, K = _dims(A, B, C, params)
     _check(lib().sp_gemm(A.data_ptr(), B.data_ptr(), C.data_ptr(), M, N, K, scheme, _pp(params), _stream_handle(stream)))
+
+
+def gemm_noalloc(A, B, C, scheme: int = ROW_MAJOR, params: Optional[SpParams] = None, stream=None,
+                 check_status: bool = False) -> None:
+    """gemm() that performs no device allocation: its scratch is a fixed array inside the library
+    (at most 65536 tiles; calls on one device must not overlap).  For callers whose device memory is
+    entirely owned by their own pool, or that cannot afford an allocation's hidden synchronisation.
+    With ``check_status`` the call synchronises the stream and raises if a device-side wait expired."""
+    M, N, K = _dims(A, B, C, params)
+    word = ctypes.c_int32(0)
+    _check(lib().sp_gemm_noalloc(A.data_ptr(), B.data_ptr(), C.data_ptr(), M, N, K, scheme, _pp(params),
+                                 _stream_handle(stream), ctypes.byref(word) if check_status else None))
 
 
 def gemm_trace(A, B, C, scheme: int = ROW_MAJOR, params: Optional[SpParams] = None, stream=None) -> np.ndarray:
