@@ -32,7 +32,16 @@ L2_BYTES = 126 * 2 ** 20
 
 # DRAM bytes per launch of the GEMM kernel from the ncu captures summarised under profiles/
 # (dram__bytes_read.sum + dram__bytes_write.sum), keyed by (workload, tile, scheme spec); None = not captured.
-NCU_DRAM_BYTES = {}
+NCU_DRAM_BYTES = {
+    ("cfg3", "256x256", "group_m:8"): 1.200e9,   # profiles/gemm_kernel_cfg3_group_m8_full.md (mean of 2 launches)
+    ("cfg3", "256x256", "row_major"): 2.341e9,   # profiles/l2_hit_rate_per_scheme.md
+    ("cfg3", "256x256", "group_n:8"): 1.228e9,
+    ("cfg3", "256x256", "hilbert"): 1.237e9,
+    ("cfg5", "256x256", "group_m:16"): 1.599e9,
+    ("cfg5", "256x256", "group_m:8"): 2.325e9,
+    ("cfg4", "256x256", "group_n:8"): 0.543e9,
+    ("cfg2", "128x256", "group_m:8"): 0.085e9,
+}
 
 
 def parse_scheme(spec: str):
@@ -213,8 +222,14 @@ def run_ours(args) -> int:
     value = agg["units"] / agg["ms"] / 1e9                      # TFLOP/s, whole job
     clocks = sampler.summary(t_host0, t_host1)
 
-    # burst protocol: isolated launches, best of 10 (how the pool's peak itself was measured)
-    burst_ms = min(time_steps(sp, dA, dB, dC, scheme, p, 1, stream) for _ in range(10))
+    # burst protocol: one launch timed on its own, best of 10 (how the pool's peak itself was measured); the
+    # launch before it keeps the host's launch latency out of the bracket, the sleep lets the clocks recover
+    def one_launch():
+        sp.gemm(dA, dB, dC, scheme, p, stream)
+        ms = time_steps(sp, dA, dB, dC, scheme, p, 1, stream)
+        time.sleep(0.05)
+        return ms
+    burst_ms = min(one_launch() for _ in range(10))
     row_scheme, row_p = params_for("row_major")
     for _ in range(3):
         sp.gemm(dA, dB, dC, row_scheme, row_p, stream)
@@ -250,7 +265,7 @@ def run_ours(args) -> int:
         "traffic": NCU_DRAM_BYTES.get((w.name, f"{tile_m}x{tile_n}", spec)),
         "algorithmic_flops_per_launch": flops,
         "burst": {"achieved": flops / burst_ms / 1e9, "peak": peaks["bf16_tflops"],
-                  "frac": flops / burst_ms / 1e9 / peaks["bf16_tflops"], "protocol": "best of 10 isolated launches"},
+                  "frac": flops / burst_ms / 1e9 / peaks["bf16_tflops"], "protocol": "best of 10 single launches, each queued behind one untimed launch"},
         "frac_of_nominal_2250": achieved / 2250.0,
     }
 
