@@ -63,14 +63,16 @@ def parse_scheme(spec: str):
         return sp.HILBERT, {}
     if name == "xcd":      # xcd:X[:W]  (balanced form)
         return sp.XCD, dict(num_xcds=int(a[1]), wave=int(a[2]) if len(a) > 2 else 0, xcd_balanced=1)
-    if name == "die_split":  # die_split:{m|n}:inner[:G][:i]
+    if name == "die_split":  # die_split:{m|n}:inner[:G][:i][:p]
         inner = {"row_major": sp.ROW_MAJOR, "col_major": sp.COL_MAJOR, "group_m": sp.GROUP_M, "group_n": sp.GROUP_N,
                  "morton": sp.MORTON, "hilbert": sp.HILBERT}[a[2]]
         rest = a[3:]
         inter = int("i" in rest)
         g = [int(v) for v in rest if v.isdigit()]
-        return sp.DIE_SPLIT, dict(split_axis=int(a[1] == "n"), inner_scheme=inner, inner_group=g[0] if g else 1,
-                                  interleave=inter)
+        kw = dict(split_axis=int(a[1] == "n"), inner_scheme=inner, inner_group=g[0] if g else 1, interleave=inter)
+        if "p" in rest:            # units pinned to the L2 half the topology probe found them on
+            kw["flags"] = 2
+        return sp.DIE_SPLIT, kw
     raise ValueError(f"unknown scheme spec {spec!r}")
 
 
@@ -79,10 +81,14 @@ SWEEPS = {
     "cfg2": ["row_major", "group_m:4", "group_m:8", "group_m:16", "hilbert"],
     "cfg3": ["row_major", "col_major", "group_m:2", "group_m:4", "group_m:8", "group_m:16", "group_n:2", "group_n:4",
              "group_n:8", "group_n:16", "morton", "hilbert", "xcd:2:74", "xcd:2", "die_split:m:group_m:8",
-             "die_split:n:group_m:8", "die_split:m:hilbert", "die_split:n:hilbert", "die_split:m:group_m:8:i"],
+             "die_split:n:group_m:8", "die_split:m:hilbert", "die_split:n:hilbert", "die_split:m:group_m:8:i",
+             "die_split:m:group_m:8:p", "die_split:n:group_m:8:p", "die_split:m:group_m:4:p", "die_split:n:group_n:4:p",
+             "die_split:m:hilbert:p", "die_split:m:group_n:8:p", "die_split:n:group_n:8:p", "die_split:m:group_m:16:p"],
     "cfg4": [f"group_m:{g}" for g in (1, 2, 4, 8, 16, 32, 64)] + [f"group_n:{g}" for g in (1, 2, 4, 8)],
     "cfg5": [f"group_m:{g}" for g in (1, 2, 4, 8, 16, 32)] + [f"group_n:{g}" for g in (2, 4, 8, 16, 32)] +
-            ["hilbert", "die_split:m:group_m:8", "die_split:m:hilbert", "die_split:m:group_m:8:i"],
+            ["hilbert", "die_split:m:group_m:8", "die_split:m:hilbert", "die_split:m:group_m:8:i",
+             "die_split:m:group_m:8:p", "die_split:m:group_m:16:p", "die_split:n:group_n:16:p", "die_split:m:hilbert:p",
+             "die_split:n:group_m:16:p", "die_split:m:group_n:16:p"],
 }
 DEFAULT_SCHEME = {"cfg1": "group_m:2", "cfg2": "group_m:8", "cfg3": "group_m:8", "cfg4": "group_n:2", "cfg5": "group_m:8"}
 

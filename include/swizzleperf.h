@@ -59,7 +59,11 @@ typedef enum {
 } sp_scheme;
 
 /* sp_params.flags */
-#define SP_FLAG_TRACE 1u /* reserved for sp_gemm_trace */
+#define SP_FLAG_TRACE 1u      /* reserved for sp_gemm_trace */
+#define SP_FLAG_DIE_PINNED 2u /* sp_gemm* with SP_DIE_SPLIT, interleave = 0: the persistent units whose SM sits on L2 half d
+                                 (measured by the topology probe, cached) run only the slots of half d of the tile space,
+                                 in arrival order on that half.  Needs at least as many tiles as SMs / CTAs-per-tile;
+                                 SP_ERR_UNSUPPORTED if the probe finds no usable two-way structure.  The output is the same. */
 
 typedef struct {
   uint32_t struct_size;       /* must be sizeof(sp_params)                                                  */
@@ -76,7 +80,7 @@ typedef struct {
                               /*   pair per tile); 0,0 = 256x256.  Ignored by sp_tile_map*.                 */
   int32_t out_dtype;          /* sp_gemm*: 0 = C is bf16 (round to nearest even), 1 = C is fp32             */
   int32_t b_layout;           /* sp_gemm*: 0 = B is K x N row-major, 1 = B is N x K row-major               */
-  uint32_t flags;             /* 0                                                                          */
+  uint32_t flags;             /* 0, or SP_FLAG_DIE_PINNED                                                   */
 } sp_params;
 
 /* One record per tile, written by sp_gemm_trace. */
@@ -171,6 +175,18 @@ int sp_gemm_units(int32_t tile_m, int32_t tile_n, int64_t T);
  * launches `n_blocks` trivial blocks in clusters of `cluster` (1 or 2) and records for block b
  *   smid_host[b] = %smid, start_host[b] = %globaltimer at entry.  HOST arrays of n_blocks. Synchronous. */
 int sp_probe_dispatch(int32_t n_blocks, int32_t cluster, int32_t* smid_host, uint64_t* start_host);
+
+/* Topology probe (counterpart of the paper's parsed hardware context: number of XCDs, their L2s).
+ * Every SM in turn times first-touch loads of the same SP_PROBE_LINES cache lines, each rewritten before the
+ * round; SMs whose fast/slow pattern over the lines agrees share an L2 half (die).
+ *   sm_to_die_host : HOST, capacity >= 1024 int32; entry [smid] = 0 or 1 (group 0 contains the lowest measured SM),
+ *                    -1 if that SM could not be measured.
+ *   n_sm           : HOST, receives the SM count.
+ *   confidence     : HOST, mean |agreement| in [0,1]; near 0 means no measurable two-way structure.
+ *   lat_host       : HOST, may be NULL; else n_sm * SP_PROBE_LINES uint32 minimum latencies in SM cycles.
+ * Synchronous; allocates and frees its own buffers; takes a fraction of a second. */
+#define SP_PROBE_LINES 256
+int sp_probe_topology(int32_t* sm_to_die_host, int32_t* n_sm, float* confidence, uint32_t* lat_host);
 
 /* Synchronises `stream`, then returns and clears the device status word of the current device:
  * SP_OK, or SP_ERR_TIMEOUT if a kernel gave up on a bounded wait since the last call.

@@ -58,7 +58,7 @@ TRACE_DTYPE = np.dtype([("slot", "<i4"), ("tile", "<i4"), ("smid", "<i4"), ("uni
 
 EXPORTS = ["sp_tile_count", "sp_tile_map", "sp_tile_map_device", "sp_gemm", "sp_gemm_trace", "sp_gemm_host",
            "sp_gemm_noalloc", "sp_gemm_units",
-           "sp_probe_dispatch", "sp_get_status", "sp_last_error", "sp_shutdown"]
+           "sp_probe_dispatch", "sp_probe_topology", "sp_get_status", "sp_last_error", "sp_shutdown"]
 
 
 class SpError(RuntimeError):
@@ -97,6 +97,8 @@ def lib() -> ctypes.CDLL:
         L.sp_gemm_units.argtypes = [i32, i32, i64]
         L.sp_probe_dispatch.restype = ctypes.c_int
         L.sp_probe_dispatch.argtypes = [i32, i32, vp, vp]
+        L.sp_probe_topology.restype = ctypes.c_int
+        L.sp_probe_topology.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_float), vp]
         L.sp_get_status.restype = ctypes.c_int
         L.sp_get_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32)]
         L.sp_last_error.restype = ctypes.c_char_p
@@ -248,6 +250,19 @@ def probe_dispatch(n_blocks: int, cluster: int = 1):
     start = np.zeros(n_blocks, dtype=np.uint64)
     _check(lib().sp_probe_dispatch(n_blocks, cluster, smid.ctypes.data, start.ctypes.data))
     return smid, start
+
+
+PROBE_LINES = 256
+
+
+def probe_topology():
+    """(sm_to_die[n_sm], confidence, latencies[n_sm, PROBE_LINES]) from the L2-latency probe."""
+    die = np.full(1024, -1, dtype=np.int32)
+    lat = np.zeros(1024 * PROBE_LINES, dtype=np.uint32)
+    n = ctypes.c_int32(0)
+    conf = ctypes.c_float(0)
+    _check(lib().sp_probe_topology(die.ctypes.data, ctypes.byref(n), ctypes.byref(conf), lat.ctypes.data))
+    return die[:n.value].copy(), float(conf.value), lat[:n.value * PROBE_LINES].reshape(n.value, PROBE_LINES).copy()
 
 
 def get_status(stream=None) -> int:

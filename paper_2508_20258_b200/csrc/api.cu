@@ -141,6 +141,9 @@ struct DeviceState {
   int device = -1;
   int32_t* status = nullptr;
   std::vector<TableEntry> tables;
+  int die_known = 0;            // 0: not probed, 1: usable map, -1: probe found no two-way structure
+  int sms_on_die[2] = {0, 0};
+  uint32_t die_mask[8] = {};
   void* staging = nullptr;      // device copies of A, B, C for sp_gemm_host (grow-only)
   size_t staging_bytes = 0;
 };
@@ -206,9 +209,34 @@ static int current_device(int* dev) {
 
 static int get_status_word(DeviceState* ds) {
   if (!ds->status) {
-    SP_CUDA(cudaMalloc(&ds->status, sizeof(int32_t)));
-    SP_CUDA(cudaMemset(ds->status, 0, sizeof(int32_t)));
+    SP_CUDA(cudaMalloc(&ds->status, 4 * sizeof(int32_t)));   // status word, two die counters, spare
+    SP_CUDA(cudaMemset(ds->status, 0, 4 * sizeof(int32_t)));
   }
+  return SP_OK;
+}
+
+// SM -> L2-half map of the device, probed once.  Usable only if the probe is confident, the halves
+// are equal and the two SMs of every CTA pair share a half.
+static int get_die_map(DeviceState* ds) {
+  if (ds->die_known == 0) {
+    std::vector<int32_t> die(1024, -1);
+    int n = 0;
+    float conf = 0.f;
+    int rc = probe_topology(die.data(), &n, &conf, nullptr);
+    if (rc != SP_OK) return rc;
+    bool ok = conf >= 0.8f && n <= 256;
+    int cnt[2] = {0, 0};
+    for (int i = 0; i < n && ok; ++i) {
+      if (die[i] < 0) { ok = false; break; }
+      cnt[die[i]]++;
+      if (die[i]) ds->die_mask[i >> 5] |= 1u << (i & 31);
+      if ((i & 1) && die[i] != die[i - 1]) ok = false;
+    }
+    ok = ok && cnt[0] > 0 && cnt[1] > 0 && (cnt[0] % 2) == 0 && (cnt[1] % 2) == 0;
+    ds->sms_on_die[0] = cnt[0]; ds->sms_on_die[1] = cnt[1];
+    ds->die_known = ok ? 1 : -1;
+  }
+  if (ds->die_known < 0) { set_error("the topology probe found no usable two-way L2 structure on this device"); return SP_ERR_UNSUPPORTED; }
   return SP_OK;
 }
 
@@ -292,6 +320,18 @@ static int gemm_common(const void* A, const void* B, void* C, int64_t M, int64_t
   if (call.sched.use_table) {
     rc = get_table(ds, call.sched, host_perm, scheme == kCustom, call.stream, &call.perm_dev);
     if (rc != SP_OK) return rc;
+  }
+  if (params && (params->flags & SP_FLAG_DIE_PINNED)) {
+    if (scheme != kDieSplit || call.sched.interleave) {
+      set_error("SP_FLAG_DIE_PINNED needs SP_DIE_SPLIT with interleave = 0");
+      return SP_ERR_INVALID_ARG;
+    }
+    rc = get_die_map(ds);
+    if (rc != SP_OK) return rc;
+    call.pinned = 1;
+    call.half0 = die_split_half0(call.sched);
+    call.sms_on_die[0] = ds->sms_on_die[0]; call.sms_on_die[1] = ds->sms_on_die[1];
+    for (int i = 0; i < 8; ++i) call.die_mask[i] = ds->die_mask[i];
   }
   return launch_gemm(call);
 }
@@ -405,6 +445,14 @@ int sp_probe_dispatch(int32_t n_blocks, int32_t cluster, int32_t* smid_host, uin
   int rc = current_device(&dev);
   if (rc != SP_OK) return rc;
   return probe_dispatch(n_blocks, cluster, smid_host, start_host);
+}
+
+int sp_probe_topology(int32_t* sm_to_die_host, int32_t* n_sm, float* confidence, uint32_t* lat_host) {
+  if (!sm_to_die_host || !n_sm || !confidence) { set_error("bad probe arguments"); return SP_ERR_INVALID_ARG; }
+  int dev = 0;
+  int rc = current_device(&dev);
+  if (rc != SP_OK) return rc;
+  return probe_topology(sm_to_die_host, n_sm, confidence, lat_host);
 }
 
 int sp_get_status(void* stream, int32_t* detail) {

@@ -56,6 +56,12 @@ struct GemmArgs {
   int units;
   uint32_t b_lbo, b_sbo, b_kstep;  // B operand descriptor strides in bytes
   uint32_t debug;                  // experiment switches (SP_DEBUG_FLAGS); 0 in normal use
+  // Die-pinned scheduling (SP_DIE_SPLIT with SP_FLAG_DIE_PINNED): units on L2 half d run the slots of half d only.
+  int pinned;                      // 0: slot s runs on unit s % units
+  int half0;                       // number of slots in half 0 (queue boundary)
+  int units_on_die[2];             // persistent units per die (all SMs host one CTA each)
+  int32_t* die_count;              // two device counters, zero at launch: arrival rank of a unit on its die
+  uint32_t die_mask[8];            // bit smid = die of that SM (from the topology probe)
   Sched sched;
 };
 
@@ -308,10 +314,35 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     tmem_alloc<CG>(tmem_slot, kTmemCols);
     tmem_relinquish<CG>();
   }
+  const uint32_t sched_slot = tmem_slot + 8;       // 2 words: die, rank on that die
+  if (args.pinned && threadIdx.x == 32 * 2 && rank == 0) {
+    // the leader learns which L2 half its SM belongs to and takes the next rank there;
+    // both CTAs of the unit read the pair of words after the start-up barrier
+    uint32_t smid;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+    const uint32_t die = (args.die_mask[(smid >> 5) & 7] >> (smid & 31)) & 1u;
+    const uint32_t r = (uint32_t)atomicAdd(args.die_count + die, 1);
+#pragma unroll
+    for (uint32_t c = 0; c < (uint32_t)CG; ++c) {
+      const uint32_t dst = CG == 1 ? sched_slot : mapa(sched_slot, c);
+      asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(dst), "r"(die) : "memory");
+      asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(dst + 4), "r"(r) : "memory");
+    }
+  }
   tcgen05_fence_before();
   unit_sync<CG>();
   tcgen05_fence_after();
   const uint32_t tmem_base = *tmem_slot_ptr;
+
+  // slots of this unit: s_first, s_first + s_step, ... below s_end
+  int s_first = unit, s_step = args.units, s_end = T;
+  if (args.pinned) {
+    const uint32_t die = tmem_slot_ptr[2], r = tmem_slot_ptr[3];
+    s_step = args.units_on_die[die];
+    s_first = (die ? args.half0 : 0) + (int)r;
+    s_end = die ? T : args.half0;
+    if ((int)r >= s_step) s_first = s_end;           // more arrivals than the probe predicted: this unit idles
+  }
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer
@@ -321,7 +352,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int s = unit; s < T && ok; s += args.units) {
+      for (int s = s_first; s < s_end && ok; s += s_step) {
         const int t = tile_of_slot(args, s);
         const int tm = t / Tn, tn = t - tm * Tn;
         const int row0 = tm * TILE_M + (int)rank * 128;
@@ -386,7 +417,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       uint32_t phase = 0;
       int it = 0;
       bool ok = true;
-      for (int s = unit; s < T && ok; s += args.units, ++it) {
+      for (int s = s_first; s < s_end && ok; s += s_step, ++it) {
         const int buf = it & 1;
         const uint32_t use = (uint32_t)(it >> 1) & 1u;
         const bool tracing = args.trace != nullptr;
@@ -454,7 +485,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const int quarter = warp & 3;  // TMEM lanes [32*quarter, 32*quarter + 32) are this warp's
     int it = 0;
     bool ok = true;
-    for (int s = unit; s < T && ok; s += args.units, ++it) {
+    for (int s = s_first; s < s_end && ok; s += s_step, ++it) {
       const int t = tile_of_slot(args, s);
       const int tm = t / Tn, tn = t - tm * Tn;
       const int buf = it & 1;
@@ -653,6 +684,24 @@ int launch_gemm(const GemmCall& call) {
   if (const char* e = getenv("SP_DEBUG_BDESC")) {  // bring-up only: "lbo,sbo,kstep" in bytes
     unsigned l = 0, s = 0, k = 0;
     if (sscanf(e, "%u,%u,%u", &l, &s, &k) == 3) { args.b_lbo = l; args.b_sbo = s; args.b_kstep = k; }
+  }
+  args.pinned = 0; args.half0 = 0; args.units_on_die[0] = args.units_on_die[1] = 0; args.die_count = nullptr;
+  for (int i = 0; i < 8; ++i) args.die_mask[i] = 0;
+  if (call.pinned) {
+    const int cg_ = call.tile_m / 128;
+    args.pinned = 1;
+    args.half0 = call.half0;
+    args.units_on_die[0] = call.sms_on_die[0] / cg_;
+    args.units_on_die[1] = call.sms_on_die[1] / cg_;
+    args.die_count = call.status_dev + 1;
+    for (int i = 0; i < 8; ++i) args.die_mask[i] = call.die_mask[i];
+    if (args.units != args.units_on_die[0] + args.units_on_die[1]) {
+      set_error("die-pinned scheduling needs every SM to host one CTA (%d units launched, %d expected)", args.units,
+                args.units_on_die[0] + args.units_on_die[1]);
+      return SP_ERR_UNSUPPORTED;
+    }
+    cudaError_t ce = cudaMemsetAsync(args.die_count, 0, 2 * sizeof(int32_t), call.stream);
+    if (ce != cudaSuccess) { set_error("clearing the die counters failed: %s", cudaGetErrorString(ce)); return SP_ERR_CUDA; }
   }
   args.debug = 0;
   if (const char* e = getenv("SP_DEBUG_FLAGS")) args.debug = (uint32_t)atoi(e);  // experiments only; wrong results

@@ -37,7 +37,11 @@ struct GemmCall {
   int b_nk;
   Sched sched;
   const int32_t* perm_dev;  // table for non-arithmetic schemes, else nullptr
-  int32_t* status_dev;
+  int32_t* status_dev;      // 4 device words: status, die counter 0, die counter 1, spare
+  int pinned;               // die-pinned scheduling (SP_DIE_SPLIT + SP_FLAG_DIE_PINNED)
+  int half0;                // slots in half 0
+  int sms_on_die[2];
+  uint32_t die_mask[8];
   sp_trace_rec* trace_dev;  // nullptr unless tracing
   cudaStream_t stream;
 };
@@ -48,5 +52,10 @@ int gemm_units(int tile_m, int tile_n, int64_t T);
 int launch_gemm(const GemmCall& call);
 
 int probe_dispatch(int n_blocks, int cluster, int32_t* smid_host, uint64_t* start_host);
+int probe_topology(int32_t* sm_to_die_host, int32_t* n_sm, float* confidence, uint32_t* lat_host);
+// Size of half 0 of a DIE_SPLIT schedule, in slots.
+inline int die_split_half0(const Sched& c) {
+  return c.axis == 0 ? ((c.Tm + 1) / 2) * c.Tn : ((c.Tn + 1) / 2) * c.Tm;
+}
 
 }  // namespace sp

@@ -51,6 +51,7 @@ def test_scheme_specs_parse():
     assert bench.parse_scheme("xcd:2:74") == (sp.XCD, dict(num_xcds=2, wave=74, xcd_balanced=1))
     assert bench.parse_scheme("die_split:n:group_m:8:i") == (
         sp.DIE_SPLIT, dict(split_axis=1, inner_scheme=sp.GROUP_M, inner_group=8, interleave=1))
+    assert bench.parse_scheme("die_split:m:group_m:8:p")[1]["flags"] == 2
     for name, specs in bench.SWEEPS.items():
         for s in specs:
             bench.parse_scheme(s)

@@ -201,3 +201,47 @@ def test_runtime_rejections_launch_nothing():
     torch.cuda.synchronize()
     assert (C == 7.0).all()
     assert sp.get_status() == 0
+
+
+def test_die_pinned_schedule_keeps_each_half_on_one_l2_half():
+    """SP_FLAG_DIE_PINNED: units run only the slots of the tile-space half that matches the L2 half
+    (die) their SM was measured on; every tile still runs exactly once and C has the same bits."""
+    die, conf, _ = sp.probe_topology()
+    if conf < 0.8 or (die < 0).any():
+        pytest.skip("no two-way L2 structure measured on this device")
+    M = N = 8192
+    K = 256
+    A, B = synth.make_int_inputs(M, N, K, seed=8)
+    dA, dB = dev_bf16(A), dev_bf16(B)
+    ref = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    sp.gemm(dA, dB, ref, sp.ROW_MAJOR, sp.make_params(tile_m=256, tile_n=256))
+    for tile in [(256, 256), (128, 256)]:
+        for axis in (0, 1):
+            kw = dict(split_axis=axis, inner_scheme=sp.GROUP_M, inner_group=4)
+            p = sp.make_params(tile_m=tile[0], tile_n=tile[1], flags=2, **kw)
+            dC = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+            tr = sp.gemm_trace(dA, dB, dC, sp.DIE_SPLIT, p)
+            assert sp.get_status() == 0
+            assert torch.equal(dC.view(torch.int16), ref.view(torch.int16))
+            want = R.tile_map(M, N, tile[0], tile[1], sp.DIE_SPLIT, R.Params(**kw))
+            assert tr["tile"].tolist() == want                       # record s still describes slot s
+            h0 = len(R.die_split_halves(-(-M // tile[0]), -(-N // tile[1]), axis, sp.GROUP_M, 4)[0])
+            on_die = die[tr["smid"]]
+            assert len(set(on_die[:h0].tolist())) == 1 and len(set(on_die[h0:].tolist())) == 1
+            assert on_die[0] != on_die[-1]
+    with pytest.raises(sp.SpError) as e:                              # pinning is defined for the split order only
+        sp.gemm(dA, dB, ref, sp.GROUP_M, sp.make_params(tile_m=256, tile_n=256, group=4, flags=2))
+    assert e.value.status == sp.ERR_INVALID_ARG
+
+
+def test_topology_probe_finds_two_equal_l2_halves_and_pairs_stay_together():
+    die, conf, lat = sp.probe_topology()
+    assert len(die) == torch.cuda.get_device_properties(0).multi_processor_count
+    assert lat.shape == (len(die), 256) and (lat > 0).all()
+    if conf < 0.8:
+        pytest.skip("no two-way L2 structure measured on this device")
+    assert set(die.tolist()) == {0, 1} and (die == 0).sum() == (die == 1).sum()
+    assert (die[0::2] == die[1::2]).all()          # the two SMs of a CTA pair share a half
+    near = np.median(lat[die == 0][:, :], axis=0)  # per line: latency seen from half 0 ...
+    far = np.median(lat[die == 1][:, :], axis=0)   # ... and from half 1: one of them is the home half
+    assert (np.maximum(near, far) > 1.5 * np.minimum(near, far)).mean() > 0.9
