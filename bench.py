@@ -252,6 +252,23 @@ def run_ours(args) -> int:
         sp.gemm(dA, dB, dC, row_scheme, row_p, stream)
     row_ms = time_steps(sp, dA, dB, dC, row_scheme, row_p, args.steps, stream) / args.steps
 
+    # context only: cuBLAS (torch.matmul) on the same tensors, same back-to-back protocol, same thermal state
+    cublas = None
+    if dC.dtype == torch.bfloat16 and not b_nk:
+        ref = torch.empty_like(dC)
+        for _ in range(3):
+            torch.matmul(dA, dB, out=ref)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.steps):
+            torch.matmul(dA, dB, out=ref)
+        e1.record(stream)
+        e1.synchronize()
+        cublas = {"tflops": flops * args.steps / e0.elapsed_time(e1) / 1e9, "note": "torch.matmul, context only, not a target"}
+        del ref
+        ours_again = time_steps(sp, dA, dB, dC, scheme, p, args.steps, stream) / args.steps
+        cublas["ours_right_after_tflops"] = flops / ours_again / 1e9
+
     # end to end through the C ABI with host buffers (pinned): H2D of A and B, kernel, D2H of C, every step
     e2e = None
     if not args.no_e2e:
@@ -309,6 +326,7 @@ def run_ours(args) -> int:
                        "parallelism": "replicas only" if world > 1 else "1 GPU"},
             "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": args.steps,
             "clocks": clocks,
+            "cublas_context": cublas,
             "row_major": {"ms_per_step": row_ms, "tflops": flops / row_ms / 1e9, "speedup_of_scheme": row_ms / launch_ms},
         }
         print(json.dumps(line), flush=True)

@@ -55,7 +55,6 @@ struct GemmArgs {
   int kblocks;
   int units;
   uint32_t b_lbo, b_sbo, b_kstep;  // B operand descriptor strides in bytes
-  uint32_t debug;                  // experiment switches (SP_DEBUG_FLAGS); 0 in normal use
   // Die-pinned scheduling (SP_DIE_SPLIT with SP_FLAG_DIE_PINNED): units on L2 half d run the slots of half d only.
   int pinned;                      // 0: slot s runs on unit s % units
   int half0;                       // number of slots in half 0 (queue boundary)
@@ -65,14 +64,6 @@ struct GemmArgs {
   Sched sched;
 };
 
-// Experiment switches: results are wrong by design when any of these is set.
-enum : uint32_t {
-  kDbgSameOperands = 1u,   // every load fetches the first k-block of the first tile (all L2 hits)
-  kDbgNoStores = 2u,       // epilogue reads TMEM but stores nothing
-  kDbgNoLoads = 4u,        // producer issues no copies; stages are handed over empty
-  kDbgFreeRunMma = 8u,     // no producer at all; the MMA issuer ignores the stage barriers (pure issue rate)
-  kDbgSplitN = 16u,        // with kDbgFreeRunMma: two N/2 MMAs into two accumulators instead of one N-wide MMA
-};
 
 // status word: (role << 8) | which wait
 enum : int { kRoleProducer = 1, kRoleMma = 2, kRoleEpilogue = 3 };
@@ -348,7 +339,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     // ---------------------------------------------------------------- TMA producer
     // The whole warp walks the loop (uniform control flow, uniform operands); one elected
     // lane issues the copies.
-    if (!(args.debug & kDbgFreeRunMma)) {
+    {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
@@ -373,21 +364,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           const uint32_t full_leader = CG == 1 ? full_local : mapa(full_local, 0);
           const uint32_t sa = smem_base + stage * C::kStageBytes;
           const uint32_t sb = sa + C::kABytes;
-          const bool same = (args.debug & kDbgSameOperands) != 0;
-          const int kx = same ? 0 : kb * kBK, ry = same ? (int)rank * 128 : row0, cx = same ? (int)rank * C::kBCols : col0;
           if (elect_one()) {
-            if (args.debug & kDbgNoLoads) {
-              if (rank == 0) mbar_arrive_expect_tx(full_local, 0);
+            if (rank == 0) mbar_arrive_expect_tx(full_local, CG * C::kStageBytes);
+            tma_load_2d<CG>(sa, &tmA, kb * kBK, row0, full_leader);
+            if constexpr (B_NK) {
+              tma_load_2d<CG>(sb, &tmB, kb * kBK, col0, full_leader);
             } else {
-              if (rank == 0) mbar_arrive_expect_tx(full_local, CG * C::kStageBytes);
-              tma_load_2d<CG>(sa, &tmA, kx, ry, full_leader);
-              if constexpr (B_NK) {
-                tma_load_2d<CG>(sb, &tmB, kx, cx, full_leader);
-              } else {
 #pragma unroll
-                for (int j = 0; j < C::kBCols / 64; ++j)
-                  tma_load_2d<CG>(sb + j * (64 * kBK * 2), &tmB, cx + j * 64, kx, full_leader);
-              }
+              for (int j = 0; j < C::kBCols / 64; ++j)
+                tma_load_2d<CG>(sb + j * (64 * kBK * 2), &tmB, col0 + j * 64, kb * kBK, full_leader);
             }
           }
           __syncwarp();
@@ -428,30 +413,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         tcgen05_fence_after();
         if (tracing && lane == 0) args.trace[s].t_mma_begin = globaltimer();
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
-        if (args.debug & kDbgFreeRunMma) {
-          constexpr uint32_t idesc_half = make_idesc(TILE_M, BN / 2, !B_NK);
-          for (int kb = 0; kb < KB; ++kb) {
-            const uint32_t sa = smem_base + (kb % S) * C::kStageBytes;
-            const uint32_t sb = sa + C::kABytes;
-            if (elect_one()) {
-#pragma unroll
-              for (int k = 0; k < kBK / kUmmaK; ++k) {
-                const uint64_t da = smem_desc(sa + k * (kUmmaK * 2), 16, 1024);
-                const uint64_t db = smem_desc(sb + k * args.b_kstep, args.b_lbo, args.b_sbo);
-                if (args.debug & kDbgSplitN) {
-                  umma_bf16<CG>(d_tmem, da, db, idesc_half, (uint32_t)((kb | k) != 0));
-                  umma_bf16<CG>(d_tmem + BN / 2, da, db, idesc_half, (uint32_t)((kb | k) != 0));
-                } else {
-                  umma_bf16<CG>(d_tmem, da, db, idesc, (uint32_t)((kb | k) != 0));
-                }
-              }
-            }
-            __syncwarp();
-          }
-          if (elect_one()) umma_commit<CG>(bar_tfull + 8 * buf);
-          __syncwarp();
-          continue;
-        }
         for (int kb = 0; kb < KB; ++kb) {
           ok = mbar_wait_timed(bar_full + 8 * stage, phase, args.status, (kRoleMma << 8) | 2, tracing, &wait_data);
           ok = __all_sync(0xffffffffu, ok);
@@ -504,7 +465,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         tmem_ld_32x32b_x32(taddr + (uint32_t)(c * 32), v);
         tmem_ld_wait();
         const int col = col_base + c * 32;
-        if (row < args.M && col < args.N && !(args.debug & kDbgNoStores)) {
+        if (row < args.M && col < args.N) {
           if constexpr (OUT_F32) {
             float* dst = reinterpret_cast<float*>(args.C) + (size_t)row * (size_t)args.N + col;
 #pragma unroll
@@ -681,10 +642,6 @@ int launch_gemm(const GemmCall& call) {
     // (stride offset); the next 64 n live in the next box, 8192 bytes on (leading offset)
     args.b_lbo = 64 * kBK * 2; args.b_sbo = 1024; args.b_kstep = kUmmaK * 128;
   }
-  if (const char* e = getenv("SP_DEBUG_BDESC")) {  // bring-up only: "lbo,sbo,kstep" in bytes
-    unsigned l = 0, s = 0, k = 0;
-    if (sscanf(e, "%u,%u,%u", &l, &s, &k) == 3) { args.b_lbo = l; args.b_sbo = s; args.b_kstep = k; }
-  }
   args.pinned = 0; args.half0 = 0; args.units_on_die[0] = args.units_on_die[1] = 0; args.die_count = nullptr;
   for (int i = 0; i < 8; ++i) args.die_mask[i] = 0;
   if (call.pinned) {
@@ -703,8 +660,6 @@ int launch_gemm(const GemmCall& call) {
     cudaError_t ce = cudaMemsetAsync(args.die_count, 0, 2 * sizeof(int32_t), call.stream);
     if (ce != cudaSuccess) { set_error("clearing the die counters failed: %s", cudaGetErrorString(ce)); return SP_ERR_CUDA; }
   }
-  args.debug = 0;
-  if (const char* e = getenv("SP_DEBUG_FLAGS")) args.debug = (uint32_t)atoi(e);  // experiments only; wrong results
   args.sched = call.sched;
 
   if (cg == 1) return call.tile_n == 128 ? launch_shape<1, 128>(call, tmA, tmB, args) : launch_shape<1, 256>(call, tmA, tmB, args);
