@@ -46,10 +46,13 @@ def sample_tiles(Tm, Tn, seed):
 
 
 CASES = [
+    # the die-pinned split (flags=2) is the order the benchmark times on cfg3 and cfg5
     ("cfg3", [(sp.ROW_MAJOR, {}), (sp.GROUP_M, dict(group=8)), (sp.HILBERT, {}),
-              (sp.DIE_SPLIT, dict(split_axis=0, inner_scheme=sp.GROUP_M, inner_group=8))]),
-    ("cfg4", [(sp.GROUP_M, dict(group=4)), (sp.GROUP_N, dict(group=2))]),
-    ("cfg5", [(sp.GROUP_M, dict(group=16)), (sp.HILBERT, {})]),
+              (sp.DIE_SPLIT, dict(split_axis=0, inner_scheme=sp.GROUP_M, inner_group=8)),
+              (sp.DIE_SPLIT, dict(split_axis=0, inner_scheme=sp.GROUP_M, inner_group=8, flags=2))]),
+    ("cfg4", [(sp.ROW_MAJOR, {}), (sp.GROUP_M, dict(group=4)), (sp.GROUP_N, dict(group=2))]),
+    ("cfg5", [(sp.GROUP_M, dict(group=16)), (sp.HILBERT, {}),
+              (sp.DIE_SPLIT, dict(split_axis=0, inner_scheme=sp.GROUP_M, inner_group=8, flags=2))]),
 ]
 
 
@@ -74,7 +77,12 @@ def test_large_workload_sampled(name, schemes):
     for scheme, kw in schemes:
         dC.fill_(float("nan"))
         p = sp.make_params(tile_m=w.tile_m, tile_n=w.tile_n, out_dtype=0, **kw)
-        sp.gemm(dA, dB, dC, scheme, p)
+        try:
+            sp.gemm(dA, dB, dC, scheme, p)
+        except sp.SpError as err:
+            if kw.get("flags") and err.status == sp.ERR_UNSUPPORTED:
+                continue                      # no two-way L2 structure measured on this device
+            raise
         assert sp.get_status() == 0
         bits = dC.view(torch.int16).cpu().numpy().view(np.uint16)
         got_rows = G.bf16_bits_to_f64(bits[rows, :])
