@@ -8,7 +8,8 @@
 //   warp 0  lane 0 : TMA producer   -- A and B k-blocks into a ring of 128B-swizzled smem stages
 //   warp 1  lane 0 : MMA issuer     -- tcgen05.mma, fp32 accumulators in TMEM (two buffers);
 //                                      the warp also owns TMEM alloc / dealloc
-//   warps 2..5     : epilogue       -- tcgen05.ld, convert, 16-byte global stores, ragged-edge predication
+//   warps 2..5     : epilogue       -- tcgen05.ld, convert, stage 32 rows x 128 bytes per warp in swizzled smem,
+//                                      TMA store (full 128-byte rows; ragged edges clipped by the tensor map)
 //
 // Synchronisation: mbarriers only.  full[s]/empty[s] per smem stage, tmem_full[b]/tmem_empty[b]
 // per accumulator buffer.  In pair mode the barriers that feed the MMA issuer live in the
@@ -41,9 +42,10 @@ struct Cfg {
   static constexpr uint32_t kABytes = 128 * kBK * 2;            // 128 rows of A
   static constexpr uint32_t kBBytes = kBCols * kBK * 2;
   static constexpr uint32_t kStageBytes = kABytes + kBBytes;
-  static constexpr int kFit = (kSmemLimit - kBarrierBytes - 1024) / kStageBytes;
+  static constexpr uint32_t kEpiBytes = 4 * 2 * 4096;           // per epilogue warp: two 32-row x 128-byte staging buffers
+  static constexpr int kFit = (kSmemLimit - kBarrierBytes - 1024 - kEpiBytes) / kStageBytes;
   static constexpr int kStages = kFit > 8 ? 8 : kFit;
-  static constexpr uint32_t kSmemBytes = kStages * kStageBytes + kBarrierBytes + 1024;  // + alignment slack
+  static constexpr uint32_t kSmemBytes = kStages * kStageBytes + kEpiBytes + kBarrierBytes + 1024;  // + alignment slack
 };
 
 struct GemmArgs {
@@ -172,6 +174,20 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
   }
 }
 
+// Store a box from shared memory to the tensor described by `map` (clipped at its edges), bulk-group completion.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(map), "r"(x), "r"(y), "r"(src)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void st_shared_16(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
 __device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -275,14 +291,16 @@ __device__ __forceinline__ uint32_t pack_bf16(uint32_t lo_bits, uint32_t hi_bits
 // ------------------------------------------------------------------ the kernel
 template <int CG, int BN, bool B_NK, bool OUT_F32>
 __global__ void __launch_bounds__(kThreads, 1)
-gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmArgs args) {
+gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+            const __grid_constant__ CUtensorMap tmC, const GemmArgs args) {
   using C = Cfg<CG, BN>;
   constexpr int S = C::kStages;
   constexpr int TILE_M = 128 * CG;
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t bar_base = smem_base + S * C::kStageBytes;
+  const uint32_t epi_base = smem_base + S * C::kStageBytes;   // 1024-byte aligned: the store's 128-byte swizzle needs it
+  const uint32_t bar_base = epi_base + C::kEpiBytes;
   const uint32_t bar_full = bar_base;              // S barriers
   const uint32_t bar_empty = bar_base + 8 * S;     // S barriers
   const uint32_t bar_tfull = bar_base + 16 * S;    // 2 barriers
@@ -445,6 +463,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     // ---------------------------------------------------------------- epilogue
     const int quarter = warp & 3;  // TMEM lanes [32*quarter, 32*quarter + 32) are this warp's
     int it = 0;
+    int chunk = 0;                 // staging buffers alternate per stored chunk, across tiles
     bool ok = true;
     for (int s = s_first; s < s_end && ok; s += s_step, ++it) {
       const int t = tile_of_slot(args, s);
@@ -456,31 +475,43 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tcgen05_fence_after();
-      const int row = tm * TILE_M + (int)rank * 128 + quarter * 32 + lane;
+      const int row0 = tm * TILE_M + (int)rank * 128 + quarter * 32;   // first of this warp's 32 rows
       const int col_base = tn * BN;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN);
+      constexpr int kChunkCols = OUT_F32 ? 32 : 64;                    // 128 bytes of output per row
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        uint32_t v[32];
-        tmem_ld_32x32b_x32(taddr + (uint32_t)(c * 32), v);
+      for (int c = 0; c < BN / kChunkCols; ++c, ++chunk) {
+        uint32_t v[32], w[32];
+        tmem_ld_32x32b_x32(taddr + (uint32_t)(c * kChunkCols), v);
+        if constexpr (!OUT_F32) tmem_ld_32x32b_x32(taddr + (uint32_t)(c * kChunkCols + 32), w);
         tmem_ld_wait();
-        const int col = col_base + c * 32;
-        if (row < args.M && col < args.N) {
-          if constexpr (OUT_F32) {
-            float* dst = reinterpret_cast<float*>(args.C) + (size_t)row * (size_t)args.N + col;
+        // the buffer used two chunks ago must have been read by its store before it is overwritten
+        if (chunk >= 2) {
+          if (lane == 0) bulk_wait_read_1();
+          __syncwarp();
+        }
+        const uint32_t slice = epi_base + (uint32_t)((warp - 2) * 8192 + (chunk & 1) * 4096);
+        const uint32_t rowaddr = slice + (uint32_t)lane * 128u;
+        const uint32_t sw = (uint32_t)lane & 7u;                       // 128-byte swizzle: 16-byte unit j of row r sits at j ^ (r % 8)
+        if constexpr (OUT_F32) {
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
-              if (col + 4 * j < args.N)
-                *reinterpret_cast<uint4*>(dst + 4 * j) = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-          } else {
-            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(args.C) + (size_t)row * (size_t)args.N + col;
+          for (uint32_t j = 0; j < 8; ++j)
+            st_shared_16(rowaddr + ((j ^ sw) << 4), v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+        } else {
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-              if (col + 8 * j < args.N)
-                *reinterpret_cast<uint4*>(dst + 8 * j) =
-                    make_uint4(pack_bf16(v[8 * j], v[8 * j + 1]), pack_bf16(v[8 * j + 2], v[8 * j + 3]),
-                               pack_bf16(v[8 * j + 4], v[8 * j + 5]), pack_bf16(v[8 * j + 6], v[8 * j + 7]));
+          for (uint32_t j = 0; j < 4; ++j) {
+            st_shared_16(rowaddr + ((j ^ sw) << 4), pack_bf16(v[8 * j], v[8 * j + 1]), pack_bf16(v[8 * j + 2], v[8 * j + 3]),
+                         pack_bf16(v[8 * j + 4], v[8 * j + 5]), pack_bf16(v[8 * j + 6], v[8 * j + 7]));
+            st_shared_16(rowaddr + (((j + 4) ^ sw) << 4), pack_bf16(w[8 * j], w[8 * j + 1]), pack_bf16(w[8 * j + 2], w[8 * j + 3]),
+                         pack_bf16(w[8 * j + 4], w[8 * j + 5]), pack_bf16(w[8 * j + 6], w[8 * j + 7]));
           }
+        }
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          const int col = col_base + c * kChunkCols;
+          if (row0 < args.M && col < args.N) tma_store_2d(&tmC, slice, col, row0);
+          bulk_commit();                                              // also when nothing was stored: keeps the group count in step
         }
       }
       tcgen05_fence_before();
@@ -494,6 +525,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
       }
     }
+    if (lane == 0) bulk_wait_all();   // every store of this warp has left shared memory and reached global memory
+    __syncwarp();
   }
 
   // ------------------------------------------------------------------ teardown
@@ -520,15 +553,15 @@ static EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// bf16 row-major [rows, cols] matrix, box = box_rows x 64 elements, 128-byte swizzle.
-static int make_map(CUtensorMap* m, const void* base, int64_t rows, int64_t cols, int box_rows) {
+// Row-major [rows, cols] matrix of 2-byte (bf16) or 4-byte (fp32) elements, box = box_rows x 128 bytes, 128-byte swizzle.
+static int make_map(CUtensorMap* m, const void* base, int64_t rows, int64_t cols, int box_rows, bool f32 = false) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) { set_error("cuTensorMapEncodeTiled is not available from the driver"); return SP_ERR_CUDA; }
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-  cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * (f32 ? 4 : 2)};
+  cuuint32_t box[2] = {f32 ? 32u : 64u, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+  CUresult r = fn(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled failed (CUresult %d)", (int)r); return SP_ERR_CUDA; }
@@ -578,7 +611,8 @@ int gemm_units(int tile_m, int tile_n, int64_t T) {
 }
 
 template <int CG, int BN, bool B_NK, bool OUT_F32>
-static int launch_variant(const GemmCall& call, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArgs& args) {
+static int launch_variant(const GemmCall& call, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC,
+                          const GemmArgs& args) {
   using C = Cfg<CG, BN>;
   auto kern = gemm_kernel<CG, BN, B_NK, OUT_F32>;
   static bool configured = false;  // per instantiation; attribute is per device but identical everywhere
@@ -600,26 +634,29 @@ static int launch_variant(const GemmCall& call, const CUtensorMap& tmA, const CU
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  e = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, args);
+  e = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmC, args);
   if (e != cudaSuccess) { set_error("kernel launch failed: %s", cudaGetErrorString(e)); return SP_ERR_CUDA; }
   return SP_OK;
 }
 
 template <int CG, int BN>
-static int launch_shape(const GemmCall& call, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArgs& args) {
+static int launch_shape(const GemmCall& call, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC,
+                        const GemmArgs& args) {
   if (call.b_nk) {
-    return call.out_f32 ? launch_variant<CG, BN, true, true>(call, tmA, tmB, args)
-                        : launch_variant<CG, BN, true, false>(call, tmA, tmB, args);
+    return call.out_f32 ? launch_variant<CG, BN, true, true>(call, tmA, tmB, tmC, args)
+                        : launch_variant<CG, BN, true, false>(call, tmA, tmB, tmC, args);
   }
-  return call.out_f32 ? launch_variant<CG, BN, false, true>(call, tmA, tmB, args)
-                      : launch_variant<CG, BN, false, false>(call, tmA, tmB, args);
+  return call.out_f32 ? launch_variant<CG, BN, false, true>(call, tmA, tmB, tmC, args)
+                      : launch_variant<CG, BN, false, false>(call, tmA, tmB, tmC, args);
 }
 
 int launch_gemm(const GemmCall& call) {
   const int cg = call.tile_m / 128;
   const int bcols = call.tile_n / cg;  // B columns per CTA
-  CUtensorMap tmA, tmB;
-  int rc = make_map(&tmA, call.A, call.M, call.K, 128);
+  CUtensorMap tmA, tmB, tmC;
+  int rc = make_map(&tmC, call.C, call.M, call.N, 32, call.out_f32 != 0);   // one epilogue warp stores 32 rows x 128 bytes
+  if (rc != SP_OK) return rc;
+  rc = make_map(&tmA, call.A, call.M, call.K, 128);
   if (rc != SP_OK) return rc;
   if (call.b_nk) rc = make_map(&tmB, call.B, call.N, call.K, bcols);   // N x K, K contiguous: one box of bcols rows
   else rc = make_map(&tmB, call.B, call.K, call.N, 64);                // K x N, N contiguous: boxes of 64 k x 64 n
@@ -662,8 +699,8 @@ int launch_gemm(const GemmCall& call) {
   }
   args.sched = call.sched;
 
-  if (cg == 1) return call.tile_n == 128 ? launch_shape<1, 128>(call, tmA, tmB, args) : launch_shape<1, 256>(call, tmA, tmB, args);
-  return call.tile_n == 128 ? launch_shape<2, 128>(call, tmA, tmB, args) : launch_shape<2, 256>(call, tmA, tmB, args);
+  if (cg == 1) return call.tile_n == 128 ? launch_shape<1, 128>(call, tmA, tmB, tmC, args) : launch_shape<1, 256>(call, tmA, tmB, tmC, args);
+  return call.tile_n == 128 ? launch_shape<2, 128>(call, tmA, tmB, tmC, args) : launch_shape<2, 256>(call, tmA, tmB, tmC, args);
 }
 
 }  // namespace sp
