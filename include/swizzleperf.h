@@ -188,6 +188,14 @@ int sp_probe_dispatch(int32_t n_blocks, int32_t cluster, int32_t* smid_host, uin
 #define SP_PROBE_LINES 256
 int sp_probe_topology(int32_t* sm_to_die_host, int32_t* n_sm, float* confidence, uint32_t* lat_host);
 
+/* Self-test of the bounded device-side wait every kernel role uses: a one-thread kernel waits on a barrier that
+ * nothing arrives on, with a limit of timeout_us (1 .. 1000000).  The wait must expire, record its code and let the
+ * kernel end normally (no trap, no fault; the context stays usable).
+ *   code      : HOST, receives the status word the wait recorded (non-zero when it expired as designed).
+ *   waited_us : HOST, receives how long the wait lasted.
+ * Synchronous; clears the status word afterwards. */
+int sp_selftest_timeout(int32_t timeout_us, int32_t* code, int64_t* waited_us);
+
 /* Synchronises `stream`, then returns and clears the device status word of the current device:
  * SP_OK, or SP_ERR_TIMEOUT if a kernel gave up on a bounded wait since the last call.
  * *detail (HOST, may be NULL) receives the raw word (which wait, which role). */

@@ -58,7 +58,7 @@ TRACE_DTYPE = np.dtype([("slot", "<i4"), ("tile", "<i4"), ("smid", "<i4"), ("uni
 
 EXPORTS = ["sp_tile_count", "sp_tile_map", "sp_tile_map_device", "sp_gemm", "sp_gemm_trace", "sp_gemm_host",
            "sp_gemm_noalloc", "sp_gemm_units",
-           "sp_probe_dispatch", "sp_probe_topology", "sp_get_status", "sp_last_error", "sp_shutdown"]
+           "sp_probe_dispatch", "sp_probe_topology", "sp_selftest_timeout", "sp_get_status", "sp_last_error", "sp_shutdown"]
 
 
 class SpError(RuntimeError):
@@ -99,6 +99,8 @@ def lib() -> ctypes.CDLL:
         L.sp_probe_dispatch.argtypes = [i32, i32, vp, vp]
         L.sp_probe_topology.restype = ctypes.c_int
         L.sp_probe_topology.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_float), vp]
+        L.sp_selftest_timeout.restype = ctypes.c_int
+        L.sp_selftest_timeout.argtypes = [i32, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int64)]
         L.sp_get_status.restype = ctypes.c_int
         L.sp_get_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32)]
         L.sp_last_error.restype = ctypes.c_char_p
@@ -263,6 +265,14 @@ def probe_topology():
     conf = ctypes.c_float(0)
     _check(lib().sp_probe_topology(die.ctypes.data, ctypes.byref(n), ctypes.byref(conf), lat.ctypes.data))
     return die[:n.value].copy(), float(conf.value), lat[:n.value * PROBE_LINES].reshape(n.value, PROBE_LINES).copy()
+
+
+def selftest_timeout(timeout_us: int):
+    """(status code recorded, microseconds waited) of a device-side wait that is made to expire."""
+    code = ctypes.c_int32(0)
+    waited = ctypes.c_int64(0)
+    _check(lib().sp_selftest_timeout(timeout_us, ctypes.byref(code), ctypes.byref(waited)))
+    return int(code.value), int(waited.value)
 
 
 def get_status(stream=None) -> int:

@@ -455,6 +455,18 @@ int sp_probe_topology(int32_t* sm_to_die_host, int32_t* n_sm, float* confidence,
   return probe_topology(sm_to_die_host, n_sm, confidence, lat_host);
 }
 
+int sp_selftest_timeout(int32_t timeout_us, int32_t* code, int64_t* waited_us) {
+  if (timeout_us < 1 || timeout_us > 1000000 || !code || !waited_us) { set_error("bad self-test arguments"); return SP_ERR_INVALID_ARG; }
+  int dev = 0;
+  int rc = current_device(&dev);
+  if (rc != SP_OK) return rc;
+  std::lock_guard<std::mutex> lock(g_mu);
+  DeviceState* ds = device_state(dev);
+  rc = get_status_word(ds);
+  if (rc != SP_OK) return rc;
+  return selftest_timeout(ds->status, timeout_us, code, waited_us);
+}
+
 int sp_get_status(void* stream, int32_t* detail) {
   int dev = 0;
   int rc = current_device(&dev);

@@ -128,13 +128,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 
 // Bounded wait.  Returns false after kTimeoutNs or once the status word is set by anyone.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, int32_t* status, int code) {
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, int32_t* status, int code,
+                                            unsigned long long timeout_ns = kTimeoutNs) {
   const unsigned long long t0 = globaltimer();
   for (uint32_t i = 1;; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 63u) == 0) {
       if (*(volatile int32_t*)status != 0) return false;
-      if (globaltimer() - t0 > kTimeoutNs) {
+      if (globaltimer() - t0 > timeout_ns) {
         atomicCAS(status, 0, code);
         return false;
       }
@@ -533,6 +534,40 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   tcgen05_fence_before();
   unit_sync<CG>();
   if (warp == 1) tmem_dealloc<CG>(tmem_base, kTmemCols);
+}
+
+// Self-test of the bounded wait: a barrier nobody arrives on.  The wait must give up after
+// `timeout_ns`, record its code and let the kernel end normally.
+__global__ void selftest_wait_kernel(int32_t* status, unsigned long long timeout_ns, unsigned long long* waited_ns) {
+  __shared__ __align__(8) unsigned long long bar;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const unsigned long long t0 = globaltimer();
+    const bool ok = mbar_wait_slow(smem_u32(&bar), 0, status, (kRoleEpilogue << 8) | 0x7f, timeout_ns);
+    *waited_ns = ok ? 0ull : globaltimer() - t0;
+  }
+}
+
+int selftest_timeout(int32_t* status_dev, int timeout_us, int32_t* code_host, int64_t* waited_us_host) {
+  unsigned long long* d_waited = nullptr;
+  cudaError_t e = cudaMalloc(&d_waited, sizeof(unsigned long long));
+  if (e == cudaSuccess) e = cudaMemset(status_dev, 0, sizeof(int32_t));
+  if (e == cudaSuccess) {
+    selftest_wait_kernel<<<1, 32>>>(status_dev, (unsigned long long)timeout_us * 1000ull, d_waited);
+    e = cudaGetLastError();
+  }
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  unsigned long long waited = 0;
+  int32_t code = 0;
+  if (e == cudaSuccess) e = cudaMemcpy(&waited, d_waited, sizeof waited, cudaMemcpyDeviceToHost);
+  if (e == cudaSuccess) e = cudaMemcpy(&code, status_dev, sizeof code, cudaMemcpyDeviceToHost);
+  if (e == cudaSuccess) e = cudaMemset(status_dev, 0, sizeof(int32_t));
+  cudaFree(d_waited);
+  if (e != cudaSuccess) { set_error("wait self-test failed: %s", cudaGetErrorString(e)); return SP_ERR_CUDA; }
+  *code_host = code;
+  *waited_us_host = (int64_t)(waited / 1000ull);
+  return SP_OK;
 }
 
 // ------------------------------------------------------------------ host side

@@ -51,6 +51,7 @@ int gemm_units(int tile_m, int tile_n, int64_t T);
 // Encodes tensor maps and launches the kernel.  Returns an sp_status.
 int launch_gemm(const GemmCall& call);
 
+int selftest_timeout(int32_t* status_dev, int timeout_us, int32_t* code_host, int64_t* waited_us_host);
 int probe_dispatch(int n_blocks, int cluster, int32_t* smid_host, uint64_t* start_host);
 int probe_topology(int32_t* sm_to_die_host, int32_t* n_sm, float* confidence, uint32_t* lat_host);
 // Size of half 0 of a DIE_SPLIT schedule, in slots.

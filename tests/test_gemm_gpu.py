@@ -245,3 +245,16 @@ def test_topology_probe_finds_two_equal_l2_halves_and_pairs_stay_together():
     near = np.median(lat[die == 0][:, :], axis=0)  # per line: latency seen from half 0 ...
     far = np.median(lat[die == 1][:, :], axis=0)   # ... and from half 1: one of them is the home half
     assert (np.maximum(near, far) > 1.5 * np.minimum(near, far)).mean() > 0.9
+
+
+def test_bounded_wait_expires_with_a_status_and_leaves_the_context_usable():
+    """Failure detection without a fault: a wait on a barrier nobody arrives on gives up after its
+    limit, records (role << 8 | wait) and the kernel ends normally."""
+    code, waited = sp.selftest_timeout(20000)                 # 20 ms
+    assert code == (3 << 8) | 0x7f
+    assert 20000 <= waited < 200000
+    assert sp.get_status() == 0                               # the word was cleared
+    A, B = synth.make_int_inputs(256, 256, 64, seed=1)        # and the device still computes
+    ref, _ = G.gemm_full(A, B)
+    got, _ = run_gemm(A, B, sp.ROW_MAJOR, (256, 256), "fp32")
+    assert np.array_equal(got, ref)
