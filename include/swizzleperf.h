@@ -167,6 +167,17 @@ int sp_gemm_host(const void* A_host, const void* B_host, void* C_host, int64_t M
 int sp_gemm_noalloc(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t K, int scheme,
                     const sp_params* params, void* stream, int32_t* status_host);
 
+/* out (N x M) = transpose of in (M x N) for 16-bit elements, under a tile order (paper: the transpose kernel, its
+ * largest reported win, whose tile grid is re-ordered for L2 locality of both the reads and the transposed writes).
+ * The matrix is cut into SP_TRANSPOSE_TILE x SP_TRANSPOSE_TILE tiles; `scheme` / `params` order that tile grid exactly
+ * as for sp_tile_map(M, N, 64, 64, ...); persistent CTAs take slots with a fixed stride.
+ *   in  : DEVICE, M x N row-major, 2-byte elements (bf16, fp16, int16: bits are moved, not interpreted), read-only.
+ *   out : DEVICE, N x M row-major, fully overwritten; must not overlap `in`.
+ * Errors: SP_ERR_INVALID_ARG, SP_ERR_ALIGNMENT (pointers not 16-byte aligned, M or N not a multiple of 8),
+ * SP_ERR_NOT_BIJECTIVE, SP_ERR_UNSUPPORTED, SP_ERR_DEVICE, SP_ERR_CUDA.  Asynchronous on `stream`. */
+#define SP_TRANSPOSE_TILE 64
+int sp_transpose(const void* in, void* out, int64_t M, int64_t N, int scheme, const sp_params* params, void* stream);
+
 /* Number of persistent CTAs (tile 128xN) or CTA pairs (tile 256xN) sp_gemm launches for T tiles;
  * slot s is run by unit s % units in round s / units.  Returns -1 on error. */
 int sp_gemm_units(int32_t tile_m, int32_t tile_n, int64_t T);

@@ -57,7 +57,7 @@ TRACE_DTYPE = np.dtype([("slot", "<i4"), ("tile", "<i4"), ("smid", "<i4"), ("uni
                         ("mma_wait_acc", "<u4"), ("load_wait_stage", "<u4"), ("epi_wait_acc", "<u4")])
 
 EXPORTS = ["sp_tile_count", "sp_tile_map", "sp_tile_map_device", "sp_gemm", "sp_gemm_trace", "sp_gemm_host",
-           "sp_gemm_noalloc", "sp_gemm_units",
+           "sp_gemm_noalloc", "sp_transpose", "sp_gemm_units",
            "sp_probe_dispatch", "sp_probe_topology", "sp_selftest_timeout", "sp_get_status", "sp_last_error", "sp_shutdown"]
 
 
@@ -93,6 +93,8 @@ def lib() -> ctypes.CDLL:
         L.sp_gemm_host.argtypes = [vp, vp, vp, i64, i64, i64, ctypes.c_int, pp, vp]
         L.sp_gemm_noalloc.restype = ctypes.c_int
         L.sp_gemm_noalloc.argtypes = [vp, vp, vp, i64, i64, i64, ctypes.c_int, pp, vp, ctypes.POINTER(ctypes.c_int32)]
+        L.sp_transpose.restype = ctypes.c_int
+        L.sp_transpose.argtypes = [vp, vp, i64, i64, ctypes.c_int, pp, vp]
         L.sp_gemm_units.restype = ctypes.c_int
         L.sp_gemm_units.argtypes = [i32, i32, i64]
         L.sp_probe_dispatch.restype = ctypes.c_int
@@ -241,6 +243,20 @@ def gemm_host(A, B, C, scheme: int = ROW_MAJOR, params: Optional[SpParams] = Non
         raise ValueError("shape mismatch")
     _check(lib().sp_gemm_host(_host_ptr(A), _host_ptr(B), _host_ptr(C), M, N, K, scheme, _pp(params),
                               _stream_handle(stream)))
+
+
+TRANSPOSE_TILE = 64
+
+
+def transpose(x, out, scheme: int = ROW_MAJOR, params: Optional[SpParams] = None, stream=None) -> None:
+    """out [N, M] = x [M, N] transposed, 2-byte elements, tiles visited in the given order (asynchronous)."""
+    M, N = x.shape
+    if tuple(out.shape) != (N, M) or x.element_size() != 2 or out.element_size() != 2:
+        raise ValueError("need a [M, N] input and a [N, M] output of 2-byte elements")
+    for t in (x, out):
+        if not t.is_cuda or not t.is_contiguous():
+            raise ValueError("x and out must be contiguous CUDA tensors")
+    _check(lib().sp_transpose(x.data_ptr(), out.data_ptr(), M, N, scheme, _pp(params), _stream_handle(stream)))
 
 
 def gemm_units(tile_m: int, tile_n: int, T: int) -> int:
