@@ -402,6 +402,69 @@ def run_sweep(args, sp, w, dA, dB, dC, params_for, flops, stream) -> int:
     return 0
 
 
+TRANSPOSE_SWEEP = ["row_major", "col_major", "group_m:2", "group_m:4", "group_m:8", "group_m:16", "group_m:32", "group_n:4",
+                   "group_n:8", "group_n:16", "morton", "hilbert", "xcd:2", "xcd:8", "die_split:m:group_m:8",
+                   "die_split:m:group_m:8:i"]
+
+
+def run_transpose(args) -> int:
+    """Second workload (the paper's largest win): 16-bit transpose under each tile order.  HBM bound:
+    algorithmic bytes = 2 * M * N * 2 (every element read once, written once).  JSON lines to stdout."""
+    import torch
+    import paper_2508_20258_b200 as sp
+    M, N = (int(v) for v in args.transpose.split("x"))
+    torch.cuda.set_device(0)
+    rng = np.random.Generator(np.random.PCG64(7))
+    x = torch.from_numpy(rng.integers(-32768, 32768, size=(M, N), dtype=np.int16)).cuda()
+    out = torch.empty((N, M), dtype=torch.int16, device="cuda")
+    stream = torch.cuda.current_stream()
+    peaks = benchutil.measured_peaks(ROOT)
+    nbytes = 2.0 * M * N * 2
+    specs = args.scheme.split(",") if args.scheme else TRANSPOSE_SWEEP
+
+    def timed(spec, n):
+        scheme, kw = parse_scheme(spec)
+        p = sp.make_params(**kw)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(n):
+            sp.transpose(x, out, scheme, p, stream)
+        e1.record(stream)
+        e1.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    if args.profile_sweep:
+        for spec in specs:
+            timed(spec, 1)
+        assert sp.get_status() == 0
+        print(json.dumps({"profile_sweep": "transpose", "shape": [M, N], "launch_order": specs}), flush=True)
+        return 0
+    for spec in specs:
+        timed(spec, 3)
+        one = timed(spec, 5)
+        n = int(max(10, min(1000, 200.0 / one)))
+        ms = min(timed(spec, n) for _ in range(2))
+        gbs = nbytes / ms / 1e6
+        print(json.dumps({"transpose": [M, N], "scheme": spec, "ms": ms, "GB/s": gbs,
+                          "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                       "frac": gbs / peaks["hbm_gbs"], "peak_kind": f"copy bandwidth, {peaks['source']}"}}),
+              flush=True)
+    assert sp.get_status() == 0
+    xt = torch.empty_like(out)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for _ in range(3):
+        xt.copy_(x.t())
+    e0.record(stream)
+    for _ in range(20):
+        xt.copy_(x.t())
+    e1.record(stream)
+    e1.synchronize()
+    ms = e0.elapsed_time(e1) / 20
+    print(json.dumps({"transpose": [M, N], "scheme": "torch copy_ of a transposed view (context only)", "ms": ms,
+                      "GB/s": nbytes / ms / 1e6}), flush=True)
+    return 0
+
+
 def main() -> int:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -418,7 +481,10 @@ def main() -> int:
     ap.add_argument("--b-layout", default="kn", choices=["kn", "nk"], help="B stored K x N (default) or N x K")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--transpose", default=None, metavar="MxN", help="time sp_transpose on an M x N 16-bit matrix instead")
     args = ap.parse_args()
+    if args.transpose:
+        return run_transpose(args)
     if args.impl == "reference":
         return run_reference(args)
     return run_ours(args)

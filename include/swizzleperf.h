@@ -196,7 +196,7 @@ int sp_probe_dispatch(int32_t n_blocks, int32_t cluster, int32_t* smid_host, uin
  *   confidence     : HOST, mean |agreement| in [0,1]; near 0 means no measurable two-way structure.
  *   lat_host       : HOST, may be NULL; else n_sm * SP_PROBE_LINES uint32 minimum latencies in SM cycles.
  * Synchronous; allocates and frees its own buffers; takes a fraction of a second. */
-#define SP_PROBE_LINES 256
+#define SP_PROBE_LINES 128
 int sp_probe_topology(int32_t* sm_to_die_host, int32_t* n_sm, float* confidence, uint32_t* lat_host);
 
 /* Self-test of the bounded device-side wait every kernel role uses: a one-thread kernel waits on a barrier that

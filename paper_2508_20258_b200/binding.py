@@ -270,7 +270,7 @@ def probe_dispatch(n_blocks: int, cluster: int = 1):
     return smid, start
 
 
-PROBE_LINES = 256
+PROBE_LINES = 128
 
 
 def probe_topology():

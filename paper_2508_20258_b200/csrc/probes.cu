@@ -15,7 +15,7 @@ namespace sp {
 
 constexpr int kProbeLines = SP_PROBE_LINES;
 constexpr int kProbeBytes = 4 << 20;
-constexpr int kProbeRepeats = 3;
+constexpr int kProbeRepeats = 2;
 
 __global__ void probe_reset_kernel(uint32_t* buf, const uint32_t* offsets, int n, uint32_t value) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;

@@ -237,7 +237,7 @@ def test_die_pinned_schedule_keeps_each_half_on_one_l2_half():
 def test_topology_probe_finds_two_equal_l2_halves_and_pairs_stay_together():
     die, conf, lat = sp.probe_topology()
     assert len(die) == torch.cuda.get_device_properties(0).multi_processor_count
-    assert lat.shape == (len(die), 256) and (lat > 0).all()
+    assert lat.shape == (len(die), sp.binding.PROBE_LINES) and (lat > 0).all()
     if conf < 0.8:
         pytest.skip("no two-way L2 structure measured on this device")
     assert set(die.tolist()) == {0, 1} and (die == 0).sum() == (die == 1).sum()
