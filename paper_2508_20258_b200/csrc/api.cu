@@ -269,10 +269,10 @@ static int get_table(DeviceState* ds, const Sched& c, const std::vector<int32_t>
   return SP_OK;
 }
 
-static int gemm_common(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t K, int scheme,
-                       const sp_params* params, void* stream, sp_trace_rec* trace, bool want_trace) {
+// Argument checks shared by every GEMM entry point; fills the resolved shape options.
+int validate_gemm_args(const void* A, const void* B, const void* C, int64_t M, int64_t N, int64_t K, const sp_params* params,
+                       int* tile_m_out, int* tile_n_out, int* out_f32_out, int* b_nk_out) {
   if (!A || !B || !C) { set_error("A, B and C must not be NULL"); return SP_ERR_INVALID_ARG; }
-  if (want_trace && !trace) { set_error("trace buffer must not be NULL"); return SP_ERR_INVALID_ARG; }
   if (M <= 0 || N <= 0 || K <= 0) { set_error("M, N, K must be positive"); return SP_ERR_INVALID_ARG; }
   if (M >= (1ll << 31) || N >= (1ll << 31) || K >= (1ll << 31)) { set_error("dimension too large"); return SP_ERR_UNSUPPORTED; }
   if (params && params->struct_size != sizeof(sp_params)) {
@@ -290,6 +290,16 @@ static int gemm_common(const void* A, const void* B, void* C, int64_t M, int64_t
   if ((out_f32 != 0 && out_f32 != 1) || (b_nk != 0 && b_nk != 1)) { set_error("bad out_dtype / b_layout"); return SP_ERR_INVALID_ARG; }
   if (((uintptr_t)A | (uintptr_t)B | (uintptr_t)C) & 15u) { set_error("A, B, C must be 16-byte aligned"); return SP_ERR_ALIGNMENT; }
   if ((K % 8) != 0 || (N % 8) != 0) { set_error("K and N must be multiples of 8 (16-byte row pitch)"); return SP_ERR_ALIGNMENT; }
+  *tile_m_out = tile_m; *tile_n_out = tile_n; *out_f32_out = out_f32; *b_nk_out = b_nk;
+  return SP_OK;
+}
+
+static int gemm_common(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t K, int scheme,
+                       const sp_params* params, void* stream, sp_trace_rec* trace, bool want_trace) {
+  if (want_trace && !trace) { set_error("trace buffer must not be NULL"); return SP_ERR_INVALID_ARG; }
+  int tile_m, tile_n, out_f32, b_nk;
+  int rc0 = validate_gemm_args(A, B, C, M, N, K, params, &tile_m, &tile_n, &out_f32, &b_nk);
+  if (rc0 != SP_OK) return rc0;
 
   GemmCall call;
   memset(&call, 0, sizeof call);

@@ -58,28 +58,13 @@ using namespace sp;
 
 extern "C" int sp_gemm_noalloc(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t K, int scheme,
                                const sp_params* params, void* stream, int32_t* status_host) {
-  if (!A || !B || !C) { set_error("A, B and C must not be NULL"); return SP_ERR_INVALID_ARG; }
-  if (M <= 0 || N <= 0 || K <= 0) { set_error("M, N, K must be positive"); return SP_ERR_INVALID_ARG; }
-  if (M >= (1ll << 31) || N >= (1ll << 31) || K >= (1ll << 31)) { set_error("dimension too large"); return SP_ERR_UNSUPPORTED; }
-  if (params && params->struct_size != sizeof(sp_params)) {
-    set_error("sp_params.struct_size is %u, expected %zu", params->struct_size, sizeof(sp_params));
-    return SP_ERR_INVALID_ARG;
-  }
-  int tile_m = params ? params->tile_m : 0, tile_n = params ? params->tile_n : 0;
-  if (tile_m == 0 && tile_n == 0) { tile_m = 256; tile_n = 256; }
-  if (!((tile_m == 128 || tile_m == 256) && (tile_n == 128 || tile_n == 256))) {
-    set_error("unsupported tile %dx%d (supported: 128x128, 128x256, 256x128, 256x256)", tile_m, tile_n);
-    return SP_ERR_UNSUPPORTED;
-  }
-  const int out_f32 = params ? params->out_dtype : 0;
-  const int b_nk = params ? params->b_layout : 0;
-  if ((out_f32 != 0 && out_f32 != 1) || (b_nk != 0 && b_nk != 1)) { set_error("bad out_dtype / b_layout"); return SP_ERR_INVALID_ARG; }
-  if (((uintptr_t)A | (uintptr_t)B | (uintptr_t)C) & 15u) { set_error("A, B, C must be 16-byte aligned"); return SP_ERR_ALIGNMENT; }
-  if ((K % 8) != 0 || (N % 8) != 0) { set_error("K and N must be multiples of 8 (16-byte row pitch)"); return SP_ERR_ALIGNMENT; }
+  int tile_m, tile_n, out_f32, b_nk;
+  int rc = validate_gemm_args(A, B, C, M, N, K, params, &tile_m, &tile_n, &out_f32, &b_nk);
+  if (rc != SP_OK) return rc;
 
   GemmCall call;
   memset(&call, 0, sizeof call);
-  int rc = resolve_sched(M, N, tile_m, tile_n, scheme, params, &call.sched);
+  rc = resolve_sched(M, N, tile_m, tile_n, scheme, params, &call.sched);
   if (rc != SP_OK) return rc;
   if (call.sched.T > kNoAllocMaxTiles) {
     set_error("sp_gemm_noalloc handles at most %d tiles; this problem has %d (use a larger tile or sp_gemm)",

@@ -20,6 +20,11 @@ void set_error(const char* fmt, ...);
 // Validates sizes and parameters and fills `out`.  Returns an sp_status.
 int resolve_sched(int64_t M, int64_t N, int32_t tileM, int32_t tileN, int scheme, const sp_params* params, Sched* out);
 
+// Argument checks shared by every GEMM entry point (NULL, sizes, struct version, tile shape, dtype/layout flags,
+// alignment); fills the resolved tile shape and flags.  Returns an sp_status.
+int validate_gemm_args(const void* A, const void* B, const void* C, int64_t M, int64_t N, int64_t K, const sp_params* params,
+                       int* tile_m, int* tile_n, int* out_f32, int* b_nk);
+
 // Evaluates the remap on the host (closed forms, curve walks, caller table) and checks
 // that it is a bijection.  Returns SP_OK or SP_ERR_NOT_BIJECTIVE / SP_ERR_INVALID_ARG.
 int build_perm_host(const Sched& sched, const int32_t* custom, std::vector<int32_t>& perm);
