@@ -55,25 +55,26 @@ def parse_scheme(spec: str):
         return sp.ROW_MAJOR, {}
     if name == "col_major":
         return sp.COL_MAJOR, {}
-    if name == "group_m":
-        return sp.GROUP_M, dict(group=int(a[1]))
+    if name == "group_m":      # group_m:G[:s]   (s = serpentine bands)
+        return sp.GROUP_M, dict(group=int(a[1]), **({"flags": 4} if "s" in a[2:] else {}))
     if name == "group_n":
-        return sp.GROUP_N, dict(group=int(a[1]))
+        return sp.GROUP_N, dict(group=int(a[1]), **({"flags": 4} if "s" in a[2:] else {}))
     if name == "morton":
         return sp.MORTON, {}
     if name == "hilbert":
         return sp.HILBERT, {}
     if name == "xcd":      # xcd:X[:W]  (balanced form)
         return sp.XCD, dict(num_xcds=int(a[1]), wave=int(a[2]) if len(a) > 2 else 0, xcd_balanced=1)
-    if name == "die_split":  # die_split:{m|n}:inner[:G][:i][:p]
+    if name == "die_split":  # die_split:{m|n}:inner[:G][:i][:p][:s]
         inner = {"row_major": sp.ROW_MAJOR, "col_major": sp.COL_MAJOR, "group_m": sp.GROUP_M, "group_n": sp.GROUP_N,
                  "morton": sp.MORTON, "hilbert": sp.HILBERT}[a[2]]
         rest = a[3:]
         inter = int("i" in rest)
         g = [int(v) for v in rest if v.isdigit()]
         kw = dict(split_axis=int(a[1] == "n"), inner_scheme=inner, inner_group=g[0] if g else 1, interleave=inter)
-        if "p" in rest:            # units pinned to the L2 half the topology probe found them on
-            kw["flags"] = 2
+        flags = (2 if "p" in rest else 0) | (4 if "s" in rest else 0)   # p: units pinned to their L2 half; s: serpentine
+        if flags:
+            kw["flags"] = flags
         return sp.DIE_SPLIT, kw
     raise ValueError(f"unknown scheme spec {spec!r}")
 

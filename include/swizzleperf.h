@@ -60,6 +60,9 @@ typedef enum {
 
 /* sp_params.flags */
 #define SP_FLAG_TRACE 1u      /* reserved for sp_gemm_trace */
+#define SP_FLAG_SERPENTINE 4u /* SP_GROUP_M / SP_GROUP_N (also as inner order of SP_DIE_SPLIT), in sp_tile_map* and sp_gemm*:
+                                 odd bands are walked in the opposite direction, so a band starts on the panels the
+                                 previous band used last */
 #define SP_FLAG_DIE_PINNED 2u /* sp_gemm* with SP_DIE_SPLIT, interleave = 0: the persistent units whose SM sits on L2 half d
                                  (measured by the topology probe, cached) run only the slots of half d of the tile space,
                                  in arrival order on that half.  Needs at least as many tiles as SMs / CTAs-per-tile;
@@ -80,7 +83,7 @@ typedef struct {
                               /*   pair per tile); 0,0 = 256x256.  Ignored by sp_tile_map*.                 */
   int32_t out_dtype;          /* sp_gemm*: 0 = C is bf16 (round to nearest even), 1 = C is fp32             */
   int32_t b_layout;           /* sp_gemm*: 0 = B is K x N row-major, 1 = B is N x K row-major               */
-  uint32_t flags;             /* 0, or SP_FLAG_DIE_PINNED                                                   */
+  uint32_t flags;             /* 0, or SP_FLAG_DIE_PINNED | SP_FLAG_SERPENTINE                              */
 } sp_params;
 
 /* One record per tile, written by sp_gemm_trace. */

@@ -69,26 +69,33 @@ def col_major(Tm: int, Tn: int) -> List[int]:
     return out
 
 
-def group_m(Tm: int, Tn: int, G: int) -> List[int]:
+def group_m(Tm: int, Tn: int, G: int, serpentine: bool = False) -> List[int]:
     """Supertiles of G tile rows: bands of G rows; inside a band walk the columns,
-    and inside a column walk the band's rows.  The last band may have fewer rows."""
+    and inside a column walk the band's rows.  The last band may have fewer rows.
+    With ``serpentine`` every second band walks its columns from the far end back."""
     if G < 1:
         raise ValueError("group must be >= 1")
     out = []
-    for first in range(0, Tm, G):
-        for tn in range(Tn):
+    for band, first in enumerate(range(0, Tm, G)):
+        cols = range(Tn)
+        if serpentine and band % 2 == 1:
+            cols = reversed(range(Tn))
+        for tn in cols:
             for tm in range(first, min(first + G, Tm)):
                 out.append(tm * Tn + tn)
     return out
 
 
-def group_n(Tm: int, Tn: int, G: int) -> List[int]:
+def group_n(Tm: int, Tn: int, G: int, serpentine: bool = False) -> List[int]:
     """Supertiles of G tile columns: the transpose of ``group_m``."""
     if G < 1:
         raise ValueError("group must be >= 1")
     out = []
-    for first in range(0, Tn, G):
-        for tm in range(Tm):
+    for band, first in enumerate(range(0, Tn, G)):
+        rows = range(Tm)
+        if serpentine and band % 2 == 1:
+            rows = reversed(range(Tm))
+        for tm in rows:
             for tn in range(first, min(first + G, Tn)):
                 out.append(tm * Tn + tn)
     return out
@@ -203,15 +210,15 @@ def xcd(T: int, X: int, W: int = 0, balanced: bool = False) -> List[int]:
 # ----------------------------------------------------------------------------------
 # die-aware split: two halves of the tile space, each ordered on its own
 # ----------------------------------------------------------------------------------
-def _inner(Tm: int, Tn: int, scheme: int, G: int) -> List[int]:
+def _inner(Tm: int, Tn: int, scheme: int, G: int, serpentine: bool = False) -> List[int]:
     if scheme == ROW_MAJOR:
         return row_major(Tm, Tn)
     if scheme == COL_MAJOR:
         return col_major(Tm, Tn)
     if scheme == GROUP_M:
-        return group_m(Tm, Tn, G)
+        return group_m(Tm, Tn, G, serpentine)
     if scheme == GROUP_N:
-        return group_n(Tm, Tn, G)
+        return group_n(Tm, Tn, G, serpentine)
     if scheme == MORTON:
         return morton(Tm, Tn)
     if scheme == HILBERT:
@@ -219,7 +226,7 @@ def _inner(Tm: int, Tn: int, scheme: int, G: int) -> List[int]:
     raise ValueError("inner scheme must be one of the plain orders")
 
 
-def die_split_halves(Tm: int, Tn: int, axis: int, inner: int, G: int) -> Tuple[List[int], List[int]]:
+def die_split_halves(Tm: int, Tn: int, axis: int, inner: int, G: int, serpentine: bool = False) -> Tuple[List[int], List[int]]:
     """The two queues.  axis 0 halves the tile rows (half 0 = rows [0, ceil(Tm/2))),
     axis 1 halves the tile columns.  Each half is a grid of its own, ordered by the
     inner scheme; its local ids are mapped back to ids of the whole grid."""
@@ -232,7 +239,7 @@ def die_split_halves(Tm: int, Tn: int, axis: int, inner: int, G: int) -> Tuple[L
             rows = r1 - r0
             q = []
             if rows > 0:
-                for local in _inner(rows, Tn, inner, G):
+                for local in _inner(rows, Tn, inner, G, serpentine):
                     lm, ln = divmod(local, Tn)
                     q.append((r0 + lm) * Tn + ln)
             halves.append(q)
@@ -242,7 +249,7 @@ def die_split_halves(Tm: int, Tn: int, axis: int, inner: int, G: int) -> Tuple[L
             cols = c1 - c0
             q = []
             if cols > 0:
-                for local in _inner(Tm, cols, inner, G):
+                for local in _inner(Tm, cols, inner, G, serpentine):
                     lm, ln = divmod(local, cols)
                     q.append(lm * Tn + (c0 + ln))
             halves.append(q)
@@ -250,8 +257,8 @@ def die_split_halves(Tm: int, Tn: int, axis: int, inner: int, G: int) -> Tuple[L
 
 
 def die_split(Tm: int, Tn: int, axis: int = 0, inner: int = ROW_MAJOR, G: int = 1,
-              interleave: bool = False) -> List[int]:
-    h0, h1 = die_split_halves(Tm, Tn, axis, inner, G)
+              interleave: bool = False, serpentine: bool = False) -> List[int]:
+    h0, h1 = die_split_halves(Tm, Tn, axis, inner, G, serpentine)
     if not interleave:
         return h0 + h1
     out = []
@@ -283,6 +290,7 @@ class Params:
     inner_group: int = 1
     interleave: int = 0
     custom_perm: Optional[Sequence[int]] = field(default=None)
+    flags: int = 0          # bit 2 (value 4): serpentine bands; bit 1 (value 2) only affects placement, not the map
 
 
 def tile_map(M: int, N: int, tile_m: int, tile_n: int, scheme: int, p: Optional[Params] = None) -> List[int]:
@@ -294,9 +302,9 @@ def tile_map(M: int, N: int, tile_m: int, tile_n: int, scheme: int, p: Optional[
     elif scheme == COL_MAJOR:
         out = col_major(Tm, Tn)
     elif scheme == GROUP_M:
-        out = group_m(Tm, Tn, p.group)
+        out = group_m(Tm, Tn, p.group, bool(p.flags & 4))
     elif scheme == GROUP_N:
-        out = group_n(Tm, Tn, p.group)
+        out = group_n(Tm, Tn, p.group, bool(p.flags & 4))
     elif scheme == MORTON:
         out = morton(Tm, Tn)
     elif scheme == HILBERT:
@@ -304,7 +312,7 @@ def tile_map(M: int, N: int, tile_m: int, tile_n: int, scheme: int, p: Optional[
     elif scheme == XCD:
         out = xcd(T, p.num_xcds, p.wave, bool(p.xcd_balanced))
     elif scheme == DIE_SPLIT:
-        out = die_split(Tm, Tn, p.split_axis, p.inner_scheme, p.inner_group, bool(p.interleave))
+        out = die_split(Tm, Tn, p.split_axis, p.inner_scheme, p.inner_group, bool(p.interleave), bool(p.flags & 4))
     elif scheme == CUSTOM:
         if p.custom_perm is None:
             raise ValueError("custom scheme needs a table")

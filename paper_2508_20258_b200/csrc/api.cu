@@ -45,6 +45,7 @@ int resolve_sched(int64_t M, int64_t N, int32_t tileM, int32_t tileN, int scheme
     case kGroupM: case kGroupN:
       if (!p || p->group < 1) { set_error("group must be >= 1"); return SP_ERR_INVALID_ARG; }
       c.group = p->group;
+      c.serp = (p->flags & SP_FLAG_SERPENTINE) != 0;
       break;
     case kXcd:
       if (!p || p->num_xcds < 1) { set_error("num_xcds must be >= 1"); return SP_ERR_INVALID_ARG; }
@@ -61,6 +62,7 @@ int resolve_sched(int64_t M, int64_t N, int32_t tileM, int32_t tileN, int scheme
       if (c.inner == kGroupM || c.inner == kGroupN) {
         if (p->inner_group < 1) { set_error("inner_group must be >= 1"); return SP_ERR_INVALID_ARG; }
         c.inner_group = p->inner_group;
+        c.serp = (p->flags & SP_FLAG_SERPENTINE) != 0;
       }
       break;
     case kCustom:

@@ -25,6 +25,7 @@ struct Sched {
   int scheme;        // sp_scheme
   int Tm, Tn, T;     // tile grid
   int group;         // GROUP_M / GROUP_N
+  int serp;          // GROUP_M / GROUP_N (also as inner order): odd bands walk the other way (boustrophedon)
   int X, W, balanced;  // XCD: chiplets, window (already resolved: W >= 1), balanced flag
   int axis, inner, inner_group, interleave;  // DIE_SPLIT
   int use_table;     // 1: the scheduler reads perm[s] from memory
@@ -81,18 +82,20 @@ SP_HD bool curve_cell(int kind, int k, int Tm, int Tn, uint32_t d, int& tm, int&
 }
 
 // Arithmetic orders on a (Tm x Tn) grid; returns the grid-local id tm * Tn + tn.
-SP_HD int plain_order(int scheme, int Tm, int Tn, int G, int s) {
+SP_HD int plain_order(int scheme, int Tm, int Tn, int G, int serp, int s) {
   switch (scheme) {
     case kCol: return (s % Tm) * Tn + s / Tm;
     case kGroupM: {
       const int band = G * Tn;
       const int b = s / band, first = b * G, g = imin(G, Tm - first), r = s - b * band;
-      return (first + r % g) * Tn + r / g;
+      const int tn = (serp && (b & 1)) ? Tn - 1 - r / g : r / g;
+      return (first + r % g) * Tn + tn;
     }
     case kGroupN: {
       const int band = G * Tm;
       const int b = s / band, first = b * G, g = imin(G, Tn - first), r = s - b * band;
-      return (r / g) * Tn + first + r % g;
+      const int tm = (serp && (b & 1)) ? Tm - 1 - r / g : r / g;
+      return tm * Tn + first + r % g;
     }
     default: return s;
   }
@@ -155,7 +158,7 @@ SP_HD bool arithmetic_scheme(const Sched& c) {
 SP_HD int slot_to_tile(const Sched& c, int s) {
   switch (c.scheme) {
     case kRow: case kCol: case kGroupM: case kGroupN:
-      return plain_order(c.scheme, c.Tm, c.Tn, c.group, s);
+      return plain_order(c.scheme, c.Tm, c.Tn, c.group, c.serp, s);
     case kMorton: case kHilbert: {
       int tm, tn;
       curve_cell(c.scheme, curve_order(c.Tm, c.Tn), c.Tm, c.Tn, (uint32_t)s, tm, tn);
@@ -168,7 +171,7 @@ SP_HD int slot_to_tile(const Sched& c, int s) {
     }
     case kDieSplit: {
       const HalfPos p = die_split_pos(c, s);
-      const int local = plain_order(c.inner, p.rows, p.cols, c.inner_group, p.idx);
+      const int local = plain_order(c.inner, p.rows, p.cols, c.inner_group, c.serp, p.idx);
       return (p.row0 + local / p.cols) * c.Tn + p.col0 + local % p.cols;
     }
     default: return s;

@@ -48,7 +48,9 @@ def test_device_remap_matches_oracle(M, N, tm, tn):
              (sp.XCD, dict(num_xcds=2, wave=74, xcd_balanced=1)), (sp.XCD, dict(num_xcds=8, xcd_balanced=1)),
              (sp.DIE_SPLIT, dict(split_axis=0, inner_scheme=sp.HILBERT)),
              (sp.DIE_SPLIT, dict(split_axis=1, inner_scheme=sp.GROUP_M, inner_group=8, interleave=1)),
-             (sp.DIE_SPLIT, dict(split_axis=1, inner_scheme=sp.MORTON, interleave=1))]
+             (sp.DIE_SPLIT, dict(split_axis=1, inner_scheme=sp.MORTON, interleave=1)),
+             (sp.GROUP_M, dict(group=8, flags=4)), (sp.GROUP_N, dict(group=3, flags=4)),
+             (sp.DIE_SPLIT, dict(split_axis=0, inner_scheme=sp.GROUP_M, inner_group=8, flags=4))]
     for scheme, kw in cases:
         want = R.tile_map(M, N, tm, tn, scheme, R.Params(**kw))
         got = sp.tile_map_device(M, N, tm, tn, scheme, sp.make_params(**kw)).cpu().numpy().tolist()

@@ -86,6 +86,28 @@ def test_group_hand_examples():
     assert R.row_major(2, 3) == [0, 1, 2, 3, 4, 5]
 
 
+def test_serpentine_bands_by_hand():
+    # 4 x 3 grid, bands of 2 rows: the second band walks its columns right to left
+    assert R.group_m(4, 3, 2, serpentine=True) == [0, 3, 1, 4, 2, 5, 8, 11, 7, 10, 6, 9]
+    # 3 x 4 grid, bands of 2 columns: the second band walks its rows bottom to top
+    assert R.group_n(3, 4, 2, serpentine=True) == [0, 1, 4, 5, 8, 9, 10, 11, 6, 7, 2, 3]
+    for Tm, Tn, G in [(5, 7, 2), (8, 8, 3), (1, 9, 4)]:
+        plain, serp = R.group_m(Tm, Tn, G), R.group_m(Tm, Tn, G, True)
+        assert R.is_bijection(serp, Tm * Tn)
+        band = G * Tn
+        for b in range(0, Tm * Tn, band):
+            chunk_p, chunk_s = plain[b:b + band], serp[b:b + band]
+            g = len(chunk_p) // Tn
+            if (b // band) % 2 == 0:
+                assert chunk_s == chunk_p
+            else:   # same band, columns in reverse order, rows inside a column unchanged
+                cols = [chunk_p[i * g:(i + 1) * g] for i in range(Tn)]
+                assert chunk_s == [t for col in reversed(cols) for t in col]
+        # the first tile column of a band is the last one of the band before
+        for b in range(band, Tm * Tn, band):
+            assert serp[b] % Tn == serp[b - 1] % Tn
+
+
 @given(Tm=st.integers(1, 60), Tn=st.integers(1, 60), G=st.integers(1, 80))
 @settings(max_examples=150, deadline=None)
 def test_group_reductions(Tm, Tn, G):

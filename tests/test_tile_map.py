@@ -21,6 +21,8 @@ def test_plain_and_grouped_orders(Tm, Tn, G):
     assert _lib_map(Tm, Tn, sp.COL_MAJOR) == R.col_major(Tm, Tn)
     assert _lib_map(Tm, Tn, sp.GROUP_M, group=G) == R.group_m(Tm, Tn, G)
     assert _lib_map(Tm, Tn, sp.GROUP_N, group=G) == R.group_n(Tm, Tn, G)
+    assert _lib_map(Tm, Tn, sp.GROUP_M, group=G, flags=4) == R.group_m(Tm, Tn, G, True)
+    assert _lib_map(Tm, Tn, sp.GROUP_N, group=G, flags=4) == R.group_n(Tm, Tn, G, True)
 
 
 @given(Tm=st.integers(1, 70), Tn=st.integers(1, 70))
@@ -60,6 +62,8 @@ def test_xcd(T, X, W, bal):
 def test_die_split(Tm, Tn, axis, inner, G, inter):
     got = _lib_map(Tm, Tn, sp.DIE_SPLIT, split_axis=axis, inner_scheme=inner, inner_group=G, interleave=int(inter))
     assert got == R.die_split(Tm, Tn, axis, inner, G, inter)
+    got = _lib_map(Tm, Tn, sp.DIE_SPLIT, split_axis=axis, inner_scheme=inner, inner_group=G, interleave=int(inter), flags=4)
+    assert got == R.die_split(Tm, Tn, axis, inner, G, inter, True)
 
 
 def test_front_door_matches_oracle_on_the_five_workload_grids():
