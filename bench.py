@@ -175,11 +175,19 @@ def run_ours(args) -> int:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     sp.lib()  # fail loudly if the extension is missing
 
-    w = synth.WORKLOADS[args.workload]
+    b_nk = int(args.b_layout == "nk")
+    if args.shape:                             # free shape for ablations: N(0,1) inputs, seed 5, 256x256 tiles, bf16 out
+        Ms, Ns, Ks = (int(v) for v in args.shape.split("x"))
+        w = synth.Workload(args.shape, Ms, Ns, Ks, "normal", 1.0, 5, 256, 256, "bf16")
+        A, B = synth.make_inputs(Ms, Ns, Ks, w.dist, w.std, w.seed, bool(b_nk))
+        SWEEPS[w.name] = ["row_major", "group_m:4", "group_m:8", "group_m:16", "hilbert", "die_split:m:group_m:8:p"]
+        DEFAULT_SCHEME[w.name] = "group_m:8"
+        args.workload = w.name
+    else:
+        w = synth.WORKLOADS[args.workload]
+        _, A, B = synth.make_workload(args.workload, b_is_nk=bool(b_nk))
     tile_m, tile_n = (int(v) for v in args.tile.split("x")) if args.tile else (w.tile_m, w.tile_n)
     out_f32 = int(w.out_dtype == "fp32")
-    b_nk = int(args.b_layout == "nk")
-    _, A, B = synth.make_workload(args.workload, b_is_nk=bool(b_nk))
     dA = torch.from_numpy(A.view(np.int16)).cuda().view(torch.bfloat16)
     dB = torch.from_numpy(B.view(np.int16)).cuda().view(torch.bfloat16)
     dC = torch.empty((w.M, w.N), dtype=torch.float32 if out_f32 else torch.bfloat16, device="cuda")
@@ -190,6 +198,16 @@ def run_ours(args) -> int:
     def params_for(spec):
         scheme, kw = parse_scheme(spec)
         return scheme, sp.make_params(tile_m=tile_m, tile_n=tile_n, out_dtype=out_f32, b_layout=b_nk, **kw)
+
+    def supported(spec):                       # the die-pinned orders need at least as many tiles as units
+        s_, p_ = params_for(spec)
+        try:
+            sp.gemm(dA, dB, dC, s_, p_, stream)
+            return True
+        except sp.SpError as err:
+            if err.status == sp.ERR_UNSUPPORTED:
+                return False
+            raise
 
     def barrier():
         if world > 1:
@@ -202,7 +220,7 @@ def run_ours(args) -> int:
     if args.sweep:
         return run_sweep(args, sp, w, dA, dB, dC, params_for, flops, stream)
     if args.profile_sweep:                     # one launch per scheme, in SWEEPS order: the command ncu wraps
-        specs = args.scheme.split(",") if args.scheme else SWEEPS[args.workload]
+        specs = [x for x in (args.scheme.split(",") if args.scheme else SWEEPS[args.workload]) if supported(x)]
         for spec in specs:
             s_, p_ = params_for(spec)
             sp.gemm(dA, dB, dC, s_, p_, stream)
@@ -343,7 +361,14 @@ def run_sweep_sustained(args, sp, w, dA, dB, dC, params_for, flops, stream) -> i
     """Every scheme timed on its own in back-to-back launches (about 0.3 s each, two passes): the power-capped
     steady state, where traffic saved by a tile order shows up as clock and therefore as time."""
     import torch
-    specs = args.scheme.split(",") if args.scheme else SWEEPS[args.workload]
+    specs = []
+    for spec in (args.scheme.split(",") if args.scheme else SWEEPS[args.workload]):
+        try:
+            sp.gemm(dA, dB, dC, *params_for(spec), stream)
+            specs.append(spec)
+        except sp.SpError as err:
+            if err.status != sp.ERR_UNSUPPORTED:
+                raise
     acc = {spec: [] for spec in specs}
     for _ in range(2):
         for spec in specs:
@@ -473,6 +498,7 @@ def main() -> int:
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg3", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--shape", default=None, metavar="MxNxK", help="free GEMM shape instead of a named workload (ablations)")
     ap.add_argument("--scheme", default=None)
     ap.add_argument("--tile", default=None, help="MxN override, e.g. 128x256")
     ap.add_argument("--kernel-only", action="store_true", help="time the kernel only (the command profilers wrap)")
