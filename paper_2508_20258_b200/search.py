@@ -1,0 +1,132 @@
+"""Enumerative search for the best tile order of one GEMM: the paper's optimisation loop without the LLM.
+
+The paper's loop proposes a remap, validates it (a non-bijective remap is a failure), runs and
+checks the kernel against the ground truth, measures a bottleneck metric, appends the attempt
+to a history buffer and keeps the best validated candidate.  Here the proposals come from a
+fixed list of parameterised orders instead of a language model, validation is the library's own
+bijectivity gate plus bit-identity of C with the row-major run (a swizzle only reorders tiles),
+and the ranking metric is the measured time of back-to-back launches (the L2 hit rate the paper
+ranks by needs a profiler; `profiles/` shows the two agree in ordering).
+
+    python -m paper_2508_20258_b200.search --shape 8192x8192x8192
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import sys
+from dataclasses import asdict, dataclass, field
+from typing import Dict, List, Optional, Sequence, Tuple
+
+from . import binding as sp
+
+
+@dataclass
+class Attempt:
+    name: str
+    scheme: int
+    params: Dict
+    status: str = "pending"          # "ok" | "broken" (not a bijection) | "unsupported" | "wrong" (C differs)
+    ms: Optional[float] = None
+    tflops: Optional[float] = None
+    speedup: Optional[float] = None  # over the first validated attempt (row-major)
+    note: str = ""
+
+
+@dataclass
+class SearchResult:
+    best: Optional[Attempt]
+    history: List[Attempt] = field(default_factory=list)
+
+
+def default_candidates(units: int) -> List[Tuple[str, int, Dict]]:
+    c: List[Tuple[str, int, Dict]] = [("row_major", sp.ROW_MAJOR, {}), ("col_major", sp.COL_MAJOR, {})]
+    for g in (2, 4, 8, 16, 32):
+        c.append((f"group_m:{g}", sp.GROUP_M, dict(group=g)))
+        c.append((f"group_n:{g}", sp.GROUP_N, dict(group=g)))
+    c += [("morton", sp.MORTON, {}), ("hilbert", sp.HILBERT, {})]
+    # the paper's formula as printed (may be rejected) and its balanced form, per wave of resident units
+    c.append((f"xcd:2:{units}:literal", sp.XCD, dict(num_xcds=2, wave=units, xcd_balanced=0)))
+    c.append((f"xcd:8:{units}:literal", sp.XCD, dict(num_xcds=8, wave=units, xcd_balanced=0)))
+    c.append((f"xcd:2:{units}", sp.XCD, dict(num_xcds=2, wave=units, xcd_balanced=1)))
+    for axis, an in ((0, "m"), (1, "n")):
+        for g in (4, 8, 16):
+            c.append((f"die_split:{an}:group_m:{g}:p", sp.DIE_SPLIT,
+                      dict(split_axis=axis, inner_scheme=sp.GROUP_M, inner_group=g, flags=2)))
+        c.append((f"die_split:{an}:hilbert:p", sp.DIE_SPLIT, dict(split_axis=axis, inner_scheme=sp.HILBERT, flags=2)))
+    return c
+
+
+def search(A, B, C, tile: Tuple[int, int] = (256, 256), candidates: Optional[Sequence[Tuple[str, int, Dict]]] = None,
+           launches: int = 50, out_dtype: int = 0, b_layout: int = 0, verbose: bool = False) -> SearchResult:
+    """Tries every candidate order on C = A.B (CUDA tensors) and returns the history and the fastest valid one."""
+    import torch
+
+    M, K = A.shape
+    N = B.shape[0] if b_layout else B.shape[1]
+    T = sp.tile_count(M, N, tile[0], tile[1])
+    units = sp.gemm_units(tile[0], tile[1], T)
+    cands = list(candidates) if candidates is not None else default_candidates(units)
+    flops = 2.0 * M * N * K
+    res = SearchResult(best=None)
+    truth = None
+    base_ms = None
+    for name, scheme, kw in cands:
+        att = Attempt(name=name, scheme=scheme, params=dict(kw))
+        res.history.append(att)
+        p = sp.make_params(tile_m=tile[0], tile_n=tile[1], out_dtype=out_dtype, b_layout=b_layout, **kw)
+        try:
+            sp.tile_map(M, N, tile[0], tile[1], scheme, p)                    # validation: must be a bijection
+            C.zero_()
+            sp.gemm(A, B, C, scheme, p)
+            sp.get_status()
+        except sp.SpError as e:
+            att.status = "broken" if e.status == sp.ERR_NOT_BIJECTIVE else "unsupported"
+            att.note = str(e)
+            continue
+        bits = C.view(torch.int16 if C.element_size() == 2 else torch.int32)
+        if truth is None:
+            truth = bits.clone()                                              # ground truth: the first valid run
+        elif not torch.equal(bits, truth):
+            att.status = "wrong"
+            continue
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(launches):
+            sp.gemm(A, B, C, scheme, p)
+        e1.record()
+        e1.synchronize()
+        att.ms = e0.elapsed_time(e1) / launches
+        att.tflops = flops / att.ms / 1e9
+        base_ms = base_ms or att.ms
+        att.speedup = base_ms / att.ms
+        att.status = "ok"
+        if res.best is None or att.ms < res.best.ms:
+            res.best = att
+        if verbose:
+            print(json.dumps(asdict(att)), flush=True)
+    return res
+
+
+def main(argv=None) -> int:
+    import torch
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--shape", default="8192x8192x8192")
+    ap.add_argument("--tile", default="256x256")
+    ap.add_argument("--launches", type=int, default=100)
+    a = ap.parse_args(argv)
+    M, N, K = (int(v) for v in a.shape.split("x"))
+    tile = tuple(int(v) for v in a.tile.split("x"))
+    g = torch.Generator(device="cuda").manual_seed(0)
+    A = torch.randn((M, K), device="cuda", generator=g).bfloat16()
+    B = torch.randn((K, N), device="cuda", generator=g).bfloat16()
+    C = torch.empty((M, N), device="cuda", dtype=torch.bfloat16)
+    r = search(A, B, C, tile, launches=a.launches, verbose=True)
+    print(json.dumps({"best": asdict(r.best) if r.best else None,
+                      "tried": len(r.history), "broken": [h.name for h in r.history if h.status == "broken"]}))
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())
