@@ -289,3 +289,13 @@ def test_bit_swap_pattern_breaks_when_grid_changes():
         assert R.is_bijection([swap(p) for p in range(n)], n)
     for n in (6, 20, 100):
         assert not R.is_bijection([swap(p) for p in range(n)], n)
+
+
+def test_exactly_when_the_printed_formula_is_a_bijection():
+    """Counting argument: chiplet x receives ceil(n/X) ids if x < n mod X, else floor(n/X), but the printed
+    form starts every chiplet at x * ceil(n/X); the ranges tile [0, n) only if at most one (the last)
+    chiplet is short: n mod X in {0, X-1}, or X > n (then it is the identity)."""
+    for n in range(1, 161):
+        for X in range(1, 25):
+            bij = R.is_bijection(R.xcd_window(n, X, False), n)
+            assert bij == (X > n or n % X in (0, X - 1)), (n, X)
