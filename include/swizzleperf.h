@@ -66,7 +66,8 @@ typedef enum {
 #define SP_FLAG_DIE_PINNED 2u /* sp_gemm* with SP_DIE_SPLIT, interleave = 0: the persistent units whose SM sits on L2 half d
                                  (measured by the topology probe, cached) run only the slots of half d of the tile space,
                                  in arrival order on that half.  Needs at least as many tiles as SMs / CTAs-per-tile;
-                                 SP_ERR_UNSUPPORTED if the probe finds no usable two-way structure.  The output is the same. */
+                                 SP_ERR_UNSUPPORTED if the probe finds no usable two-way structure.  The output is the same, and every
+                                 tile runs exactly once wherever the units land.  At most 64 such launches in flight per device. */
 
 typedef struct {
   uint32_t struct_size;       /* must be sizeof(sp_params)                                                  */
@@ -201,6 +202,11 @@ int sp_probe_dispatch(int32_t n_blocks, int32_t cluster, int32_t* smid_host, uin
  * Synchronous; allocates and frees its own buffers; takes a fraction of a second. */
 #define SP_PROBE_LINES 128
 int sp_probe_topology(int32_t* sm_to_die_host, int32_t* n_sm, float* confidence, uint32_t* lat_host);
+
+/* Self-test (host only) of the rank assignment of die-pinned scheduling: with n0 / n1 units expected on the two L2
+ * halves and arrivals0 of the n0 + n1 units actually landing on half 0, every (half, rank) pair must be handed out
+ * exactly once.  Returns SP_OK, or SP_ERR_NOT_BIJECTIVE if the assignment would skip or repeat work. */
+int sp_selftest_pinned_tickets(int32_t n0, int32_t n1, int32_t arrivals0);
 
 /* Self-test of the bounded device-side wait every kernel role uses: a one-thread kernel waits on a barrier that
  * nothing arrives on, with a limit of timeout_us (1 .. 1000000).  The wait must expire, record its code and let the

@@ -58,7 +58,7 @@ TRACE_DTYPE = np.dtype([("slot", "<i4"), ("tile", "<i4"), ("smid", "<i4"), ("uni
 
 EXPORTS = ["sp_tile_count", "sp_tile_map", "sp_tile_map_device", "sp_gemm", "sp_gemm_trace", "sp_gemm_host",
            "sp_gemm_noalloc", "sp_transpose", "sp_gemm_units",
-           "sp_probe_dispatch", "sp_probe_topology", "sp_selftest_timeout", "sp_get_status", "sp_last_error", "sp_shutdown"]
+           "sp_probe_dispatch", "sp_probe_topology", "sp_selftest_timeout", "sp_selftest_pinned_tickets", "sp_get_status", "sp_last_error", "sp_shutdown"]
 
 
 class SpError(RuntimeError):
@@ -101,6 +101,8 @@ def lib() -> ctypes.CDLL:
         L.sp_probe_dispatch.argtypes = [i32, i32, vp, vp]
         L.sp_probe_topology.restype = ctypes.c_int
         L.sp_probe_topology.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_float), vp]
+        L.sp_selftest_pinned_tickets.restype = ctypes.c_int
+        L.sp_selftest_pinned_tickets.argtypes = [i32, i32, i32]
         L.sp_selftest_timeout.restype = ctypes.c_int
         L.sp_selftest_timeout.argtypes = [i32, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int64)]
         L.sp_get_status.restype = ctypes.c_int

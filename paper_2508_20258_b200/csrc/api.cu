@@ -143,6 +143,7 @@ struct DeviceState {
   int device = -1;
   int32_t* status = nullptr;
   std::vector<TableEntry> tables;
+  unsigned die_pair_next = 0;   // rotation over the counter pairs
   int die_known = 0;            // 0: not probed, 1: usable map, -1: probe found no two-way structure
   int sms_on_die[2] = {0, 0};
   uint32_t die_mask[8] = {};
@@ -155,6 +156,7 @@ static std::vector<DeviceState> g_devs;
 static uint64_t g_stamp = 0;
 constexpr size_t kMaxTables = 64;
 
+constexpr int kDiePairs = 64;   // die-pinned launches that may be in flight at once on one device (different streams)
 static std::mutex g_valid_mu;
 static std::vector<Sched> g_validated;
 
@@ -211,8 +213,9 @@ static int current_device(int* dev) {
 
 static int get_status_word(DeviceState* ds) {
   if (!ds->status) {
-    SP_CUDA(cudaMalloc(&ds->status, 4 * sizeof(int32_t)));   // status word, two die counters, spare
-    SP_CUDA(cudaMemset(ds->status, 0, 4 * sizeof(int32_t)));
+    // status word, then kDiePairs pairs of arrival counters handed to die-pinned launches in rotation
+    SP_CUDA(cudaMalloc(&ds->status, (2 + 2 * kDiePairs) * sizeof(int32_t)));
+    SP_CUDA(cudaMemset(ds->status, 0, (2 + 2 * kDiePairs) * sizeof(int32_t)));
   }
   return SP_OK;
 }
@@ -341,6 +344,7 @@ static int gemm_common(const void* A, const void* B, void* C, int64_t M, int64_t
     rc = get_die_map(ds);
     if (rc != SP_OK) return rc;
     call.pinned = 1;
+    call.die_count_dev = ds->status + 2 + 2 * (int)(ds->die_pair_next++ % kDiePairs);
     call.half0 = die_split_half0(call.sched);
     call.sms_on_die[0] = ds->sms_on_die[0]; call.sms_on_die[1] = ds->sms_on_die[1];
     for (int i = 0; i < 8; ++i) call.die_mask[i] = ds->die_mask[i];
@@ -496,6 +500,22 @@ int sp_probe_topology(int32_t* sm_to_die_host, int32_t* n_sm, float* confidence,
   int rc = current_device(&dev);
   if (rc != SP_OK) return rc;
   return probe_topology(sm_to_die_host, n_sm, confidence, lat_host);
+}
+
+int sp_selftest_pinned_tickets(int32_t n0, int32_t n1, int32_t arrivals0) {
+  if (n0 < 0 || n1 < 0 || arrivals0 < 0 || arrivals0 > n0 + n1 || n0 + n1 > (1 << 20)) { set_error("bad arguments"); return SP_ERR_INVALID_ARG; }
+  std::vector<int> taken((size_t)(n0 + n1), 0);
+  for (int die = 0; die < 2; ++die) {
+    const int arrivals = die ? n0 + n1 - arrivals0 : arrivals0;
+    for (int r = 0; r < arrivals; ++r) {
+      int d, k;
+      pinned_ticket(n0, n1, die, r, d, k);
+      if (d < 0 || d > 1 || k < 0 || k >= (d ? n1 : n0)) { set_error("ticket out of range"); return SP_ERR_NOT_BIJECTIVE; }
+      taken[(size_t)(d ? n0 + k : k)]++;
+    }
+  }
+  for (int v : taken) if (v != 1) { set_error("a (half, rank) pair was not taken exactly once"); return SP_ERR_NOT_BIJECTIVE; }
+  return SP_OK;
 }
 
 int sp_selftest_timeout(int32_t timeout_us, int32_t* code, int64_t* waited_us) {

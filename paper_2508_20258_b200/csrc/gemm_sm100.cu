@@ -134,8 +134,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     // both CTAs of the unit read the pair of words after the start-up barrier
     uint32_t smid;
     asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
-    const uint32_t die = (args.die_mask[(smid >> 5) & 7] >> (smid & 31)) & 1u;
-    const uint32_t r = (uint32_t)atomicAdd(args.die_count + die, 1);
+    const int my_die = (int)((args.die_mask[(smid >> 5) & 7] >> (smid & 31)) & 1u);
+    const int arrival = atomicAdd(args.die_count + my_die, 1);
+    int die_i, rank_i;   // normally (my_die, arrival); re-assigned only if the GPU is shared and placement is uneven
+    pinned_ticket(args.units_on_die[0], args.units_on_die[1], my_die, arrival, die_i, rank_i);
+    const uint32_t die = (uint32_t)die_i, r = (uint32_t)rank_i;
 #pragma unroll
     for (uint32_t c = 0; c < (uint32_t)CG; ++c) {
       const uint32_t dst = CG == 1 ? sched_slot : mapa(sched_slot, c);
@@ -155,7 +158,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     s_step = args.units_on_die[die];
     s_first = (die ? args.half0 : 0) + (int)r;
     s_end = die ? T : args.half0;
-    if ((int)r >= s_step) s_first = s_end;           // more arrivals than the probe predicted: this unit idles
   }
 
   if (warp == 0) {
@@ -526,7 +528,7 @@ int launch_gemm(const GemmCall& call) {
     args.half0 = call.half0;
     args.units_on_die[0] = call.sms_on_die[0] / cg_;
     args.units_on_die[1] = call.sms_on_die[1] / cg_;
-    args.die_count = call.status_dev + 1;
+    args.die_count = call.die_count_dev;
     for (int i = 0; i < 8; ++i) args.die_mask[i] = call.die_mask[i];
     if (args.units != args.units_on_die[0] + args.units_on_die[1]) {
       set_error("die-pinned scheduling needs every SM to host one CTA (%d units launched, %d expected)", args.units,

@@ -142,6 +142,15 @@ SP_HD int die_split_slot(const Sched& c, int half, int idx) {
   return idx + h1;
 }
 
+// Die-pinned scheduling: the r-th unit (0-based) to arrive on L2 half `die`, where n[d] units are expected on half d
+// and exactly n[0] + n[1] units exist.  A unit beyond the expected count of its half takes a rank left free on the
+// other half, from the top down, so that every (half, rank) pair is taken exactly once under any placement.
+SP_HD void pinned_ticket(int n0, int n1, int die, int r, int& die_out, int& rank_out) {
+  const int n_own = die ? n1 : n0, n_other = die ? n0 : n1;
+  if (r < n_own) { die_out = die; rank_out = r; }
+  else { die_out = die ^ 1; rank_out = n_other - 1 - (r - n_own); }
+}
+
 SP_HD bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
 
 // True when slot_to_tile needs no table for this configuration.

@@ -127,3 +127,13 @@ def test_paper_example_through_the_library():
     with pytest.raises(sp.SpError) as e:      # 148 blocks over 8 chiplets: printed form leaves the range
         sp.tile_map(128, 148 * 128, 128, 128, sp.XCD, sp.make_params(num_xcds=8))
     assert e.value.status == sp.ERR_NOT_BIJECTIVE
+
+
+def test_die_pinned_rank_assignment_covers_every_rank_under_any_placement():
+    """If the GPU is shared, more units than measured may land on one L2 half; the surplus must take exactly
+    the ranks left free on the other half (host self-test of the function the kernel uses)."""
+    L = sp.lib()
+    for n0, n1 in [(37, 37), (74, 74), (1, 1), (3, 5), (0, 4)]:
+        for arrivals0 in range(0, n0 + n1 + 1):
+            assert L.sp_selftest_pinned_tickets(n0, n1, arrivals0) == sp.OK, (n0, n1, arrivals0)
+    assert L.sp_selftest_pinned_tickets(2, 2, 5) == sp.ERR_INVALID_ARG
