@@ -80,8 +80,9 @@ typedef struct {
   int32_t inner_group;        /* SP_DIE_SPLIT: G of the inner scheme                                        */
   int32_t interleave;         /* SP_DIE_SPLIT: 0 = concatenated halves, 1 = alternating merge               */
   const int32_t* custom_perm; /* SP_CUSTOM: HOST array of T tile ids (validated, copied)                    */
-  int32_t tile_m, tile_n;     /* sp_gemm*: 128x128, 128x256 (one CTA per tile) or 256x128, 256x256 (a CTA   */
-                              /*   pair per tile); 0,0 = 256x256.  Ignored by sp_tile_map*.                 */
+  int32_t tile_m, tile_n;     /* sp_gemm*: 128x128, 128x256 (one CTA per tile), 256x128, 256x256 (a CTA pair */
+                              /*   per tile) or 256x512 (a CTA pair runs two 256x256 MMA tiles that share    */
+                              /*   the A panel); 0,0 = 256x256.  Ignored by sp_tile_map*.                    */
   int32_t out_dtype;          /* sp_gemm*: 0 = C is bf16 (round to nearest even), 1 = C is fp32             */
   int32_t b_layout;           /* sp_gemm*: 0 = B is K x N row-major, 1 = B is N x K row-major               */
   uint32_t flags;             /* 0, or SP_FLAG_DIE_PINNED | SP_FLAG_SERPENTINE                              */

@@ -286,8 +286,8 @@ int validate_gemm_args(const void* A, const void* B, const void* C, int64_t M, i
   }
   int tile_m = params ? params->tile_m : 0, tile_n = params ? params->tile_n : 0;
   if (tile_m == 0 && tile_n == 0) { tile_m = 256; tile_n = 256; }
-  if (!((tile_m == 128 || tile_m == 256) && (tile_n == 128 || tile_n == 256))) {
-    set_error("unsupported tile %dx%d (supported: 128x128, 128x256, 256x128, 256x256)", tile_m, tile_n);
+  if (!(((tile_m == 128 || tile_m == 256) && (tile_n == 128 || tile_n == 256)) || (tile_m == 256 && tile_n == 512))) {
+    set_error("unsupported tile %dx%d (supported: 128x128, 128x256, 256x128, 256x256, 256x512)", tile_m, tile_n);
     return SP_ERR_UNSUPPORTED;
   }
   const int out_f32 = params ? params->out_dtype : 0;

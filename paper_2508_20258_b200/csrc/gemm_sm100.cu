@@ -1,7 +1,9 @@
 // Persistent, warp-specialised bf16 GEMM for sm_100a whose tile order is a remap of slot ids
 // (the paper's swizzle: each block recomputes which output tile it works on).
 //
-// One persistent unit = one CTA (tile 128 x BN) or a CTA pair (tile 256 x BN, cta_group::2).
+// One persistent unit = one CTA (tile 128 x BN) or a CTA pair (tile 256 x BN, cta_group::2).  BN = 512 is two
+// 256-wide MMA tiles that share the A panel (one accumulator each, no double buffering): a quarter less operand
+// traffic from L2 per flop, at the price of an epilogue that is not hidden behind the next tile's mainloop.
 // Unit u runs slots u, u + units, u + 2*units, ...; slot s computes tile slot_to_tile(s).
 //
 // Warp roles (192 threads):
@@ -31,13 +33,18 @@ namespace sp {
 
 constexpr int kBK = 64;          // k extent of one stage: 64 bf16 = one 128-byte swizzle row
 constexpr int kUmmaK = 16;       // k extent of one tcgen05.mma with 16-bit inputs
-constexpr int kThreads = 192;
 constexpr uint32_t kSmemLimit = 232448;  // 227 KiB opt-in maximum per CTA
 constexpr uint32_t kBarrierBytes = 1024;
 constexpr int kTmemCols = 512;
 
 template <int CG, int BN>
 struct Cfg {
+  static constexpr int kMmaN = BN > 256 ? 256 : BN;             // N of one tcgen05.mma
+  static constexpr int kNT = BN / kMmaN;                        // MMA tiles side by side in one scheduler tile
+  static constexpr int kBufs = kNT == 1 ? 2 : 1;                // accumulator buffers of BN columns in the 512 TMEM columns
+  static constexpr int kEpiWarps = 4;                           // one per TMEM lane quarter
+  static constexpr int kThreads = 64 + 32 * kEpiWarps;          // producer warp, MMA warp, epilogue warps
+  static constexpr int kMmaCols = kMmaN / CG;                   // columns of B one CTA supplies to one MMA
   static constexpr int kBCols = BN / CG;                        // columns of B held by one CTA
   static constexpr uint32_t kABytes = 128 * kBK * 2;            // 128 rows of A
   static constexpr uint32_t kBBytes = kBCols * kBK * 2;
@@ -95,7 +102,7 @@ __device__ __forceinline__ uint32_t pack_bf16(uint32_t lo_bits, uint32_t hi_bits
 
 // ------------------------------------------------------------------ the kernel
 template <int CG, int BN, bool B_NK, bool OUT_F32>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__((Cfg<CG, BN>::kThreads), 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const __grid_constant__ CUtensorMap tmC, const GemmArgs args) {
   using C = Cfg<CG, BN>;
@@ -121,7 +128,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < S; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_empty + 8 * i, 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(bar_tfull + 8 * i, 1); mbar_init(bar_tempty + 8 * i, 4 * CG); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_tfull + 8 * i, 1); mbar_init(bar_tempty + 8 * i, C::kEpiWarps * CG); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -172,7 +179,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const int t = tile_of_slot(args, s);
         const int tm = t / Tn, tn = t - tm * Tn;
         const int row0 = tm * TILE_M + (int)rank * 128;
-        const int col0 = tn * BN + (int)rank * C::kBCols;
+        const int col0 = tn * BN + (int)rank * C::kMmaCols;        // + c * kMmaN for the c-th MMA tile
         const bool tracing = args.trace != nullptr && rank == 0;
         uint32_t waited = 0;
         if (tracing && lane == 0) {
@@ -193,11 +200,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             if (rank == 0) mbar_arrive_expect_tx(full_local, CG * C::kStageBytes);
             tma_load_2d<CG>(sa, &tmA, kb * kBK, row0, full_leader);
             if constexpr (B_NK) {
-              tma_load_2d<CG>(sb, &tmB, kb * kBK, col0, full_leader);
+#pragma unroll
+              for (int c = 0; c < C::kNT; ++c)
+                tma_load_2d<CG>(sb + c * (C::kMmaCols * kBK * 2), &tmB, kb * kBK, col0 + c * C::kMmaN, full_leader);
             } else {
 #pragma unroll
-              for (int j = 0; j < C::kBCols / 64; ++j)
-                tma_load_2d<CG>(sb + j * (64 * kBK * 2), &tmB, col0 + j * 64, kb * kBK, full_leader);
+              for (int j = 0; j < C::kBCols / 64; ++j) {   // boxes of 64 columns, MMA tile by MMA tile
+                constexpr int per = C::kMmaCols / 64;
+                tma_load_2d<CG>(sb + j * (64 * kBK * 2), &tmB, col0 + (j / per) * C::kMmaN + (j % per) * 64, kb * kBK, full_leader);
+              }
             }
           }
           __syncwarp();
@@ -222,43 +233,54 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     // ---------------------------------------------------------------- MMA issuer (leader CTA only)
     // Whole warp in the loop, one elected lane issues: descriptors stay warp-uniform values.
     if (rank == 0) {
-      constexpr uint32_t idesc = make_idesc(TILE_M, BN, !B_NK);
+      constexpr uint32_t idesc = make_idesc(TILE_M, C::kMmaN, !B_NK);
       int stage = 0;
       uint32_t phase = 0;
       int it = 0;
       bool ok = true;
+      // Accumulator parts.  One MMA tile per scheduler tile: one part, alternating between two TMEM buffers.
+      // Two MMA tiles (BN = 512): two parts, each with its own pair of barriers, so the epilogue can drain the
+      // first while the second is still being computed, and the next tile can start on the first part while the
+      // second is being drained.
       for (int s = s_first; s < s_end && ok; s += s_step, ++it) {
-        const int buf = it & 1;
-        const uint32_t use = (uint32_t)(it >> 1) & 1u;
+        const int buf = it % C::kBufs;
+        const uint32_t use = C::kNT == 1 ? ((uint32_t)(it / C::kBufs) & 1u) : ((uint32_t)it & 1u);
         const bool tracing = args.trace != nullptr;
         uint32_t wait_acc = 0, wait_data = 0;
-        ok = mbar_wait_timed(bar_tempty + 8 * buf, use ^ 1u, args.status, (kRoleMma << 8) | 1, tracing, &wait_acc);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        tcgen05_fence_after();
         if (tracing && lane == 0) args.trace[s].t_mma_begin = globaltimer();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
-        for (int kb = 0; kb < KB; ++kb) {
+        for (int kb = 0; kb < KB && ok; ++kb) {
           ok = mbar_wait_timed(bar_full + 8 * stage, phase, args.status, (kRoleMma << 8) | 2, tracing, &wait_data);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tcgen05_fence_after();
           const uint32_t sa = smem_base + stage * C::kStageBytes;
           const uint32_t sb = sa + C::kABytes;
-          if (elect_one()) {
 #pragma unroll
-            for (int k = 0; k < kBK / kUmmaK; ++k) {
-              const uint64_t da = smem_desc(sa + k * (kUmmaK * 2), 16, 1024);
-              const uint64_t db = smem_desc(sb + k * args.b_kstep, args.b_lbo, args.b_sbo);
-              umma_bf16<CG>(d_tmem, da, db, idesc, (uint32_t)((kb | k) != 0));
+          for (int c = 0; c < C::kNT; ++c) {
+            const int part = C::kNT == 1 ? buf : c;
+            if (kb == 0) {                       // the part must have been drained by the epilogue of its previous use
+              ok = mbar_wait_timed(bar_tempty + 8 * part, use ^ 1u, args.status, (kRoleMma << 8) | 1, tracing, &wait_acc);
+              ok = __all_sync(0xffffffffu, ok);
+              if (!ok) break;
+              tcgen05_fence_after();
             }
-            umma_commit<CG>(bar_empty + 8 * stage);
+            const uint32_t d_tmem = tmem_base + (uint32_t)(C::kNT == 1 ? buf * BN : c * C::kMmaN);
+            if (elect_one()) {
+#pragma unroll
+              for (int k = 0; k < kBK / kUmmaK; ++k) {
+                const uint64_t da = smem_desc(sa + k * (kUmmaK * 2), 16, 1024);
+                const uint64_t db = smem_desc(sb + c * (C::kMmaCols * kBK * 2) + k * args.b_kstep, args.b_lbo, args.b_sbo);
+                umma_bf16<CG>(d_tmem, da, db, idesc, (uint32_t)((kb | k) != 0));
+              }
+              if (kb == KB - 1) umma_commit<CG>(bar_tfull + 8 * part);   // this part is complete
+            }
+            __syncwarp();
           }
+          if (!ok) break;
+          if (elect_one()) umma_commit<CG>(bar_empty + 8 * stage);
           __syncwarp();
           if (++stage == S) { stage = 0; phase ^= 1u; }
         }
-        if (ok && elect_one()) umma_commit<CG>(bar_tfull + 8 * buf);
-        __syncwarp();
         if (tracing && lane == 0) {
           sp_trace_rec* rec = args.trace + s;
           rec->mma_wait_data = wait_data; rec->mma_wait_acc = wait_acc; rec->t_mma_issued = globaltimer();
@@ -275,61 +297,112 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     for (int s = s_first; s < s_end && ok; s += s_step, ++it) {
       const int t = tile_of_slot(args, s);
       const int tm = t / Tn, tn = t - tm * Tn;
-      const int buf = it & 1;
-      const uint32_t use = (uint32_t)(it >> 1) & 1u;
+      const int buf = it % C::kBufs;
+      const uint32_t use = C::kNT == 1 ? ((uint32_t)(it / C::kBufs) & 1u) : ((uint32_t)it & 1u);
       uint32_t wait_epi = 0;
-      ok = mbar_wait_timed(bar_tfull + 8 * buf, use, args.status, (kRoleEpilogue << 8) | 1, args.trace != nullptr, &wait_epi);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      tcgen05_fence_after();
       const int row0 = tm * TILE_M + (int)rank * 128 + quarter * 32;   // first of this warp's 32 rows
-      const int col_base = tn * BN;
-      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN);
       constexpr int kChunkCols = OUT_F32 ? 32 : 64;                    // 128 bytes of output per row
+      constexpr int kPartCols = C::kNT == 1 ? BN : C::kMmaN;
 #pragma unroll 1
-      for (int c = 0; c < BN / kChunkCols; ++c, ++chunk) {
-        uint32_t v[32], w[32];
-        tmem_ld_32x32b_x32(taddr + (uint32_t)(c * kChunkCols), v);
-        if constexpr (!OUT_F32) tmem_ld_32x32b_x32(taddr + (uint32_t)(c * kChunkCols + 32), w);
-        tmem_ld_wait();
-        // the buffer used two chunks ago must have been read by its store before it is overwritten
-        if (chunk >= 2) {
-          if (lane == 0) bulk_wait_read_1();
+      for (int c = 0; c < C::kNT && ok; ++c) {                         // accumulator parts, in the order they complete
+        const int part = C::kNT == 1 ? buf : c;
+        ok = mbar_wait_timed(bar_tfull + 8 * part, use, args.status, (kRoleEpilogue << 8) | 1, args.trace != nullptr, &wait_epi);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tcgen05_fence_after();
+        const int col_base = tn * BN + c * kPartCols;
+        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(C::kNT == 1 ? buf * BN : c * C::kMmaN);
+        if constexpr (C::kNT == 2 && !OUT_F32) {
+          // Nothing hides this epilogue behind a second accumulator buffer, so the part is emptied into registers
+          // first (packed bf16: 128 registers for 256 columns) and handed back to the MMA issuer at once; staging
+          // and storing then overlap the mainloop that has already resumed.
+          uint32_t pk[kPartCols / 2];
+#pragma unroll
+          for (int q = 0; q < kPartCols / 64; ++q) {
+            uint32_t v[32], w[32];
+            tmem_ld_32x32b_x32(taddr + (uint32_t)(q * 64), v);
+            tmem_ld_32x32b_x32(taddr + (uint32_t)(q * 64 + 32), w);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              pk[q * 32 + j] = pack_bf16(v[2 * j], v[2 * j + 1]);
+              pk[q * 32 + 16 + j] = pack_bf16(w[2 * j], w[2 * j + 1]);
+            }
+          }
+          tcgen05_fence_before();
           __syncwarp();
-        }
-        const uint32_t slice = epi_base + (uint32_t)((warp - 2) * 8192 + (chunk & 1) * 4096);
-        const uint32_t rowaddr = slice + (uint32_t)lane * 128u;
-        const uint32_t sw = (uint32_t)lane & 7u;                       // 128-byte swizzle: 16-byte unit j of row r sits at j ^ (r % 8)
-        if constexpr (OUT_F32) {
+          if (lane == 0) {
+            const uint32_t te = bar_tempty + 8 * part;
+            mbar_arrive_cluster(CG == 1 ? te : mapa(te, 0));
+          }
 #pragma unroll
-          for (uint32_t j = 0; j < 8; ++j)
-            st_shared_16(rowaddr + ((j ^ sw) << 4), v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+          for (int q = 0; q < kPartCols / 64; ++q, ++chunk) {
+            if (chunk >= 2) {
+              if (lane == 0) bulk_wait_read_1();
+              __syncwarp();
+            }
+            const uint32_t slice = epi_base + (uint32_t)((warp - 2) * 8192 + (chunk & 1) * 4096);
+            const uint32_t rowaddr = slice + (uint32_t)lane * 128u;
+            const uint32_t sw = (uint32_t)lane & 7u;
+#pragma unroll
+            for (uint32_t j = 0; j < 8; ++j)
+              st_shared_16(rowaddr + ((j ^ sw) << 4), pk[q * 32 + 4 * j], pk[q * 32 + 4 * j + 1], pk[q * 32 + 4 * j + 2],
+                           pk[q * 32 + 4 * j + 3]);
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+              const int col = col_base + q * 64;
+              if (row0 < args.M && col < args.N) tma_store_2d(&tmC, slice, col, row0);
+              bulk_commit();
+            }
+          }
         } else {
+#pragma unroll 1
+        for (int q = 0; q < kPartCols / kChunkCols; ++q, ++chunk) {
+          uint32_t v[32], w[32];
+          tmem_ld_32x32b_x32(taddr + (uint32_t)(q * kChunkCols), v);
+          if constexpr (!OUT_F32) tmem_ld_32x32b_x32(taddr + (uint32_t)(q * kChunkCols + 32), w);
+          tmem_ld_wait();
+          // the buffer used two chunks ago must have been read by its store before it is overwritten
+          if (chunk >= 2) {
+            if (lane == 0) bulk_wait_read_1();
+            __syncwarp();
+          }
+          const uint32_t slice = epi_base + (uint32_t)((warp - 2) * 8192 + (chunk & 1) * 4096);
+          const uint32_t rowaddr = slice + (uint32_t)lane * 128u;
+          const uint32_t sw = (uint32_t)lane & 7u;                     // 128-byte swizzle: 16-byte unit j of row r sits at j ^ (r % 8)
+          if constexpr (OUT_F32) {
 #pragma unroll
-          for (uint32_t j = 0; j < 4; ++j) {
-            st_shared_16(rowaddr + ((j ^ sw) << 4), pack_bf16(v[8 * j], v[8 * j + 1]), pack_bf16(v[8 * j + 2], v[8 * j + 3]),
-                         pack_bf16(v[8 * j + 4], v[8 * j + 5]), pack_bf16(v[8 * j + 6], v[8 * j + 7]));
-            st_shared_16(rowaddr + (((j + 4) ^ sw) << 4), pack_bf16(w[8 * j], w[8 * j + 1]), pack_bf16(w[8 * j + 2], w[8 * j + 3]),
-                         pack_bf16(w[8 * j + 4], w[8 * j + 5]), pack_bf16(w[8 * j + 6], w[8 * j + 7]));
+            for (uint32_t j = 0; j < 8; ++j)
+              st_shared_16(rowaddr + ((j ^ sw) << 4), v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+          } else {
+#pragma unroll
+            for (uint32_t j = 0; j < 4; ++j) {
+              st_shared_16(rowaddr + ((j ^ sw) << 4), pack_bf16(v[8 * j], v[8 * j + 1]), pack_bf16(v[8 * j + 2], v[8 * j + 3]),
+                           pack_bf16(v[8 * j + 4], v[8 * j + 5]), pack_bf16(v[8 * j + 6], v[8 * j + 7]));
+              st_shared_16(rowaddr + (((j + 4) ^ sw) << 4), pack_bf16(w[8 * j], w[8 * j + 1]), pack_bf16(w[8 * j + 2], w[8 * j + 3]),
+                           pack_bf16(w[8 * j + 4], w[8 * j + 5]), pack_bf16(w[8 * j + 6], w[8 * j + 7]));
+            }
+          }
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            const int col = col_base + q * kChunkCols;
+            if (row0 < args.M && col < args.N) tma_store_2d(&tmC, slice, col, row0);
+            bulk_commit();                                            // also when nothing was stored: keeps the group count in step
           }
         }
-        fence_async_smem();
+        tcgen05_fence_before();
         __syncwarp();
         if (lane == 0) {
-          const int col = col_base + c * kChunkCols;
-          if (row0 < args.M && col < args.N) tma_store_2d(&tmC, slice, col, row0);
-          bulk_commit();                                              // also when nothing was stored: keeps the group count in step
+          const uint32_t te = bar_tempty + 8 * part;
+          mbar_arrive_cluster(CG == 1 ? te : mapa(te, 0));
+        }
         }
       }
-      tcgen05_fence_before();
-      __syncwarp();
-      if (lane == 0) {
-        const uint32_t te = bar_tempty + 8 * buf;
-        mbar_arrive_cluster(CG == 1 ? te : mapa(te, 0));
-        if (args.trace && rank == 0 && warp == 2) {
-          args.trace[s].t_end = globaltimer();
-          args.trace[s].epi_wait_acc = wait_epi;
-        }
+      if (ok && lane == 0 && args.trace && rank == 0 && warp == 2) {
+        args.trace[s].t_end = globaltimer();
+        args.trace[s].epi_wait_acc = wait_epi;
       }
     }
     if (lane == 0) bulk_wait_all();   // every store of this warp has left shared memory and reached global memory
@@ -425,7 +498,7 @@ static int max_units() {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemBytes) != cudaSuccess) return -1;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(sms / CG * CG));
-    cfg.blockDim = dim3(kThreads);
+    cfg.blockDim = dim3(C::kThreads);
     cfg.dynamicSmemBytes = C::kSmemBytes;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -440,7 +513,7 @@ static int max_units() {
 }
 
 int gemm_units(int tile_m, int tile_n, int64_t T) {
-  int64_t units = tile_m == 256 ? (tile_n == 128 ? max_units<2, 128>() : max_units<2, 256>())
+  int64_t units = tile_m == 256 ? (tile_n == 128 ? max_units<2, 128>() : tile_n == 256 ? max_units<2, 256>() : max_units<2, 512>())
                                 : (tile_n == 128 ? max_units<1, 128>() : max_units<1, 256>());
   if (units <= 0) return -1;
   if (const char* e = getenv("SP_MAX_UNITS")) {  // experiments only: cap the number of persistent units
@@ -465,7 +538,7 @@ static int launch_variant(const GemmCall& call, const CUtensorMap& tmA, const CU
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(args.units * CG));
-  cfg.blockDim = dim3(kThreads);
+  cfg.blockDim = dim3(C::kThreads);
   cfg.dynamicSmemBytes = C::kSmemBytes;
   cfg.stream = call.stream;
   cudaLaunchAttribute attr[1];
@@ -493,7 +566,7 @@ static int launch_shape(const GemmCall& call, const CUtensorMap& tmA, const CUte
 
 int launch_gemm(const GemmCall& call) {
   const int cg = call.tile_m / 128;
-  const int bcols = call.tile_n / cg;  // B columns per CTA
+  const int bcols = (call.tile_n > 256 ? 256 : call.tile_n) / cg;  // B columns one CTA supplies to one MMA
   CUtensorMap tmA, tmB, tmC;
   int rc = make_map(&tmC, call.C, call.M, call.N, 32, call.out_f32 != 0);   // one epilogue warp stores 32 rows x 128 bytes
   if (rc != SP_OK) return rc;
@@ -541,6 +614,7 @@ int launch_gemm(const GemmCall& call) {
   args.sched = call.sched;
 
   if (cg == 1) return call.tile_n == 128 ? launch_shape<1, 128>(call, tmA, tmB, tmC, args) : launch_shape<1, 256>(call, tmA, tmB, tmC, args);
+  if (call.tile_n == 512) return launch_shape<2, 512>(call, tmA, tmB, tmC, args);
   return call.tile_n == 128 ? launch_shape<2, 128>(call, tmA, tmB, tmC, args) : launch_shape<2, 256>(call, tmA, tmB, tmC, args);
 }
 

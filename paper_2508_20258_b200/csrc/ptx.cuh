@@ -88,10 +88,9 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t
 // mbar_wait that also adds the cycles spent waiting to *acc when tracing.
 __device__ __forceinline__ bool mbar_wait_timed(uint32_t bar, uint32_t parity, int32_t* status, int code, bool timed,
                                                 uint32_t* acc) {
-  if (mbar_try_wait(bar, parity)) return true;
-  if (!timed) return mbar_wait_slow(bar, parity, status, code);
-  const long long c0 = clock64();
-  const bool ok = mbar_wait_slow(bar, parity, status, code);
+  if (!timed) return mbar_wait(bar, parity, status, code);
+  const long long c0 = clock64();   // try_wait may itself suspend the thread for a while: time the whole wait
+  const bool ok = mbar_wait(bar, parity, status, code);
   *acc += (uint32_t)(clock64() - c0);
   return ok;
 }
@@ -119,6 +118,7 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t sr
                : "memory");
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }

@@ -61,7 +61,7 @@ def test_device_remap_matches_oracle(M, N, tm, tn):
 
 
 # ------------------------------------------------------------------ exact cases
-SHAPES = [(128, 128), (128, 256), (256, 128), (256, 256)]
+SHAPES = [(128, 128), (128, 256), (256, 128), (256, 256), (256, 512)]
 
 
 @pytest.mark.parametrize("tile", SHAPES)
@@ -112,7 +112,8 @@ def test_cfg1_full(scheme, kw):
 
 
 @pytest.mark.parametrize("M,N,K,tile,out", [(640, 896, 1000, (128, 128), "bf16"), (1160, 600, 520, (128, 256), "fp32"),
-                                             (1160, 1096, 776, (256, 256), "bf16"), (904, 648, 1288, (256, 128), "bf16")])
+                                             (1160, 1096, 776, (256, 256), "bf16"), (904, 648, 1288, (256, 128), "bf16"), (1160, 1608, 776, (256, 512), "bf16"),
+                                             (520, 2056, 328, (256, 512), "fp32")])
 @pytest.mark.parametrize("b_is_nk", [False, True])
 def test_ragged_sizes_full(M, N, K, tile, out, b_is_nk):
     """Several tiles, ragged M / N tails, K not a multiple of the 64-wide k-block."""
