@@ -42,7 +42,7 @@ struct Cfg {
   static constexpr int kMmaN = BN > 256 ? 256 : BN;             // N of one tcgen05.mma
   static constexpr int kNT = BN / kMmaN;                        // MMA tiles side by side in one scheduler tile
   static constexpr int kBufs = kNT == 1 ? 2 : 1;                // accumulator buffers of BN columns in the 512 TMEM columns
-  static constexpr int kEpiWarps = 4;                           // one per TMEM lane quarter
+  static constexpr int kEpiWarps = kNT == 1 ? 4 : 8;            // one per TMEM lane quarter and accumulator part
   static constexpr int kThreads = 64 + 32 * kEpiWarps;          // producer warp, MMA warp, epilogue warps
   static constexpr int kMmaCols = kMmaN / CG;                   // columns of B one CTA supplies to one MMA
   static constexpr int kBCols = BN / CG;                        // columns of B held by one CTA
@@ -128,7 +128,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < S; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_empty + 8 * i, 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(bar_tfull + 8 * i, 1); mbar_init(bar_tempty + 8 * i, C::kEpiWarps * CG); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_tfull + 8 * i, 1); mbar_init(bar_tempty + 8 * i, 4 * CG); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -248,6 +248,56 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const bool tracing = args.trace != nullptr;
         uint32_t wait_acc = 0, wait_data = 0;
         if (tracing && lane == 0) args.trace[s].t_mma_begin = globaltimer();
+        if constexpr (C::kNT == 2) {
+          // K-blocks are issued in groups: the first two and the last two k-blocks of a tile as pairs, the rest one by
+          // one.  Inside a group the first MMA tile's MMAs come before the second's.  The first accumulator part is then
+          // complete 1024 cycles of MMAs before the second, and the next tile starts on it equally early: the epilogue
+          // warps of one part drain it while the tensor pipe works on the other.  The body keeps the full look-ahead.
+          int kb = 0;
+          while (kb < KB && ok) {
+            const bool paired = KB >= 4 && (kb == 0 || kb == KB - 2);
+            const int g = paired ? 2 : 1;
+            uint32_t st0 = 0, st1 = 0;
+            for (int i = 0; i < g && ok; ++i) {                    // operands of the whole group must have landed
+              ok = mbar_wait_timed(bar_full + 8 * stage, phase, args.status, (kRoleMma << 8) | 2, tracing, &wait_data);
+              if (i == 0) st0 = (uint32_t)stage; else st1 = (uint32_t)stage;
+              if (++stage == S) { stage = 0; phase ^= 1u; }
+            }
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tcgen05_fence_after();
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+              if (kb == 0) {                                        // the part must have been drained by the previous tile's epilogue
+                ok = mbar_wait_timed(bar_tempty + 8 * c, use ^ 1u, args.status, (kRoleMma << 8) | 1, tracing, &wait_acc);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tcgen05_fence_after();
+              }
+              if (elect_one()) {
+                for (int i = 0; i < g; ++i) {
+                  const uint32_t sa = smem_base + (i == 0 ? st0 : st1) * C::kStageBytes;
+                  const uint32_t sb = sa + C::kABytes + (uint32_t)(c * C::kMmaCols * kBK * 2);
+#pragma unroll
+                  for (int k = 0; k < kBK / kUmmaK; ++k) {
+                    const uint64_t da = smem_desc(sa + k * (kUmmaK * 2), 16, 1024);
+                    const uint64_t db = smem_desc(sb + k * args.b_kstep, args.b_lbo, args.b_sbo);
+                    umma_bf16<CG>(tmem_base + (uint32_t)(c * C::kMmaN), da, db, idesc, (uint32_t)(((kb + i) | k) != 0));
+                  }
+                }
+                if (kb + g == KB) umma_commit<CG>(bar_tfull + 8 * c);     // this part is complete
+              }
+              __syncwarp();
+            }
+            if (!ok) break;
+            if (elect_one()) {
+              umma_commit<CG>(bar_empty + 8 * st0);
+              if (g == 2) umma_commit<CG>(bar_empty + 8 * st1);
+            }
+            __syncwarp();
+            kb += g;
+          }
+        } else {
         for (int kb = 0; kb < KB && ok; ++kb) {
           ok = mbar_wait_timed(bar_full + 8 * stage, phase, args.status, (kRoleMma << 8) | 2, tracing, &wait_data);
           ok = __all_sync(0xffffffffu, ok);
@@ -281,6 +331,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           __syncwarp();
           if (++stage == S) { stage = 0; phase ^= 1u; }
         }
+        }
         if (tracing && lane == 0) {
           sp_trace_rec* rec = args.trace + s;
           rec->mma_wait_data = wait_data; rec->mma_wait_acc = wait_acc; rec->t_mma_issued = globaltimer();
@@ -291,6 +342,90 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   } else {
     // ---------------------------------------------------------------- epilogue
     const int quarter = warp & 3;  // TMEM lanes [32*quarter, 32*quarter + 32) are this warp's
+    if constexpr (C::kNT == 2) {
+      // Two MMA tiles per scheduler tile: no second accumulator buffer hides this epilogue.  Four warps serve each
+      // accumulator part.  A warp empties its 32 lanes x 256 columns into registers (packed bf16), hands the part back
+      // to the MMA issuer at once, and only then stages and stores (one 4 KiB slice per warp), which overlaps the
+      // mainloop that has already resumed; the other part's warps are never held up by these stores.
+      const int c = (warp - 2) >> 2;                               // the part this warp serves
+      const uint32_t slice = epi_base + (uint32_t)((warp - 2) * 4096);
+      const uint32_t rowaddr = slice + (uint32_t)lane * 128u;
+      const uint32_t sw = (uint32_t)lane & 7u;
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c * C::kMmaN);
+      int it2 = 0;
+      bool ok2 = true;
+      for (int s = s_first; s < s_end && ok2; s += s_step, ++it2) {
+        const int t = tile_of_slot(args, s);
+        const int tm = t / Tn, tn = t - tm * Tn;
+        const uint32_t use = (uint32_t)it2 & 1u;
+        const int row0 = tm * TILE_M + (int)rank * 128 + quarter * 32;
+        const int col_base = tn * BN + c * C::kMmaN;
+        uint32_t wait_epi = 0;
+        ok2 = mbar_wait_timed(bar_tfull + 8 * c, use, args.status, (kRoleEpilogue << 8) | 1, args.trace != nullptr, &wait_epi);
+        ok2 = __all_sync(0xffffffffu, ok2);
+        if (!ok2) break;
+        tcgen05_fence_after();
+        if constexpr (!OUT_F32) {
+          uint32_t pk[C::kMmaN / 2];
+#pragma unroll
+          for (int q = 0; q < C::kMmaN / 32; ++q) {
+            uint32_t v[32];
+            tmem_ld_32x32b_x32(taddr + (uint32_t)(q * 32), v);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 16; ++j) pk[q * 16 + j] = pack_bf16(v[2 * j], v[2 * j + 1]);
+          }
+          tcgen05_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(mapa(bar_tempty + 8 * c, 0));
+#pragma unroll
+          for (int q = 0; q < C::kMmaN / 64; ++q) {
+            if (lane == 0) bulk_wait_read_0();                      // the slice's previous store has read it
+            __syncwarp();
+#pragma unroll
+            for (uint32_t j = 0; j < 8; ++j)
+              st_shared_16(rowaddr + ((j ^ sw) << 4), pk[q * 32 + 4 * j], pk[q * 32 + 4 * j + 1], pk[q * 32 + 4 * j + 2],
+                           pk[q * 32 + 4 * j + 3]);
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+              const int col = col_base + q * 64;
+              if (row0 < args.M && col < args.N) tma_store_2d(&tmC, slice, col, row0);
+              bulk_commit();
+            }
+          }
+        } else {
+          // fp32 output: 256 columns do not fit in registers; chunk by chunk, the part is released at the end
+#pragma unroll 1
+          for (int q = 0; q < C::kMmaN / 32; ++q) {
+            uint32_t v[32];
+            tmem_ld_32x32b_x32(taddr + (uint32_t)(q * 32), v);
+            tmem_ld_wait();
+            if (lane == 0) bulk_wait_read_0();
+            __syncwarp();
+#pragma unroll
+            for (uint32_t j = 0; j < 8; ++j)
+              st_shared_16(rowaddr + ((j ^ sw) << 4), v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+              const int col = col_base + q * 32;
+              if (row0 < args.M && col < args.N) tma_store_2d(&tmC, slice, col, row0);
+              bulk_commit();
+            }
+          }
+          tcgen05_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(mapa(bar_tempty + 8 * c, 0));
+        }
+        if (lane == 0 && args.trace && rank == 0 && warp == 6) {   // the second part finishes last
+          args.trace[s].t_end = globaltimer();
+          args.trace[s].epi_wait_acc = wait_epi;
+        }
+      }
+      if (lane == 0) bulk_wait_all();
+      __syncwarp();
+    } else {
     int it = 0;
     int chunk = 0;                 // staging buffers alternate per stored chunk, across tiles
     bool ok = true;
@@ -312,51 +447,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         tcgen05_fence_after();
         const int col_base = tn * BN + c * kPartCols;
         const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(C::kNT == 1 ? buf * BN : c * C::kMmaN);
-        if constexpr (C::kNT == 2 && !OUT_F32) {
-          // Nothing hides this epilogue behind a second accumulator buffer, so the part is emptied into registers
-          // first (packed bf16: 128 registers for 256 columns) and handed back to the MMA issuer at once; staging
-          // and storing then overlap the mainloop that has already resumed.
-          uint32_t pk[kPartCols / 2];
-#pragma unroll
-          for (int q = 0; q < kPartCols / 64; ++q) {
-            uint32_t v[32], w[32];
-            tmem_ld_32x32b_x32(taddr + (uint32_t)(q * 64), v);
-            tmem_ld_32x32b_x32(taddr + (uint32_t)(q * 64 + 32), w);
-            tmem_ld_wait();
-#pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              pk[q * 32 + j] = pack_bf16(v[2 * j], v[2 * j + 1]);
-              pk[q * 32 + 16 + j] = pack_bf16(w[2 * j], w[2 * j + 1]);
-            }
-          }
-          tcgen05_fence_before();
-          __syncwarp();
-          if (lane == 0) {
-            const uint32_t te = bar_tempty + 8 * part;
-            mbar_arrive_cluster(CG == 1 ? te : mapa(te, 0));
-          }
-#pragma unroll
-          for (int q = 0; q < kPartCols / 64; ++q, ++chunk) {
-            if (chunk >= 2) {
-              if (lane == 0) bulk_wait_read_1();
-              __syncwarp();
-            }
-            const uint32_t slice = epi_base + (uint32_t)((warp - 2) * 8192 + (chunk & 1) * 4096);
-            const uint32_t rowaddr = slice + (uint32_t)lane * 128u;
-            const uint32_t sw = (uint32_t)lane & 7u;
-#pragma unroll
-            for (uint32_t j = 0; j < 8; ++j)
-              st_shared_16(rowaddr + ((j ^ sw) << 4), pk[q * 32 + 4 * j], pk[q * 32 + 4 * j + 1], pk[q * 32 + 4 * j + 2],
-                           pk[q * 32 + 4 * j + 3]);
-            fence_async_smem();
-            __syncwarp();
-            if (lane == 0) {
-              const int col = col_base + q * 64;
-              if (row0 < args.M && col < args.N) tma_store_2d(&tmC, slice, col, row0);
-              bulk_commit();
-            }
-          }
-        } else {
+        {
 #pragma unroll 1
         for (int q = 0; q < kPartCols / kChunkCols; ++q, ++chunk) {
           uint32_t v[32], w[32];
@@ -407,6 +498,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     }
     if (lane == 0) bulk_wait_all();   // every store of this warp has left shared memory and reached global memory
     __syncwarp();
+    }
   }
 
   // ------------------------------------------------------------------ teardown
