@@ -33,6 +33,7 @@ L2_BYTES = 126 * 2 ** 20
 # DRAM bytes per launch of the GEMM kernel from the ncu captures summarised under profiles/
 # (dram__bytes_read.sum + dram__bytes_write.sum), keyed by (workload, tile, scheme spec); None = not captured.
 NCU_DRAM_BYTES = {
+    ("cfg3", "256x512", "group_n:8"): 0.940e9,   # profiles/gemm_kernel_cfg3_256x512_full.md
     ("cfg3", "256x256", "die_split:m:group_m:8:p"): 1.071e9,   # profiles/l2_hit_rate_per_scheme.md
     ("cfg5", "256x256", "die_split:m:group_m:8:p"): 1.247e9,
     ("cfg3", "256x256", "group_m:8"): 1.200e9,   # profiles/gemm_kernel_cfg3_group_m8_full.md (mean of 2 launches)
@@ -96,6 +97,10 @@ SWEEPS = {
 DEFAULT_SCHEME = {"cfg1": "group_m:2", "cfg2": "group_m:8", "cfg3": "die_split:m:group_m:8:p", "cfg4": "row_major",
                   "cfg5": "die_split:m:group_m:8:p"}
 FALLBACK_SCHEME = {"cfg3": "group_m:8", "cfg5": "group_m:16"}   # if the topology probe finds no two-way L2 structure
+# 8192^3 is timed with two 256x256 2-CTA MMA tiles per scheduler tile (they share the A panel: a quarter less operand
+# traffic from L2); the plain 256x256 scheduler tile is timed beside it and reported in the same line.
+DEFAULT_TILE = {"cfg3": "256x512"}
+DEFAULT_SCHEME_BY_TILE = {("cfg3", "256x512"): "group_n:8", ("cfg5", "256x512"): "die_split:m:group_m:8:p"}
 
 
 def dist_env():
@@ -186,6 +191,8 @@ def run_ours(args) -> int:
     else:
         w = synth.WORKLOADS[args.workload]
         _, A, B = synth.make_workload(args.workload, b_is_nk=bool(b_nk))
+    if not args.tile and args.workload in DEFAULT_TILE and not (args.sweep or args.sweep_sustained or args.profile_sweep):
+        args.tile = DEFAULT_TILE[args.workload]
     tile_m, tile_n = (int(v) for v in args.tile.split("x")) if args.tile else (w.tile_m, w.tile_n)
     out_f32 = int(w.out_dtype == "fp32")
     dA = torch.from_numpy(A.view(np.int16)).cuda().view(torch.bfloat16)
@@ -228,7 +235,7 @@ def run_ours(args) -> int:
         print(json.dumps({"profile_sweep": w.name, "tile": f"{tile_m}x{tile_n}", "launch_order": specs}), flush=True)
         return 0
 
-    spec = args.scheme or DEFAULT_SCHEME[args.workload]
+    spec = args.scheme or DEFAULT_SCHEME_BY_TILE.get((args.workload, f"{tile_m}x{tile_n}")) or DEFAULT_SCHEME[args.workload]
     scheme, p = params_for(spec)
     try:
         sp.gemm(dA, dB, dC, scheme, p, stream)
@@ -273,6 +280,27 @@ def run_ours(args) -> int:
         sp.gemm(dA, dB, dC, row_scheme, row_p, stream)
     row_ms = time_steps(sp, dA, dB, dC, row_scheme, row_p, args.steps, stream) / args.steps
 
+    # the workload's nominal scheduler tile, when the timed one differs from it
+    nominal = None
+    if (tile_m, tile_n) != (w.tile_m, w.tile_n):
+        nspec = DEFAULT_SCHEME[args.workload]
+        ns, kw = parse_scheme(nspec)
+        npar = sp.make_params(tile_m=w.tile_m, tile_n=w.tile_n, out_dtype=out_f32, b_layout=b_nk, **kw)
+        try:
+            sp.gemm(dA, dB, dC, ns, npar, stream)
+        except sp.SpError:
+            nspec = FALLBACK_SCHEME.get(args.workload, "row_major")
+            ns, kw = parse_scheme(nspec)
+            npar = sp.make_params(tile_m=w.tile_m, tile_n=w.tile_n, out_dtype=out_f32, b_layout=b_nk, **kw)
+        for _ in range(3):
+            sp.gemm(dA, dB, dC, ns, npar, stream)
+        n_ms = time_steps(sp, dA, dB, dC, ns, npar, args.steps, stream) / args.steps
+        nrs, nrkw = parse_scheme("row_major")
+        nrp = sp.make_params(tile_m=w.tile_m, tile_n=w.tile_n, out_dtype=out_f32, b_layout=b_nk)
+        nr_ms = time_steps(sp, dA, dB, dC, nrs, nrp, args.steps, stream) / args.steps
+        nominal = {"tile": f"{w.tile_m}x{w.tile_n}", "scheme": nspec, "ms_per_step": n_ms, "tflops": flops / n_ms / 1e9,
+                   "row_major_tflops": flops / nr_ms / 1e9, "speedup_over_row_major": nr_ms / n_ms}
+
     # context only: cuBLAS (torch.matmul) on the same tensors, same back-to-back protocol, same thermal state
     cublas = None
     if dC.dtype == torch.bfloat16 and not b_nk:
@@ -314,7 +342,7 @@ def run_ours(args) -> int:
     launch_ms = ms_total / args.steps
     achieved = flops / launch_ms / 1e9
     roofline = {
-        "bound": "tensor", "kernel": f"gemm_kernel<CG={tile_m // 128},BN={tile_n}>", "achieved": achieved,
+        "bound": "tensor", "kernel": f"gemm_kernel<CG={tile_m // 128},BN={tile_n}>" + (" (two 256x256 2-CTA MMA tiles sharing A)" if tile_n == 512 else ""), "achieved": achieved,
         "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops_sustained"],
         "peak_kind": f"cuBLAS bf16 sustained, {peaks['source']}; launches are timed back to back inside the step loop",
         "traffic": NCU_DRAM_BYTES.get((w.name, f"{tile_m}x{tile_n}", spec)),
@@ -347,7 +375,7 @@ def run_ours(args) -> int:
                        "parallelism": "replicas only" if world > 1 else "1 GPU"},
             "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": args.steps,
             "clocks": clocks,
-            "cublas_context": cublas,
+            "nominal_tile": nominal, "cublas_context": cublas,
             "row_major": {"ms_per_step": row_ms, "tflops": flops / row_ms / 1e9, "speedup_of_scheme": row_ms / launch_ms},
         }
         print(json.dumps(line), flush=True)

@@ -243,7 +243,9 @@ def test_topology_probe_finds_two_equal_l2_halves_and_pairs_stay_together():
     assert lat.shape == (len(die), sp.binding.PROBE_LINES) and (lat > 0).all()
     if conf < 0.8:
         pytest.skip("no two-way L2 structure measured on this device")
-    assert set(die.tolist()) == {0, 1} and (die == 0).sum() == (die == 1).sum()
+    # the two halves need not be equal: parts differ in which SMs are fused off (74/74 and 72/76 have been seen)
+    n0, n1 = int((die == 0).sum()), int((die == 1).sum())
+    assert set(die.tolist()) == {0, 1} and n0 % 2 == 0 and n1 % 2 == 0 and abs(n0 - n1) <= len(die) // 8
     assert (die[0::2] == die[1::2]).all()          # the two SMs of a CTA pair share a half
     near = np.median(lat[die == 0][:, :], axis=0)  # per line: latency seen from half 0 ...
     far = np.median(lat[die == 1][:, :], axis=0)   # ... and from half 1: one of them is the home half

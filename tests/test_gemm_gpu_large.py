@@ -46,19 +46,25 @@ def sample_tiles(Tm, Tn, seed):
 
 
 CASES = [
-    # the die-pinned split (flags=2) is the order the benchmark times on cfg3 and cfg5
-    ("cfg3", [(sp.ROW_MAJOR, {}), (sp.GROUP_M, dict(group=8)), (sp.HILBERT, {}),
+    # cfg3 with two MMA tiles per scheduler tile (256x512) and GROUP_N(8) is what the benchmark times by default
+    ("cfg3", (256, 512), [(sp.GROUP_N, dict(group=8)), (sp.ROW_MAJOR, {}),
+                          (sp.DIE_SPLIT, dict(split_axis=1, inner_scheme=sp.GROUP_N, inner_group=4, flags=2))]),
+    # the die-pinned split (flags=2) is the order the benchmark times on the 256x256 tile and on cfg5
+    ("cfg3", None, [(sp.ROW_MAJOR, {}), (sp.GROUP_M, dict(group=8)), (sp.HILBERT, {}),
               (sp.DIE_SPLIT, dict(split_axis=0, inner_scheme=sp.GROUP_M, inner_group=8)),
               (sp.DIE_SPLIT, dict(split_axis=0, inner_scheme=sp.GROUP_M, inner_group=8, flags=2))]),
-    ("cfg4", [(sp.ROW_MAJOR, {}), (sp.GROUP_M, dict(group=4)), (sp.GROUP_N, dict(group=2))]),
-    ("cfg5", [(sp.GROUP_M, dict(group=16)), (sp.HILBERT, {}),
+    ("cfg4", None, [(sp.ROW_MAJOR, {}), (sp.GROUP_M, dict(group=4)), (sp.GROUP_N, dict(group=2))]),
+    ("cfg5", None, [(sp.GROUP_M, dict(group=16)), (sp.HILBERT, {}),
               (sp.DIE_SPLIT, dict(split_axis=0, inner_scheme=sp.GROUP_M, inner_group=8, flags=2))]),
 ]
 
 
-@pytest.mark.parametrize("name,schemes", CASES)
-def test_large_workload_sampled(name, schemes):
+@pytest.mark.parametrize("name,tile,schemes", CASES)
+def test_large_workload_sampled(name, tile, schemes):
     w, A, B = synth.make_workload(name)
+    if tile is not None:
+        import dataclasses
+        w = dataclasses.replace(w, tile_m=tile[0], tile_n=tile[1])
     dA, dB = dev_bf16(A), dev_bf16(B)
     dC = torch.empty((w.M, w.N), dtype=torch.bfloat16, device="cuda")
     rows = sample_rows(w.M, w.tile_m)
