@@ -6,11 +6,12 @@
 // traffic from L2 per flop, at the price of an epilogue that is not hidden behind the next tile's mainloop.
 // Unit u runs slots u, u + units, u + 2*units, ...; slot s computes tile slot_to_tile(s).
 //
-// Warp roles (192 threads):
-//   warp 0  lane 0 : TMA producer   -- A and B k-blocks into a ring of 128B-swizzled smem stages
-//   warp 1  lane 0 : MMA issuer     -- tcgen05.mma, fp32 accumulators in TMEM (two buffers);
-//                                      the warp also owns TMEM alloc / dealloc
-//   warps 2..5     : epilogue       -- tcgen05.ld, convert, stage 32 rows x 128 bytes per warp in swizzled smem,
+// Warp roles (192 threads; 320 for BN = 512):
+//   warp 0         : TMA producer   -- A and B k-blocks into a ring of 128B-swizzled smem stages (whole warp in the
+//                                      loop, one elected lane issues)
+//   warp 1         : MMA issuer     -- tcgen05.mma, fp32 accumulators in TMEM (two buffers, or two parts of one tile
+//                                      for BN = 512); elected lane issues; the warp also owns TMEM alloc / dealloc
+//   warps 2..5     : epilogue       -- (2..9 for BN = 512, four per accumulator part) tcgen05.ld, convert, stage 32 rows x 128 bytes per warp in swizzled smem,
 //                                      TMA store (full 128-byte rows; ragged edges clipped by the tensor map)
 //
 // Synchronisation: mbarriers only.  full[s]/empty[s] per smem stage, tmem_full[b]/tmem_empty[b]
