@@ -701,6 +701,11 @@ int launch_gemm(const GemmCall& call) {
                 args.units_on_die[0] + args.units_on_die[1]);
       return SP_ERR_UNSUPPORTED;
     }
+    // The tile space is cut into two equal halves, the SMs not always (72 / 76 has been measured): each half is
+    // served by half of the units; the surplus units of the larger side take the top ranks of the other half
+    // (the same rule that covers uneven placement), so both halves finish together.
+    args.units_on_die[0] = (args.units + 1) / 2;
+    args.units_on_die[1] = args.units / 2;
     cudaError_t ce = cudaMemsetAsync(args.die_count, 0, 2 * sizeof(int32_t), call.stream);
     if (ce != cudaSuccess) { set_error("clearing the die counters failed: %s", cudaGetErrorString(ce)); return SP_ERR_CUDA; }
   }

@@ -230,8 +230,14 @@ def test_die_pinned_schedule_keeps_each_half_on_one_l2_half():
             assert tr["tile"].tolist() == want                       # record s still describes slot s
             h0 = len(R.die_split_halves(-(-M // tile[0]), -(-N // tile[1]), axis, sp.GROUP_M, 4)[0])
             on_die = die[tr["smid"]]
-            assert len(set(on_die[:h0].tolist())) == 1 and len(set(on_die[h0:].tolist())) == 1
-            assert on_die[0] != on_die[-1]
+            # each half runs on one L2 half; where the GPU's halves have unequal SM counts (72 / 76) the surplus
+            # units of the larger side help out on the other half of the tile space
+            d0 = int(np.bincount(on_die[:h0], minlength=2).argmax())
+            d1 = int(np.bincount(on_die[h0:], minlength=2).argmax())
+            assert d0 != d1
+            assert (on_die[:h0] == d0).mean() >= 0.9 and (on_die[h0:] == d1).mean() >= 0.9
+            if (die == 0).sum() == (die == 1).sum():
+                assert (on_die[:h0] == d0).all() and (on_die[h0:] == d1).all()
     with pytest.raises(sp.SpError) as e:                              # pinning is defined for the split order only
         sp.gemm(dA, dB, ref, sp.GROUP_M, sp.make_params(tile_m=256, tile_n=256, group=4, flags=2))
     assert e.value.status == sp.ERR_INVALID_ARG
