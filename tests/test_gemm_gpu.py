@@ -269,3 +269,19 @@ def test_bounded_wait_expires_with_a_status_and_leaves_the_context_usable():
     ref, _ = G.gemm_full(A, B)
     got, _ = run_gemm(A, B, sp.ROW_MAJOR, (256, 256), "fp32")
     assert np.array_equal(got, ref)
+
+
+def test_device_remap_matches_oracle_on_random_grids():
+    """Seeded random grids and parameters: the scheduler's device code against the enumerating oracle."""
+    rng = np.random.default_rng(2024)
+    for _ in range(40):
+        Tm, Tn = int(rng.integers(1, 90)), int(rng.integers(1, 90))
+        G, X, W = int(rng.integers(1, 20)), int(rng.integers(1, 12)), int(rng.integers(0, 200))
+        inner = int(rng.choice([sp.ROW_MAJOR, sp.COL_MAJOR, sp.GROUP_M, sp.GROUP_N, sp.MORTON, sp.HILBERT]))
+        axis, inter, serp = int(rng.integers(2)), int(rng.integers(2)), int(rng.integers(2)) * 4
+        for scheme, kw in [(sp.GROUP_M, dict(group=G, flags=serp)), (sp.GROUP_N, dict(group=G, flags=serp)),
+                           (sp.MORTON, {}), (sp.HILBERT, {}), (sp.XCD, dict(num_xcds=X, wave=W, xcd_balanced=1)),
+                           (sp.DIE_SPLIT, dict(split_axis=axis, inner_scheme=inner, inner_group=G, interleave=inter, flags=serp))]:
+            want = R.tile_map(Tm * 64, Tn * 64, 64, 64, scheme, R.Params(**kw))
+            got = sp.tile_map_device(Tm * 64, Tn * 64, 64, 64, scheme, sp.make_params(**kw)).cpu().numpy().tolist()
+            assert got == want, (Tm, Tn, scheme, kw)
