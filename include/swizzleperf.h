@@ -204,6 +204,15 @@ int sp_probe_dispatch(int32_t n_blocks, int32_t cluster, int32_t* smid_host, uin
 #define SP_PROBE_LINES 128
 int sp_probe_topology(int32_t* sm_to_die_host, int32_t* n_sm, float* confidence, uint32_t* lat_host);
 
+/* Effective L2 capacity probe (counterpart of the paper's "L2 size per XCD" context).  For each working-set size every
+ * participating SM reads the whole set repeatedly with loads that bypass L1; the aggregate read rate of the repeat passes
+ * drops once the set no longer fits in what the L2 holds for those readers.
+ *   sizes_bytes : HOST, n_sizes (1..256) working-set sizes, each a multiple of 16 in [4 KiB, 1 GiB].
+ *   half        : -1 = all SMs read; 0 / 1 = only the SMs measured on that L2 half (runs the topology probe if needed).
+ *   gbps_out    : HOST, n_sizes aggregate read rates in GB/s.
+ * Synchronous; allocates and frees a buffer of the largest size. */
+int sp_probe_l2_capacity(int32_t n_sizes, const int64_t* sizes_bytes, int32_t half, float* gbps_out);
+
 /* Self-test (host only) of the rank assignment of die-pinned scheduling: with n0 / n1 units expected on the two L2
  * halves and arrivals0 of the n0 + n1 units actually landing on half 0, every (half, rank) pair must be handed out
  * exactly once.  Returns SP_OK, or SP_ERR_NOT_BIJECTIVE if the assignment would skip or repeat work. */

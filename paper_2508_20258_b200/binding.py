@@ -58,7 +58,7 @@ TRACE_DTYPE = np.dtype([("slot", "<i4"), ("tile", "<i4"), ("smid", "<i4"), ("uni
 
 EXPORTS = ["sp_tile_count", "sp_tile_map", "sp_tile_map_device", "sp_gemm", "sp_gemm_trace", "sp_gemm_host",
            "sp_gemm_noalloc", "sp_transpose", "sp_gemm_units",
-           "sp_probe_dispatch", "sp_probe_topology", "sp_selftest_timeout", "sp_selftest_pinned_tickets", "sp_get_status", "sp_last_error", "sp_shutdown"]
+           "sp_probe_dispatch", "sp_probe_topology", "sp_probe_l2_capacity", "sp_selftest_timeout", "sp_selftest_pinned_tickets", "sp_get_status", "sp_last_error", "sp_shutdown"]
 
 
 class SpError(RuntimeError):
@@ -101,6 +101,8 @@ def lib() -> ctypes.CDLL:
         L.sp_probe_dispatch.argtypes = [i32, i32, vp, vp]
         L.sp_probe_topology.restype = ctypes.c_int
         L.sp_probe_topology.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_float), vp]
+        L.sp_probe_l2_capacity.restype = ctypes.c_int
+        L.sp_probe_l2_capacity.argtypes = [i32, vp, i32, vp]
         L.sp_selftest_pinned_tickets.restype = ctypes.c_int
         L.sp_selftest_pinned_tickets.argtypes = [i32, i32, i32]
         L.sp_selftest_timeout.restype = ctypes.c_int
@@ -283,6 +285,14 @@ def probe_topology():
     conf = ctypes.c_float(0)
     _check(lib().sp_probe_topology(die.ctypes.data, ctypes.byref(n), ctypes.byref(conf), lat.ctypes.data))
     return die[:n.value].copy(), float(conf.value), lat[:n.value * PROBE_LINES].reshape(n.value, PROBE_LINES).copy()
+
+
+def probe_l2_capacity(sizes_bytes, half: int = -1) -> np.ndarray:
+    """Aggregate re-read rate (GB/s) per working-set size; half = -1 all SMs, 0 / 1 one L2 half's SMs only."""
+    sizes = np.ascontiguousarray(np.asarray(sizes_bytes, dtype=np.int64))
+    out = np.zeros(len(sizes), dtype=np.float32)
+    _check(lib().sp_probe_l2_capacity(len(sizes), sizes.ctypes.data, half, out.ctypes.data))
+    return out
 
 
 def selftest_timeout(timeout_us: int):

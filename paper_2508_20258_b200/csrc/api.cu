@@ -502,6 +502,22 @@ int sp_probe_topology(int32_t* sm_to_die_host, int32_t* n_sm, float* confidence,
   return probe_topology(sm_to_die_host, n_sm, confidence, lat_host);
 }
 
+int sp_probe_l2_capacity(int32_t n_sizes, const int64_t* sizes_bytes, int32_t half, float* gbps_out) {
+  if (n_sizes < 1 || n_sizes > 256 || !sizes_bytes || !gbps_out || half < -1 || half > 1) { set_error("bad probe arguments"); return SP_ERR_INVALID_ARG; }
+  int dev = 0;
+  int rc = current_device(&dev);
+  if (rc != SP_OK) return rc;
+  uint32_t mask[8] = {};
+  if (half >= 0) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    DeviceState* ds = device_state(dev);
+    rc = get_die_map(ds);
+    if (rc != SP_OK) return rc;
+    for (int i = 0; i < 8; ++i) mask[i] = ds->die_mask[i];
+  }
+  return probe_l2_capacity(n_sizes, sizes_bytes, half, mask, gbps_out);
+}
+
 int sp_selftest_pinned_tickets(int32_t n0, int32_t n1, int32_t arrivals0) {
   if (n0 < 0 || n1 < 0 || arrivals0 < 0 || arrivals0 > n0 + n1 || n0 + n1 > (1 << 20)) { set_error("bad arguments"); return SP_ERR_INVALID_ARG; }
   std::vector<int> taken((size_t)(n0 + n1), 0);

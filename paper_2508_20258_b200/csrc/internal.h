@@ -65,6 +65,7 @@ int launch_transpose(const void* in, void* out, int64_t M, int64_t N, const Sche
 int selftest_timeout(int32_t* status_dev, int timeout_us, int32_t* code_host, int64_t* waited_us_host);
 int probe_dispatch(int n_blocks, int cluster, int32_t* smid_host, uint64_t* start_host);
 int probe_topology(int32_t* sm_to_die_host, int32_t* n_sm, float* confidence, uint32_t* lat_host);
+int probe_l2_capacity(int n_sizes, const int64_t* sizes_bytes, int half, const uint32_t* die_mask_host, float* gbps_out);
 // Size of half 0 of a DIE_SPLIT schedule, in slots.
 inline int die_split_half0(const Sched& c) {
   return c.axis == 0 ? ((c.Tm + 1) / 2) * c.Tn : ((c.Tn + 1) / 2) * c.Tm;

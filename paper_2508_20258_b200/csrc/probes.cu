@@ -127,3 +127,77 @@ int probe_topology(int32_t* sm_to_die_host, int32_t* n_sm_out, float* confidence
 }
 
 }  // namespace sp
+
+namespace sp {
+
+// ------------------------------------------------------------------ effective L2 capacity
+// Every participating CTA (one per SM) reads the whole working set with 16-byte loads that bypass L1; the pass is
+// repeated, so the rate of the later passes tells whether the set still fits in what the L2 can hold for these readers.
+// With `half` >= 0 only the CTAs on that L2 half take part.
+__global__ void probe_capacity_kernel(const uint4* __restrict__ buf, size_t n16, int passes, int half, const uint32_t* die_mask,
+                                      uint32_t* sink_out) {
+  uint32_t smid;
+  asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+  if (half >= 0 && (int)((die_mask[(smid >> 5) & 7] >> (smid & 31)) & 1u) != half) return;
+  uint32_t acc = 0;
+  for (int p = 0; p < passes; ++p) {
+    // CTAs start at different offsets so that they do not all hit the same lines at the same time
+    const size_t start = ((size_t)blockIdx.x * 4099u * 64u) % n16;
+    for (size_t i = threadIdx.x; i < n16; i += blockDim.x) {
+      size_t j = start + i;
+      if (j >= n16) j -= n16;
+      uint4 v;
+      asm volatile("ld.global.cg.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(buf + j));
+      acc += v.x ^ v.y ^ v.z ^ v.w;
+    }
+  }
+  if (acc == 0x12345678u) *sink_out = acc;   // keeps the loads alive
+}
+
+int probe_l2_capacity(int n_sizes, const int64_t* sizes_bytes, int half, const uint32_t* die_mask_host, float* gbps_out) {
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+    set_error("cannot query the device");
+    return SP_ERR_CUDA;
+  }
+  int64_t max_bytes = 0;
+  for (int i = 0; i < n_sizes; ++i) {
+    if (sizes_bytes[i] < 4096 || sizes_bytes[i] > (1ll << 30) || (sizes_bytes[i] % 16) != 0) { set_error("bad working-set size"); return SP_ERR_INVALID_ARG; }
+    if (sizes_bytes[i] > max_bytes) max_bytes = sizes_bytes[i];
+  }
+  uint4* d_buf = nullptr;
+  uint32_t *d_mask = nullptr, *d_sink = nullptr;
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  cudaError_t e = cudaMalloc(&d_buf, (size_t)max_bytes);
+  if (e == cudaSuccess) e = cudaMalloc(&d_mask, 8 * sizeof(uint32_t));
+  if (e == cudaSuccess) e = cudaMalloc(&d_sink, sizeof(uint32_t));
+  if (e == cudaSuccess) e = cudaMemset(d_buf, 1, (size_t)max_bytes);
+  if (e == cudaSuccess) e = cudaMemcpy(d_mask, die_mask_host, 8 * sizeof(uint32_t), cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaEventCreate(&e0);
+  if (e == cudaSuccess) e = cudaEventCreate(&e1);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(probe_capacity_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  const int passes = 4;
+  for (int i = 0; i < n_sizes && e == cudaSuccess; ++i) {
+    const size_t n16 = (size_t)sizes_bytes[i] / 16;
+    probe_capacity_kernel<<<sms, 512, 200 * 1024>>>(d_buf, n16, 1, half, d_mask, d_sink);          // warm pass
+    cudaEventRecord(e0);
+    probe_capacity_kernel<<<sms, 512, 200 * 1024>>>(d_buf, n16, passes, half, d_mask, d_sink);
+    cudaEventRecord(e1);
+    e = cudaEventSynchronize(e1);
+    float ms = 0.f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+    int readers = sms;
+    if (half >= 0) {
+      readers = 0;
+      for (int s = 0; s < sms; ++s) readers += (int)((die_mask_host[(s >> 5) & 7] >> (s & 31)) & 1u) == half;
+    }
+    gbps_out[i] = ms > 0.f ? (float)((double)sizes_bytes[i] * passes * readers / (ms * 1e6)) : 0.f;
+  }
+  if (e0) cudaEventDestroy(e0);
+  if (e1) cudaEventDestroy(e1);
+  cudaFree(d_buf); cudaFree(d_mask); cudaFree(d_sink);
+  if (e != cudaSuccess) { set_error("capacity probe failed: %s", cudaGetErrorString(e)); return SP_ERR_CUDA; }
+  return SP_OK;
+}
+
+}  // namespace sp

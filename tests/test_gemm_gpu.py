@@ -285,3 +285,12 @@ def test_device_remap_matches_oracle_on_random_grids():
             want = R.tile_map(Tm * 64, Tn * 64, 64, 64, scheme, R.Params(**kw))
             got = sp.tile_map_device(Tm * 64, Tn * 64, 64, 64, scheme, sp.make_params(**kw)).cpu().numpy().tolist()
             assert got == want, (Tm, Tn, scheme, kw)
+
+
+def test_l2_capacity_probe_sees_the_knee():
+    MB = 1 << 20
+    rates = sp.probe_l2_capacity([16 * MB, 256 * MB], -1)
+    assert rates.shape == (2,) and (rates > 0).all()
+    assert rates[0] > 1.3 * rates[1]          # 16 MiB is served from L2, 256 MiB is not
+    with pytest.raises(sp.SpError):
+        sp.probe_l2_capacity([100], -1)       # not a multiple of 16, below the minimum
