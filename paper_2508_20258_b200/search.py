@@ -58,9 +58,19 @@ def default_candidates(units: int) -> List[Tuple[str, int, Dict]]:
     return c
 
 
-def search(A, B, C, tile: Tuple[int, int] = (256, 256), candidates: Optional[Sequence[Tuple[str, int, Dict]]] = None,
+def search(A, B, C, tile=(256, 256), candidates: Optional[Sequence[Tuple[str, int, Dict]]] = None,
            launches: int = 50, out_dtype: int = 0, b_layout: int = 0, verbose: bool = False) -> SearchResult:
-    """Tries every candidate order on C = A.B (CUDA tensors) and returns the history and the fastest valid one."""
+    """Tries every candidate order on C = A.B (CUDA tensors) and returns the history and the fastest valid one.
+    `tile` is one (tile_m, tile_n) or a list of them; every candidate is tried under every tile shape."""
+    tiles = [tuple(tile)] if isinstance(tile[0], int) else [tuple(t) for t in tile]
+    res = SearchResult(best=None)
+    state = {"truth": None, "base_ms": None}
+    for t in tiles:
+        _search_tile(A, B, C, t, candidates, launches, out_dtype, b_layout, verbose, res, state, len(tiles) > 1)
+    return res
+
+
+def _search_tile(A, B, C, tile, candidates, launches, out_dtype, b_layout, verbose, res, state, tag_tile) -> None:
     import torch
 
     M, K = A.shape
@@ -69,11 +79,10 @@ def search(A, B, C, tile: Tuple[int, int] = (256, 256), candidates: Optional[Seq
     units = sp.gemm_units(tile[0], tile[1], T)
     cands = list(candidates) if candidates is not None else default_candidates(units)
     flops = 2.0 * M * N * K
-    res = SearchResult(best=None)
-    truth = None
-    base_ms = None
+    truth = state["truth"]
+    base_ms = state["base_ms"]
     for name, scheme, kw in cands:
-        att = Attempt(name=name, scheme=scheme, params=dict(kw))
+        att = Attempt(name=(f"{tile[0]}x{tile[1]}/" if tag_tile else "") + name, scheme=scheme, params=dict(kw))
         res.history.append(att)
         p = sp.make_params(tile_m=tile[0], tile_n=tile[1], out_dtype=out_dtype, b_layout=b_layout, **kw)
         try:
@@ -106,18 +115,18 @@ def search(A, B, C, tile: Tuple[int, int] = (256, 256), candidates: Optional[Seq
             res.best = att
         if verbose:
             print(json.dumps(asdict(att)), flush=True)
-    return res
+    state["truth"], state["base_ms"] = truth, base_ms
 
 
 def main(argv=None) -> int:
     import torch
     ap = argparse.ArgumentParser()
     ap.add_argument("--shape", default="8192x8192x8192")
-    ap.add_argument("--tile", default="256x256")
+    ap.add_argument("--tile", default="256x256,256x512", help="one or more MxN scheduler tiles, comma separated")
     ap.add_argument("--launches", type=int, default=100)
     a = ap.parse_args(argv)
     M, N, K = (int(v) for v in a.shape.split("x"))
-    tile = tuple(int(v) for v in a.tile.split("x"))
+    tile = [tuple(int(v) for v in t.split("x")) for t in a.tile.split(",")]
     g = torch.Generator(device="cuda").manual_seed(0)
     A = torch.randn((M, K), device="cuda", generator=g).bfloat16()
     B = torch.randn((K, N), device="cuda", generator=g).bfloat16()
