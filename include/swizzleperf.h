@@ -142,8 +142,11 @@ int sp_gemm_trace(const void* A, const void* B, void* C, int64_t M, int64_t N, i
 
 /* sp_gemm for callers whose matrices live in HOST memory (pinned or pageable), same layouts and dtypes:
  * copies A and B to a device staging area owned by the library (grown on demand, kept until sp_shutdown),
- * runs sp_gemm, copies C back, and synchronises `stream`; C_host is valid on return.  One call at a time per
- * device (the staging area is shared).  Adds SP_ERR_TIMEOUT to sp_gemm's errors. */
+ * runs sp_gemm, copies C back, and synchronises `stream`; C_host is valid on return.  With 4096 rows or more (and
+ * neither a caller table nor SP_FLAG_DIE_PINNED) M is split into row blocks of at least 2048 rows, each computed by its
+ * own sp_gemm under the same scheme applied to the block's tile grid, so that copies in both directions overlap the
+ * compute; the result is the same.  One call at a time per device (the staging area is shared).  Adds SP_ERR_TIMEOUT
+ * to sp_gemm's errors. */
 int sp_gemm_host(const void* A_host, const void* B_host, void* C_host, int64_t M, int64_t N, int64_t K, int scheme,
                  const sp_params* params, void* stream);
 

@@ -139,6 +139,8 @@ struct TableEntry {
   uint64_t stamp;
 };
 
+constexpr int kHostChunks = 16;  // sp_gemm_host splits M into at most this many row blocks
+
 struct DeviceState {
   int device = -1;
   int32_t* status = nullptr;
@@ -149,6 +151,8 @@ struct DeviceState {
   uint32_t die_mask[8] = {};
   void* staging = nullptr;      // device copies of A, B, C for sp_gemm_host (grow-only)
   size_t staging_bytes = 0;
+  cudaStream_t copy_in = nullptr, copy_out = nullptr;   // sp_gemm_host: copies overlap the chunked compute
+  cudaEvent_t ev[2 * kHostChunks + 3] = {};
 };
 
 static std::mutex g_mu;
@@ -437,11 +441,60 @@ int sp_gemm_host(const void* A_host, const void* B_host, void* C_host, int64_t M
     dA = (char*)ds->staging; dB = dA + pad(a_bytes); dC = dB + pad(b_bytes);
   }
   cudaStream_t st = (cudaStream_t)stream;
-  SP_CUDA(cudaMemcpyAsync(dA, A_host, a_bytes, cudaMemcpyHostToDevice, st));
-  SP_CUDA(cudaMemcpyAsync(dB, B_host, b_bytes, cudaMemcpyHostToDevice, st));
-  rc = gemm_common(dA, dB, dC, M, N, K, scheme, params, stream, nullptr, false);
-  if (rc != SP_OK) return rc;
-  SP_CUDA(cudaMemcpyAsync(C_host, dC, c_bytes, cudaMemcpyDeviceToHost, st));
+  // Row blocks of C are independent: with at least two of them the copy of the next block of A and the copy-out of the
+  // previous block of C overlap the compute of the current one (both PCIe directions busy at once).  Caller tables and
+  // die-pinned orders describe the whole grid, so they take the unsplit path.
+  int64_t rows = 2048;
+  while ((M + rows - 1) / rows > kHostChunks) rows *= 2;
+  const int n_chunks = (int)((M + rows - 1) / rows);
+  const bool split = n_chunks >= 2 && scheme != kCustom && !(params && (params->flags & SP_FLAG_DIE_PINNED));
+  if (!split) {
+    SP_CUDA(cudaMemcpyAsync(dA, A_host, a_bytes, cudaMemcpyHostToDevice, st));
+    SP_CUDA(cudaMemcpyAsync(dB, B_host, b_bytes, cudaMemcpyHostToDevice, st));
+    rc = gemm_common(dA, dB, dC, M, N, K, scheme, params, stream, nullptr, false);
+    if (rc != SP_OK) return rc;
+    SP_CUDA(cudaMemcpyAsync(C_host, dC, c_bytes, cudaMemcpyDeviceToHost, st));
+    return sp_get_status(stream, nullptr);
+  }
+  cudaStream_t cin, cout;
+  cudaEvent_t* ev;
+  {
+    std::lock_guard<std::mutex> lock(g_mu);
+    DeviceState* ds = device_state(dev);
+    if (!ds->copy_in) {
+      SP_CUDA(cudaStreamCreateWithFlags(&ds->copy_in, cudaStreamNonBlocking));
+      SP_CUDA(cudaStreamCreateWithFlags(&ds->copy_out, cudaStreamNonBlocking));
+      for (auto& e : ds->ev) SP_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+    }
+    cin = ds->copy_in; cout = ds->copy_out; ev = ds->ev;
+  }
+  cudaEvent_t ev_start = ev[2 * kHostChunks], ev_b = ev[2 * kHostChunks + 1], ev_done = ev[2 * kHostChunks + 2];
+  SP_CUDA(cudaEventRecord(ev_start, st));                 // the copies start after what is already queued on `stream`
+  SP_CUDA(cudaStreamWaitEvent(cin, ev_start, 0));
+  SP_CUDA(cudaStreamWaitEvent(cout, ev_start, 0));
+  SP_CUDA(cudaMemcpyAsync(dB, B_host, b_bytes, cudaMemcpyHostToDevice, cin));
+  SP_CUDA(cudaEventRecord(ev_b, cin));
+  for (int i = 0; i < n_chunks; ++i) {
+    const int64_t r0 = (int64_t)i * rows, nr = (M - r0 < rows) ? M - r0 : rows;
+    SP_CUDA(cudaMemcpyAsync(dA + (size_t)r0 * K * 2, (const char*)A_host + (size_t)r0 * K * 2, (size_t)nr * K * 2,
+                            cudaMemcpyHostToDevice, cin));
+    SP_CUDA(cudaEventRecord(ev[i], cin));
+  }
+  SP_CUDA(cudaStreamWaitEvent(st, ev_b, 0));
+  for (int i = 0; i < n_chunks; ++i) {
+    const int64_t r0 = (int64_t)i * rows, nr = (M - r0 < rows) ? M - r0 : rows;
+    SP_CUDA(cudaStreamWaitEvent(st, ev[i], 0));
+    rc = gemm_common(dA + (size_t)r0 * K * 2, dB, dC + (size_t)r0 * N * out_elt, nr, N, K, scheme, params, stream, nullptr, false);
+    if (rc != SP_OK) break;
+    SP_CUDA(cudaEventRecord(ev[kHostChunks + i], st));
+    SP_CUDA(cudaStreamWaitEvent(cout, ev[kHostChunks + i], 0));
+    SP_CUDA(cudaMemcpyAsync((char*)C_host + (size_t)r0 * N * out_elt, dC + (size_t)r0 * N * out_elt, (size_t)nr * N * out_elt,
+                            cudaMemcpyDeviceToHost, cout));
+  }
+  SP_CUDA(cudaEventRecord(ev_done, cout));
+  SP_CUDA(cudaStreamWaitEvent(st, ev_done, 0));
+  if (rc != SP_OK) { cudaStreamSynchronize(cin); cudaStreamSynchronize(st); return rc; }
+  SP_CUDA(cudaStreamSynchronize(cin));
   return sp_get_status(stream, nullptr);
 }
 
@@ -577,6 +630,11 @@ void sp_shutdown(void) {
     d.status = nullptr;
     if (d.staging) cudaFree(d.staging);
     d.staging = nullptr; d.staging_bytes = 0;
+    if (d.copy_in) {
+      cudaStreamDestroy(d.copy_in); cudaStreamDestroy(d.copy_out);
+      for (auto& e : d.ev) if (e) { cudaEventDestroy(e); e = nullptr; }
+      d.copy_in = d.copy_out = nullptr;
+    }
   }
   g_devs.clear();
   if (have) cudaSetDevice(prev);
