@@ -312,3 +312,20 @@ def test_gemm_host_pipelined_row_blocks_match_gemm():
     hC2 = np.full((M, N), -1, dtype=np.int16)          # pageable host memory works too
     sp.gemm_host(A.view(np.int16), B.view(np.int16), hC2, scheme, p)
     assert np.array_equal(hC2, hC.numpy())
+
+
+def test_small_host_gemm_and_shutdown_then_reuse():
+    A, B = synth.make_int_inputs(512, 640, 256, seed=17)
+    ref, _ = G.gemm_full(A, B)
+    hC = np.zeros((512, 640), dtype=np.float32)
+    p = sp.make_params(tile_m=128, tile_n=128, out_dtype=1)
+    sp.gemm_host(A.view(np.int16), B.view(np.int16), hC, sp.HILBERT, p)      # below the row-block threshold: one launch
+    assert np.array_equal(hC.astype(np.float64), ref)
+    torch.cuda.synchronize()
+    sp.shutdown()                                                             # caches, staging, streams released
+    got, _ = run_gemm(A, B, sp.HILBERT, (128, 128), "fp32")                   # and rebuilt on demand
+    assert np.array_equal(got, ref)
+    hC[:] = 0
+    sp.gemm_host(A.view(np.int16), B.view(np.int16), hC, sp.DIE_SPLIT, sp.make_params(tile_m=128, tile_n=128, out_dtype=1,
+                                                                                   inner_scheme=sp.MORTON))
+    assert np.array_equal(hC.astype(np.float64), ref)
