@@ -50,6 +50,10 @@ NCU_DRAM_BYTES = {
 def parse_scheme(spec: str):
     """'group_m:8' -> (scheme id, keyword dict for make_params)."""
     import paper_2508_20258_b200 as sp
+    if spec.endswith("+k"):    # any order + stream-K split of the tail wave
+        scheme, kw = parse_scheme(spec[:-2])
+        kw["flags"] = kw.get("flags", 0) | sp.FLAG_STREAM_K
+        return scheme, kw
     a = spec.split(":")
     name = a[0]
     if name == "row_major":

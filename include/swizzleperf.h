@@ -69,6 +69,22 @@ typedef enum {
                                  SP_ERR_UNSUPPORTED if the probe finds no usable two-way structure.  The output is the same, and every
                                  tile runs exactly once wherever the units land.  At most 64 such launches in flight per device. */
 
+#define SP_FLAG_STREAM_K 8u   /* sp_gemm / sp_gemm_trace / sp_gemm_host, tiles up to 256x256: wave quantisation.  The paper's
+                                 remap picks the tile of a slot and has no counterpart for this.  When the persistent units U
+                                 do not divide the tile count T, the last R = T mod U slots of the order are split along k:
+                                 each of their tiles goes to f = min(U / R, kblocks / 4) units, piece i taking k-blocks
+                                 [i * kblocks / f, (i + 1) * kblocks / f) (sp_streamk_plan lists the pieces); nothing is
+                                 split when f < 2.  Pieces with the same i walk k in step, so they still share operand
+                                 panels in L2.  A unit whose piece ends before the tile's last k-block writes an fp32 partial
+                                 to a library workspace; the unit with the last piece adds the partials (fixed order) and
+                                 stores the tile.  C is then the same sum taken in a different order: equal run to run for
+                                 one (shape, tile, unit count), no longer bit-identical across orders or to a launch without
+                                 the flag.  Device waits on partials are bounded like every other wait and only ever point
+                                 to lower block indices.  The workspace (about 19 MB) is allocated on first use per stream,
+                                 at most 8 streams per device; not available in sp_gemm_noalloc or with SP_FLAG_DIE_PINNED
+                                 (SP_ERR_INVALID_ARG) nor for the 256x512 tile (SP_ERR_UNSUPPORTED).  In a trace the record
+                                 of a split tile describes the piece that stored it. */
+
 typedef struct {
   uint32_t struct_size;       /* must be sizeof(sp_params)                                                  */
   int32_t group;              /* G >= 1 for SP_GROUP_M / SP_GROUP_N                                         */
@@ -85,7 +101,7 @@ typedef struct {
                               /*   the A panel); 0,0 = 256x256.  Ignored by sp_tile_map*.                    */
   int32_t out_dtype;          /* sp_gemm*: 0 = C is bf16 (round to nearest even), 1 = C is fp32             */
   int32_t b_layout;           /* sp_gemm*: 0 = B is K x N row-major, 1 = B is N x K row-major               */
-  uint32_t flags;             /* 0, or SP_FLAG_DIE_PINNED | SP_FLAG_SERPENTINE                              */
+  uint32_t flags;             /* 0, or SP_FLAG_DIE_PINNED | SP_FLAG_SERPENTINE | SP_FLAG_STREAM_K            */
 } sp_params;
 
 /* One record per tile, written by sp_gemm_trace. */
@@ -189,6 +205,17 @@ int sp_transpose(const void* in, void* out, int64_t M, int64_t N, int scheme, co
 /* Number of persistent CTAs (tile 128xN) or CTA pairs (tile 256xN) sp_gemm launches for T tiles;
  * slot s is run by unit s % units in round s / units.  Returns -1 on error. */
 int sp_gemm_units(int32_t tile_m, int32_t tile_n, int64_t T);
+
+/* The k-split of SP_FLAG_STREAM_K for T tiles of kblocks k-blocks (of 64) on `units` persistent units; host only, no
+ * GPU needed.  The paper has no counterpart (see the flag).  Writes, for every unit u in [0, units), up to
+ * SP_STREAMK_MAX_SEGMENTS segments in the order the unit walks them, as 4 int32 each at
+ * out_segments[(u * SP_STREAMK_MAX_SEGMENTS + j) * 4]: {slot, k_begin, k_end, kind} with kind 0 = whole tile,
+ * 1 = contributor (partial to the workspace), 2 = owner (adds the contributors' partials, stores); unused entries
+ * have slot = -1 (with the present policy a unit has at most one segment).  *first_slot receives the first slot of
+ * the split tail (T when nothing is split): slots below it are dealt out whole, slot s to unit s % units.
+ * Returns SP_OK or SP_ERR_INVALID_ARG. */
+#define SP_STREAMK_MAX_SEGMENTS 8
+int sp_streamk_plan(int64_t T, int32_t units, int32_t kblocks, int32_t* first_slot, int32_t* out_segments);
 
 /* Launch-order probe (the counterpart of the paper's "default scheduling policy" context):
  * launches `n_blocks` trivial blocks in clusters of `cluster` (1 or 2) and records for block b

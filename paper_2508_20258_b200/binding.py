@@ -57,7 +57,7 @@ TRACE_DTYPE = np.dtype([("slot", "<i4"), ("tile", "<i4"), ("smid", "<i4"), ("uni
                         ("mma_wait_acc", "<u4"), ("load_wait_stage", "<u4"), ("epi_wait_acc", "<u4")])
 
 EXPORTS = ["sp_tile_count", "sp_tile_map", "sp_tile_map_device", "sp_gemm", "sp_gemm_trace", "sp_gemm_host",
-           "sp_gemm_noalloc", "sp_transpose", "sp_gemm_units",
+           "sp_gemm_noalloc", "sp_transpose", "sp_gemm_units", "sp_streamk_plan",
            "sp_probe_dispatch", "sp_probe_topology", "sp_probe_l2_capacity", "sp_selftest_timeout", "sp_selftest_pinned_tickets", "sp_get_status", "sp_last_error", "sp_shutdown"]
 
 
@@ -97,6 +97,8 @@ def lib() -> ctypes.CDLL:
         L.sp_transpose.argtypes = [vp, vp, i64, i64, ctypes.c_int, pp, vp]
         L.sp_gemm_units.restype = ctypes.c_int
         L.sp_gemm_units.argtypes = [i32, i32, i64]
+        L.sp_streamk_plan.restype = ctypes.c_int
+        L.sp_streamk_plan.argtypes = [i64, i32, i32, ctypes.POINTER(ctypes.c_int32), vp]
         L.sp_probe_dispatch.restype = ctypes.c_int
         L.sp_probe_dispatch.argtypes = [i32, i32, vp, vp]
         L.sp_probe_topology.restype = ctypes.c_int
@@ -265,6 +267,22 @@ def transpose(x, out, scheme: int = ROW_MAJOR, params: Optional[SpParams] = None
 
 def gemm_units(tile_m: int, tile_n: int, T: int) -> int:
     return int(lib().sp_gemm_units(tile_m, tile_n, T))
+
+
+FLAG_DIE_PINNED, FLAG_SERPENTINE, FLAG_STREAM_K = 2, 4, 8
+STREAMK_MAX_SEGMENTS = 8
+WORK_FULL, WORK_CONTRIB, WORK_OWNER = 0, 1, 2
+
+
+def streamk_plan(T: int, units: int, kblocks: int):
+    """The k-split of SP_FLAG_STREAM_K: (first_slot, segments) with segments[u] = list of (slot, k0, k1, kind)
+    in the order unit u walks them.  Host only."""
+    first = ctypes.c_int32(0)
+    out = np.zeros((units, STREAMK_MAX_SEGMENTS, 4), dtype=np.int32)
+    _check(lib().sp_streamk_plan(T, units, kblocks, ctypes.byref(first), out.ctypes.data))
+    segs = [[tuple(int(v) for v in out[u, j]) for j in range(STREAMK_MAX_SEGMENTS) if out[u, j, 0] >= 0]
+            for u in range(units)]
+    return int(first.value), segs
 
 
 def probe_dispatch(n_blocks: int, cluster: int = 1):

@@ -7,6 +7,7 @@
 #include <vector>
 
 #include "internal.h"
+#include "streamk.cuh"
 
 namespace sp {
 
@@ -152,6 +153,10 @@ struct DeviceState {
   void* staging = nullptr;      // device copies of A, B, C for sp_gemm_host (grow-only)
   size_t staging_bytes = 0;
   cudaStream_t copy_in = nullptr, copy_out = nullptr;   // sp_gemm_host: copies overlap the chunked compute
+  // SP_FLAG_STREAM_K: one workspace (partial tiles + flags) per stream that has asked for it, so that launches on
+  // different streams never share one; launches on one stream are ordered by the stream
+  struct SkSpace { cudaStream_t stream; void* mem; int32_t epoch; };
+  std::vector<SkSpace> sk_spaces;
   cudaEvent_t ev[2 * kHostChunks + 3] = {};
 };
 
@@ -160,6 +165,7 @@ static std::vector<DeviceState> g_devs;
 static uint64_t g_stamp = 0;
 constexpr size_t kMaxTables = 64;
 
+constexpr size_t kMaxSkStreams = 8;
 constexpr int kDiePairs = 64;   // die-pinned launches that may be in flight at once on one device (different streams)
 static std::mutex g_valid_mu;
 static std::vector<Sched> g_validated;
@@ -353,6 +359,36 @@ static int gemm_common(const void* A, const void* B, void* C, int64_t M, int64_t
     call.sms_on_die[0] = ds->sms_on_die[0]; call.sms_on_die[1] = ds->sms_on_die[1];
     for (int i = 0; i < 8; ++i) call.die_mask[i] = ds->die_mask[i];
   }
+  if (params && (params->flags & SP_FLAG_STREAM_K)) {
+    if (call.pinned) {
+      set_error("SP_FLAG_STREAM_K cannot be combined with SP_FLAG_DIE_PINNED");
+      return SP_ERR_INVALID_ARG;
+    }
+    if (tile_n > 256) { set_error("SP_FLAG_STREAM_K is not implemented for the 256x512 tile"); return SP_ERR_UNSUPPORTED; }
+    DeviceState::SkSpace* space = nullptr;
+    for (auto& sk : ds->sk_spaces) if (sk.stream == call.stream) space = &sk;
+    if (!space) {
+      void* mem = nullptr;
+      if (ds->sk_spaces.size() >= kMaxSkStreams) {
+        set_error("SP_FLAG_STREAM_K is in use on %zu streams already (sp_shutdown releases them)", ds->sk_spaces.size());
+        return SP_ERR_UNSUPPORTED;
+      }
+      SP_CUDA(cudaMalloc(&mem, kSkFlagBytes + kSkWorkspaceBytes));
+      cudaError_t ce = cudaMemset(mem, 0, kSkFlagBytes);
+      if (ce != cudaSuccess) { cudaFree(mem); set_error("clearing the stream-K flags failed: %s", cudaGetErrorString(ce)); return SP_ERR_CUDA; }
+      ds->sk_spaces.push_back({call.stream, mem, 0});
+      space = &ds->sk_spaces.back();
+    }
+    if (space->epoch == INT32_MAX) {   // the flags have seen every value: start over
+      SP_CUDA(cudaStreamSynchronize(call.stream));
+      SP_CUDA(cudaMemset(space->mem, 0, kSkFlagBytes));
+      space->epoch = 0;
+    }
+    call.stream_k = 1;
+    call.sk_epoch = ++space->epoch;
+    call.sk_flags_dev = (int32_t*)space->mem;
+    call.sk_ws_dev = (float*)((char*)space->mem + kSkFlagBytes);
+  }
   return launch_gemm(call);
 }
 
@@ -399,6 +435,26 @@ int sp_tile_map_device(int64_t M, int64_t N, int32_t tileM, int32_t tileN, int s
     return SP_OK;
   }
   SP_CUDA(launch_build_perm(c, out_perm_dev, st));
+  return SP_OK;
+}
+
+int sp_streamk_plan(int64_t T, int32_t units, int32_t kblocks, int32_t* first_slot, int32_t* out_segments) {
+  if (T <= 0 || T > kMaxTiles || units <= 0 || units > 4096 || kblocks <= 0 || !first_slot || !out_segments) {
+    set_error("sp_streamk_plan: bad argument (T=%lld units=%d kblocks=%d)", (long long)T, units, kblocks);
+    return SP_ERR_INVALID_ARG;
+  }
+  const SkPlan p = sk_plan(T, units, kblocks);
+  *first_slot = p.first_slot;
+  for (int64_t i = 0; i < (int64_t)units * SP_STREAMK_MAX_SEGMENTS * 4; ++i) out_segments[i] = i % 4 == 0 ? -1 : 0;
+  for (int u = 0; u < units; ++u) {
+    const int n = sk_segments(p, u, kblocks);
+    if (n > SP_STREAMK_MAX_SEGMENTS) { set_error("unit %d has %d segments", u, n); return SP_ERR_UNSUPPORTED; }
+    for (int j = 0; j < n; ++j) {
+      const Work w = sk_segment(p, u, j, kblocks);
+      int32_t* o = out_segments + ((size_t)u * SP_STREAMK_MAX_SEGMENTS + j) * 4;
+      o[0] = w.slot; o[1] = w.k0; o[2] = w.k1; o[3] = w.kind;
+    }
+  }
   return SP_OK;
 }
 
@@ -630,6 +686,8 @@ void sp_shutdown(void) {
     d.status = nullptr;
     if (d.staging) cudaFree(d.staging);
     d.staging = nullptr; d.staging_bytes = 0;
+    for (auto& sk : d.sk_spaces) cudaFree(sk.mem);
+    d.sk_spaces.clear();
     if (d.copy_in) {
       cudaStreamDestroy(d.copy_in); cudaStreamDestroy(d.copy_out);
       for (auto& e : d.ev) if (e) { cudaEventDestroy(e); e = nullptr; }

@@ -62,6 +62,10 @@ extern "C" int sp_gemm_noalloc(const void* A, const void* B, void* C, int64_t M,
   int rc = validate_gemm_args(A, B, C, M, N, K, params, &tile_m, &tile_n, &out_f32, &b_nk);
   if (rc != SP_OK) return rc;
 
+  if (params && (params->flags & SP_FLAG_STREAM_K)) {
+    set_error("SP_FLAG_STREAM_K needs a workspace and is not available in sp_gemm_noalloc");
+    return SP_ERR_INVALID_ARG;
+  }
   GemmCall call;
   memset(&call, 0, sizeof call);
   rc = resolve_sched(M, N, tile_m, tile_n, scheme, params, &call.sched);

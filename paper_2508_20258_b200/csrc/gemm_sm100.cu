@@ -29,6 +29,7 @@
 
 #include "internal.h"
 #include "ptx.cuh"
+#include "streamk.cuh"
 
 namespace sp {
 
@@ -71,6 +72,11 @@ struct GemmArgs {
   int units_on_die[2];             // persistent units per die (all SMs host one CTA each)
   int32_t* die_count;              // two device counters, zero at launch: arrival rank of a unit on its die
   uint32_t die_mask[8];            // bit smid = die of that SM (from the topology probe)
+  // Stream-K tail (SP_FLAG_STREAM_K): the last sk.tiles slots are split along k over sk.units units.
+  SkPlan sk;
+  float* sk_ws;                    // one fp32 partial tile per unit: [unit][cta of the unit][lane quarter][column][lane]
+  int32_t* sk_flags;               // one word per (unit, cta, lane quarter): set to sk_epoch once that partial is complete
+  int32_t sk_epoch;                // differs from launch to launch on one workspace, so the flags need no clearing
   Sched sched;
 };
 
@@ -159,14 +165,20 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   tcgen05_fence_after();
   const uint32_t tmem_base = *tmem_slot_ptr;
 
-  // slots of this unit: s_first, s_first + s_step, ... below s_end
-  int s_first = unit, s_step = args.units, s_end = T;
+  // whole tiles of this unit: slots s_first, s_first + s_step, ... below s_end; then its segments of the stream-K tail
+  int s_first = unit, s_step = args.units, s_end = args.sk.first_slot;
   if (args.pinned) {
     const uint32_t die = tmem_slot_ptr[2], r = tmem_slot_ptr[3];
     s_step = args.units_on_die[die];
     s_first = (die ? args.half0 : 0) + (int)r;
     s_end = die ? T : args.half0;
   }
+  const int n_whole = s_first < s_end ? (s_end - s_first + s_step - 1) / s_step : 0;
+  const int n_items = n_whole + sk_segments(args.sk, unit, KB);
+  auto work_at = [&](int i) -> Work {
+    if (i < n_whole) { Work w; w.slot = s_first + i * s_step; w.k0 = 0; w.k1 = KB; w.kind = kWorkFull; return w; }
+    return sk_segment(args.sk, unit, i - n_whole, KB);
+  };
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer
@@ -176,12 +188,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int s = s_first; s < s_end && ok; s += s_step) {
+      for (int item = 0; item < n_items && ok; ++item) {
+        const Work wk = work_at(item);
+        const int s = wk.slot;
         const int t = tile_of_slot(args, s);
         const int tm = t / Tn, tn = t - tm * Tn;
         const int row0 = tm * TILE_M + (int)rank * 128;
         const int col0 = tn * BN + (int)rank * C::kMmaCols;        // + c * kMmaN for the c-th MMA tile
-        const bool tracing = args.trace != nullptr && rank == 0;
+        const bool tracing = args.trace != nullptr && rank == 0 && wk.kind != kWorkContrib;   // a split tile is traced by the piece that stores it
         uint32_t waited = 0;
         if (tracing && lane == 0) {
           sp_trace_rec* rec = args.trace + s;
@@ -189,7 +203,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
           rec->slot = s; rec->tile = t; rec->smid = (int)smid; rec->unit = unit; rec->t_begin = globaltimer();
         }
-        for (int kb = 0; kb < KB; ++kb) {
+        for (int kb = wk.k0; kb < wk.k1; ++kb) {
           ok = mbar_wait_timed(bar_empty + 8 * stage, phase ^ 1u, args.status, (kRoleProducer << 8) | 1, tracing, &waited);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
@@ -243,10 +257,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       // Two MMA tiles (BN = 512): two parts, each with its own pair of barriers, so the epilogue can drain the
       // first while the second is still being computed, and the next tile can start on the first part while the
       // second is being drained.
-      for (int s = s_first; s < s_end && ok; s += s_step, ++it) {
+      for (; it < n_items && ok; ++it) {
+        const Work wk = work_at(it);
+        const int s = wk.slot;
         const int buf = it % C::kBufs;
         const uint32_t use = C::kNT == 1 ? ((uint32_t)(it / C::kBufs) & 1u) : ((uint32_t)it & 1u);
-        const bool tracing = args.trace != nullptr;
+        const bool tracing = args.trace != nullptr && wk.kind != kWorkContrib;
         uint32_t wait_acc = 0, wait_data = 0;
         if (tracing && lane == 0) args.trace[s].t_mma_begin = globaltimer();
         if constexpr (C::kNT == 2) {
@@ -299,7 +315,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             kb += g;
           }
         } else {
-        for (int kb = 0; kb < KB && ok; ++kb) {
+        for (int kb = wk.k0; kb < wk.k1 && ok; ++kb) {        // all k-blocks of the tile, or this unit's segment of them
           ok = mbar_wait_timed(bar_full + 8 * stage, phase, args.status, (kRoleMma << 8) | 2, tracing, &wait_data);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
@@ -309,7 +325,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
           for (int c = 0; c < C::kNT; ++c) {
             const int part = C::kNT == 1 ? buf : c;
-            if (kb == 0) {                       // the part must have been drained by the epilogue of its previous use
+            if (kb == wk.k0) {                   // the part must have been drained by the epilogue of its previous use
               ok = mbar_wait_timed(bar_tempty + 8 * part, use ^ 1u, args.status, (kRoleMma << 8) | 1, tracing, &wait_acc);
               ok = __all_sync(0xffffffffu, ok);
               if (!ok) break;
@@ -321,9 +337,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               for (int k = 0; k < kBK / kUmmaK; ++k) {
                 const uint64_t da = smem_desc(sa + k * (kUmmaK * 2), 16, 1024);
                 const uint64_t db = smem_desc(sb + c * (C::kMmaCols * kBK * 2) + k * args.b_kstep, args.b_lbo, args.b_sbo);
-                umma_bf16<CG>(d_tmem, da, db, idesc, (uint32_t)((kb | k) != 0));
+                umma_bf16<CG>(d_tmem, da, db, idesc, (uint32_t)(kb > wk.k0 || k != 0));
               }
-              if (kb == KB - 1) umma_commit<CG>(bar_tfull + 8 * part);   // this part is complete
+              if (kb == wk.k1 - 1) umma_commit<CG>(bar_tfull + 8 * part);   // this part is complete
             }
             __syncwarp();
           }
@@ -355,7 +371,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c * C::kMmaN);
       int it2 = 0;
       bool ok2 = true;
-      for (int s = s_first; s < s_end && ok2; s += s_step, ++it2) {
+      for (; it2 < n_items && ok2; ++it2) {
+        const int s = work_at(it2).slot;
         const int t = tile_of_slot(args, s);
         const int tm = t / Tn, tn = t - tm * Tn;
         const uint32_t use = (uint32_t)it2 & 1u;
@@ -430,7 +447,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     int it = 0;
     int chunk = 0;                 // staging buffers alternate per stored chunk, across tiles
     bool ok = true;
-    for (int s = s_first; s < s_end && ok; s += s_step, ++it) {
+    for (; it < n_items && ok; ++it) {
+      const Work wk = work_at(it);
+      const int s = wk.slot;
       const int t = tile_of_slot(args, s);
       const int tm = t / Tn, tn = t - tm * Tn;
       const int buf = it % C::kBufs;
@@ -442,12 +461,60 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll 1
       for (int c = 0; c < C::kNT && ok; ++c) {                         // accumulator parts, in the order they complete
         const int part = C::kNT == 1 ? buf : c;
+        // stream-K workspace of (unit u, this CTA, this lane quarter), in 16-byte units: [column / 4][lane]; one warp
+        // instruction writes (and later reads) 512 contiguous bytes
+        auto ws_of = [&](int u) -> float4* {
+          return reinterpret_cast<float4*>(args.sk_ws) + ((((size_t)u * CG + rank) * 4 + (size_t)quarter) * (BN / 4)) * 32 + lane;
+        };
+        constexpr int kPf = kChunkCols / 4;     // 16-byte units of one chunk of this thread's row
+        float4 pf[kPf];                         // owner segments: the nearest contributor's chunk, fetched one chunk ahead
+        int n_src = 0;                          // partials to add: those of units unit-1 ... unit-n_src
+        if (wk.kind == kWorkOwner) {
+          // the contributors finished these pieces at the start of their tails, long before this unit's own MMAs end:
+          // the flags are checked and the first chunk is fetched while the accumulator is still being computed
+          n_src = sk_contributors(args.sk, unit, s, KB);
+          for (int i = 1; i <= n_src && ok; ++i) {
+            bool okf = true;
+            if (lane == 0)
+              okf = flag_wait(args.sk_flags + ((unit - i) * CG + (int)rank) * 4 + quarter, args.sk_epoch, args.status, (kRoleEpilogue << 8) | 3);
+            ok = __all_sync(0xffffffffu, okf);
+          }
+          if (!ok) break;
+          __syncwarp();
+          __threadfence();
+          const float4* src = ws_of(unit - 1);
+#pragma unroll
+          for (int j = 0; j < kPf; ++j) pf[j] = __ldcg(src + j * 32);
+        }
         ok = mbar_wait_timed(bar_tfull + 8 * part, use, args.status, (kRoleEpilogue << 8) | 1, args.trace != nullptr, &wait_epi);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tcgen05_fence_after();
         const int col_base = tn * BN + c * kPartCols;
         const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(C::kNT == 1 ? buf * BN : c * C::kMmaN);
+        if (wk.kind == kWorkContrib) {
+          // a segment that does not finish its tile: the raw fp32 partial goes to the workspace, then the flag goes up
+          float4* dst = ws_of(unit);
+#pragma unroll 1
+          for (int q = 0; q < kPartCols / 32; ++q) {
+            uint32_t v[32];
+            tmem_ld_32x32b_x32(taddr + (uint32_t)(q * 32), v);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              __stcg(dst + (size_t)(q * 8 + j) * 32, make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                                                 __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3])));
+          }
+          tcgen05_fence_before();
+          __threadfence();
+          __syncwarp();
+          if (lane == 0) {
+            const uint32_t te = bar_tempty + 8 * part;
+            mbar_arrive_cluster(CG == 1 ? te : mapa(te, 0));
+            st_release_gpu(args.sk_flags + (unit * CG + (int)rank) * 4 + quarter, args.sk_epoch);
+          }
+          continue;
+        }
         {
 #pragma unroll 1
         for (int q = 0; q < kPartCols / kChunkCols; ++q, ++chunk) {
@@ -455,6 +522,27 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           tmem_ld_32x32b_x32(taddr + (uint32_t)(q * kChunkCols), v);
           if constexpr (!OUT_F32) tmem_ld_32x32b_x32(taddr + (uint32_t)(q * kChunkCols + 32), w);
           tmem_ld_wait();
+          if (n_src > 0) {
+            // fixed order of the sum: own accumulator, then units unit-1, unit-2, ...
+            auto add16 = [&](int j, const float4& a) {
+              uint32_t* d = (OUT_F32 || j < 8) ? &v[4 * j] : &w[4 * (j - 8)];
+              d[0] = __float_as_uint(__uint_as_float(d[0]) + a.x); d[1] = __float_as_uint(__uint_as_float(d[1]) + a.y);
+              d[2] = __float_as_uint(__uint_as_float(d[2]) + a.z); d[3] = __float_as_uint(__uint_as_float(d[3]) + a.w);
+            };
+#pragma unroll
+            for (int j = 0; j < kPf; ++j) add16(j, pf[j]);
+#pragma unroll 1
+            for (int i = 2; i <= n_src; ++i) {
+              const float4* src = ws_of(unit - i) + (size_t)(q * kPf) * 32;
+#pragma unroll
+              for (int j = 0; j < kPf; ++j) add16(j, __ldcg(src + j * 32));
+            }
+            if (q + 1 < kPartCols / kChunkCols) {        // next chunk's fetch overlaps this chunk's staging and store
+              const float4* src = ws_of(unit - 1) + (size_t)((q + 1) * kPf) * 32;
+#pragma unroll
+              for (int j = 0; j < kPf; ++j) pf[j] = __ldcg(src + j * 32);
+            }
+          }
           // the buffer used two chunks ago must have been read by its store before it is overwritten
           if (chunk >= 2) {
             if (lane == 0) bulk_wait_read_1();
@@ -710,6 +798,25 @@ int launch_gemm(const GemmCall& call) {
     if (ce != cudaSuccess) { set_error("clearing the die counters failed: %s", cudaGetErrorString(ce)); return SP_ERR_CUDA; }
   }
   args.sched = call.sched;
+  args.sk = SkPlan{0, args.units, call.sched.T};   // no tail: every slot is a whole tile
+  args.sk_ws = nullptr; args.sk_flags = nullptr; args.sk_epoch = 0;
+  if (call.stream_k) {
+    // units are not capped by the tile count here: a problem smaller than a wave is spread over all of them
+    const int all_units = gemm_units(call.tile_m, call.tile_n, kMaxTiles);
+    const SkPlan plan = all_units > 0 ? sk_plan(call.sched.T, all_units, args.kblocks) : args.sk;
+    if (plan.tiles > 0) {
+      if ((size_t)all_units * call.tile_m * call.tile_n * sizeof(float) > kSkWorkspaceBytes ||
+          (size_t)all_units * cg * 4 * sizeof(int32_t) > kSkFlagBytes) {
+        set_error("stream-K workspace too small for %d units of %dx%d", all_units, call.tile_m, call.tile_n);
+        return SP_ERR_UNSUPPORTED;
+      }
+      args.units = all_units;
+      args.sk = plan;
+      args.sk_ws = call.sk_ws_dev;
+      args.sk_flags = call.sk_flags_dev;
+      args.sk_epoch = call.sk_epoch;
+    }
+  }
 
   if (cg == 1) return call.tile_n == 128 ? launch_shape<1, 128>(call, tmA, tmB, tmC, args) : launch_shape<1, 256>(call, tmA, tmB, tmC, args);
   if (call.tile_n == 512) return launch_shape<2, 512>(call, tmA, tmB, tmC, args);

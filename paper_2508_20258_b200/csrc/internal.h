@@ -15,6 +15,11 @@ namespace sp {
 constexpr int64_t kMaxTiles = 1 << 24;
 constexpr int kMaxCurveSide = 4096;
 
+// Stream-K workspace of one stream: a flag per (unit, CTA, lane quarter) and one fp32 partial tile per unit.
+// 148 CTAs x 128 rows x 256 columns covers every tile shape up to 256x256 on every unit count.
+constexpr size_t kSkFlagBytes = 4096;
+constexpr size_t kSkWorkspaceBytes = (size_t)148 * 128 * 256 * 4;
+
 void set_error(const char* fmt, ...);
 
 // Validates sizes and parameters and fills `out`.  Returns an sp_status.
@@ -49,6 +54,10 @@ struct GemmCall {
   int sms_on_die[2];
   uint32_t die_mask[8];
   sp_trace_rec* trace_dev;  // nullptr unless tracing
+  int stream_k;             // SP_FLAG_STREAM_K: split the tail wave along k
+  int32_t* sk_flags_dev;    // kSkFlagBytes of flags, zero when allocated
+  int32_t sk_epoch;         // value the flags take in this launch: 1, 2, ... per workspace
+  float* sk_ws_dev;         // kSkWorkspaceBytes of partial tiles
   cudaStream_t stream;
 };
 

@@ -80,6 +80,34 @@ static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity
   }
 }
 
+__device__ __forceinline__ void st_release_gpu(int32_t* p, int32_t v) {
+  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+__device__ __forceinline__ int32_t ld_acquire_gpu(const int32_t* p) {
+  int32_t v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
+// Bounded wait for a word in global memory to take the value `want` (written by another CTA with st_release_gpu).
+static __device__ __noinline__ bool flag_wait(const int32_t* flag, int32_t want, int32_t* status, int code,
+                                              unsigned long long timeout_ns = kTimeoutNs) {
+  if (ld_acquire_gpu(flag) == want) return true;
+  const unsigned long long t0 = globaltimer();
+  for (uint32_t i = 1;; ++i) {
+    if (ld_acquire_gpu(flag) == want) return true;
+    __nanosleep(64);
+    if ((i & 63u) == 0) {
+      if (*(volatile int32_t*)status != 0) return false;
+      if (globaltimer() - t0 > timeout_ns) {
+        atomicCAS(status, 0, code);
+        return false;
+      }
+    }
+  }
+}
+
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t* status, int code) {
   if (mbar_try_wait(bar, parity)) return true;
   return mbar_wait_slow(bar, parity, status, code);
