@@ -103,8 +103,9 @@ DEFAULT_SCHEME = {"cfg1": "group_m:2", "cfg2": "group_m:8", "cfg3": "die_split:m
 FALLBACK_SCHEME = {"cfg3": "group_m:8", "cfg5": "group_m:16"}   # if the topology probe finds no two-way L2 structure
 # 8192^3 is timed with two 256x256 2-CTA MMA tiles per scheduler tile (they share the A panel: a quarter less operand
 # traffic from L2); the plain 256x256 scheduler tile is timed beside it and reported in the same line.
-DEFAULT_TILE = {"cfg3": "256x512"}
-DEFAULT_SCHEME_BY_TILE = {("cfg3", "256x512"): "group_n:8", ("cfg5", "256x512"): "die_split:m:group_m:8:p"}
+DEFAULT_TILE = {"cfg3": "256x512", "cfg2": "256x512"}   # 4096^3: A and B fit in L2, the order hardly matters, the wider tile does
+DEFAULT_SCHEME_BY_TILE = {("cfg3", "256x512"): "group_n:8", ("cfg5", "256x512"): "die_split:m:group_m:8:p",
+                          ("cfg2", "256x512"): "row_major"}
 
 
 def dist_env():
