@@ -524,6 +524,68 @@ def run_transpose(args) -> int:
     return 0
 
 
+STENCIL_SWEEP = ["row_major", "col_major", "group_m:2", "group_m:4", "group_m:8", "group_n:2", "group_n:4", "group_n:8",
+                 "morton", "hilbert", "xcd:2", "xcd:8", "die_split:m:row_major", "die_split:m:row_major:i",
+                 "die_split:m:group_m:4"]
+
+
+def run_stencil(args) -> int:
+    """Third workload (the paper's Stencil 2D): one five-point sweep over an fp32 grid under each tile order.  HBM
+    bound: algorithmic bytes = 2 * M * N * 4 (every point read once, written once; halos come from L2)."""
+    import torch
+    import paper_2508_20258_b200 as sp
+    M, N = (int(v) for v in args.stencil.split("x"))
+    torch.cuda.set_device(0)
+    g = torch.Generator(device="cuda").manual_seed(11)
+    x = torch.randn((M, N), device="cuda", generator=g, dtype=torch.float32)
+    out = torch.empty_like(x)
+    stream = torch.cuda.current_stream()
+    peaks = benchutil.measured_peaks(ROOT)
+    nbytes = 2.0 * M * N * 4
+    specs = args.scheme.split(",") if args.scheme else STENCIL_SWEEP
+
+    def timed(spec, n):
+        scheme, kw = parse_scheme(spec)
+        p = sp.make_params(**kw)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(n):
+            sp.stencil2d(x, out, 0.5, 0.125, scheme, p, stream)
+        e1.record(stream)
+        e1.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    if args.profile_sweep:
+        for spec in specs:
+            timed(spec, 1)
+        assert sp.get_status() == 0
+        print(json.dumps({"profile_sweep": "stencil2d", "shape": [M, N], "launch_order": specs}), flush=True)
+        return 0
+    for spec in specs:
+        timed(spec, 3)
+        one = timed(spec, 5)
+        n = int(max(10, min(1000, 200.0 / one)))
+        ms = min(timed(spec, n) for _ in range(2))
+        gbs = nbytes / ms / 1e6
+        print(json.dumps({"stencil2d": [M, N], "scheme": spec, "ms": ms, "GB/s": gbs,
+                          "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                       "frac": gbs / peaks["hbm_gbs"], "peak_kind": f"copy bandwidth, {peaks['source']}"}}),
+              flush=True)
+    assert sp.get_status() == 0
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for _ in range(3):
+        out.copy_(x)
+    e0.record(stream)
+    for _ in range(20):
+        out.copy_(x)
+    e1.record(stream)
+    e1.synchronize()
+    ms = e0.elapsed_time(e1) / 20
+    print(json.dumps({"stencil2d": [M, N], "scheme": "torch copy_ of the grid (context only)", "ms": ms,
+                      "GB/s": nbytes / ms / 1e6}), flush=True)
+    return 0
+
+
 def main() -> int:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -542,9 +604,12 @@ def main() -> int:
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--transpose", default=None, metavar="MxN", help="time sp_transpose on an M x N 16-bit matrix instead")
+    ap.add_argument("--stencil", default=None, metavar="MxN", help="time sp_stencil2d on an M x N fp32 grid instead")
     args = ap.parse_args()
     if args.transpose:
         return run_transpose(args)
+    if args.stencil:
+        return run_stencil(args)
     if args.impl == "reference":
         return run_reference(args)
     return run_ours(args)

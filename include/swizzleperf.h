@@ -202,6 +202,26 @@ int sp_gemm_noalloc(const void* A, const void* B, void* C, int64_t M, int64_t N,
 #define SP_TRANSPOSE_TILE 64
 int sp_transpose(const void* in, void* out, int64_t M, int64_t N, int scheme, const sp_params* params, void* stream);
 
+/* One sweep of the five-point stencil over an fp32 grid, under a tile order (paper: "Stencil 2D", one of its science
+ * kernels, whose block grid is re-ordered so that blocks sharing halo data meet in one L2; the paper does not print
+ * the stencil: the five-point star with the rim carried over is this library's reading):
+ *   out[i][j] = c_center * in[i][j] + c_neighbor * (in[i-1][j] + in[i+1][j] + in[i][j-1] + in[i][j+1])
+ *                                                            for 0 < i < M-1 and 0 < j < N-1,
+ *   out[i][j] = in[i][j]                                     on the rim (also the whole grid when M < 3 or N < 3).
+ * Arithmetic in fp32: the four neighbours are added in pairs, (north + south) + (west + east), then one fused
+ * multiply-add onto c_center * in[i][j].  The grid is cut into SP_STENCIL_TILE_M x SP_STENCIL_TILE_N tiles;
+ * `scheme` / `params` order that tile grid exactly as for sp_tile_map(M, N, 64, 128, ...); persistent CTAs take
+ * slots with a fixed stride.
+ *   in  : DEVICE, M x N row-major fp32, read-only.
+ *   out : DEVICE, M x N row-major fp32, fully overwritten; must not overlap `in`.
+ * Errors: SP_ERR_INVALID_ARG (NULL, sizes, in == out, NaN coefficient), SP_ERR_ALIGNMENT (pointers not 16-byte
+ * aligned, N not a multiple of 4), SP_ERR_NOT_BIJECTIVE, SP_ERR_UNSUPPORTED, SP_ERR_DEVICE, SP_ERR_CUDA.
+ * Asynchronous on `stream`. */
+#define SP_STENCIL_TILE_M 64
+#define SP_STENCIL_TILE_N 128
+int sp_stencil2d(const void* in, void* out, int64_t M, int64_t N, float c_center, float c_neighbor, int scheme,
+                 const sp_params* params, void* stream);
+
 /* Number of persistent CTAs (tile 128xN) or CTA pairs (tile 256xN) sp_gemm launches for T tiles;
  * slot s is run by unit s % units in round s / units.  Returns -1 on error. */
 int sp_gemm_units(int32_t tile_m, int32_t tile_n, int64_t T);

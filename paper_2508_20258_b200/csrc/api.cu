@@ -585,6 +585,39 @@ int sp_transpose(const void* in, void* out, int64_t M, int64_t N, int scheme, co
   return launch_transpose(in, out, M, N, sched, perm_dev, ds->status, (cudaStream_t)stream);
 }
 
+int sp_stencil2d(const void* in, void* out, int64_t M, int64_t N, float c_center, float c_neighbor, int scheme,
+                 const sp_params* params, void* stream) {
+  if (!in || !out) { set_error("in and out must not be NULL"); return SP_ERR_INVALID_ARG; }
+  if (M <= 0 || N <= 0) { set_error("M and N must be positive"); return SP_ERR_INVALID_ARG; }
+  if (M >= (1ll << 31) - 256 || N >= (1ll << 31) - 256) { set_error("dimension too large"); return SP_ERR_UNSUPPORTED; }
+  if (((uintptr_t)in | (uintptr_t)out) & 15u) { set_error("in and out must be 16-byte aligned"); return SP_ERR_ALIGNMENT; }
+  if ((N % 4) != 0) { set_error("N must be a multiple of 4 (16-byte row pitch)"); return SP_ERR_ALIGNMENT; }
+  if (in == out) { set_error("the sweep is not in place: out must not overlap in"); return SP_ERR_INVALID_ARG; }
+  if (!(c_center == c_center) || !(c_neighbor == c_neighbor)) { set_error("coefficients must not be NaN"); return SP_ERR_INVALID_ARG; }
+  Sched sched;
+  int rc = resolve_sched(M, N, SP_STENCIL_TILE_M, SP_STENCIL_TILE_N, scheme, params, &sched);
+  if (rc != SP_OK) return rc;
+  std::vector<int32_t> host_perm;
+  if (scheme == kCustom || !already_validated(sched)) {
+    rc = build_perm_host(sched, params ? params->custom_perm : nullptr, host_perm);
+    if (rc != SP_OK) return rc;
+    if (scheme != kCustom) remember_validated(sched);
+  }
+  int dev = 0;
+  rc = current_device(&dev);
+  if (rc != SP_OK) return rc;
+  std::lock_guard<std::mutex> lock(g_mu);
+  DeviceState* ds = device_state(dev);
+  rc = get_status_word(ds);
+  if (rc != SP_OK) return rc;
+  const int32_t* perm_dev = nullptr;
+  if (sched.use_table) {
+    rc = get_table(ds, sched, host_perm, scheme == kCustom, (cudaStream_t)stream, &perm_dev);
+    if (rc != SP_OK) return rc;
+  }
+  return launch_stencil(in, out, M, N, c_center, c_neighbor, sched, perm_dev, ds->status, (cudaStream_t)stream);
+}
+
 int sp_gemm_units(int32_t tile_m, int32_t tile_n, int64_t T) {
   int dev = 0;
   if (current_device(&dev) != SP_OK) return -1;

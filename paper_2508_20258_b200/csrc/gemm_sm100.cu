@@ -663,6 +663,22 @@ int make_map(CUtensorMap* m, const void* base, int64_t rows, int64_t cols, int b
   return SP_OK;
 }
 
+// Row-major [rows, cols] fp32 matrix, box = box_rows x box_cols elements, no shared-memory swizzle; parts of a box
+// outside the matrix read as zero.
+int make_map_plain(CUtensorMap* m, const void* base, int64_t rows, int64_t cols, int box_rows, int box_cols) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) { set_error("cuTensorMapEncodeTiled is not available from the driver"); return SP_ERR_CUDA; }
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 4};
+  cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled failed (CUresult %d)", (int)r); return SP_ERR_CUDA; }
+  return SP_OK;
+}
+
 // Co-resident persistent units for one tile shape: one CTA per SM, or as many CTA pairs as the
 // device can hold at once (asked of the occupancy calculator, cached per shape).
 template <int CG, int BN>

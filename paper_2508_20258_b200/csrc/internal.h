@@ -69,6 +69,9 @@ int launch_gemm(const GemmCall& call);
 // Tensor map of a row-major [rows, cols] matrix of 2-byte (or, with f32, 4-byte) elements with boxes of
 // box_rows x 128 bytes and the 128-byte shared-memory swizzle.  `m` is a CUtensorMap.
 int make_map(struct CUtensorMap_st* m, const void* base, int64_t rows, int64_t cols, int box_rows, bool f32);
+int make_map_plain(struct CUtensorMap_st* m, const void* base, int64_t rows, int64_t cols, int box_rows, int box_cols);
+int launch_stencil(const void* in, void* out, int64_t M, int64_t N, float c_center, float c_neighbor, const Sched& sched,
+                   const int32_t* perm_dev, int32_t* status_dev, cudaStream_t stream);
 int launch_transpose(const void* in, void* out, int64_t M, int64_t N, const Sched& sched, const int32_t* perm_dev,
                      int32_t* status_dev, cudaStream_t stream);
 int selftest_timeout(int32_t* status_dev, int timeout_us, int32_t* code_host, int64_t* waited_us_host);
