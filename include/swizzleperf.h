@@ -85,6 +85,17 @@ typedef enum {
                                  (SP_ERR_INVALID_ARG) nor for the 256x512 tile (SP_ERR_UNSUPPORTED).  In a trace the record
                                  of a split tile describes the piece that stored it. */
 
+#define SP_FLAG_OVERLAP 16u   /* sp_gemm only.  The caller states that this launch is independent of the kernel before it on the
+                                 stream: it reads nothing that kernel writes, and it may start writing C while that kernel is
+                                 still running.  The launch is then made with programmatic stream serialisation and never
+                                 waits for its predecessor; every GEMM launch of this library signals at its start that its
+                                 successor may be scheduled.  CTAs of the next GEMM then take over SMs as the CTAs of the
+                                 previous one finish, which fills the partly empty last wave of back-to-back independent
+                                 GEMMs.  The paper has no counterpart.  A launch that first has to build its tile table (first
+                                 use of a non-arithmetic order) is made without the overlap.  Not with SP_FLAG_DIE_PINNED,
+                                 SP_FLAG_STREAM_K or tracing (SP_ERR_INVALID_ARG).  It still completes after its predecessor, so the
+                                 stream order seen by everything else (copies, events, other kernels) is unchanged. */
+
 typedef struct {
   uint32_t struct_size;       /* must be sizeof(sp_params)                                                  */
   int32_t group;              /* G >= 1 for SP_GROUP_M / SP_GROUP_N                                         */
@@ -101,7 +112,7 @@ typedef struct {
                               /*   the A panel); 0,0 = 256x256.  Ignored by sp_tile_map*.                    */
   int32_t out_dtype;          /* sp_gemm*: 0 = C is bf16 (round to nearest even), 1 = C is fp32             */
   int32_t b_layout;           /* sp_gemm*: 0 = B is K x N row-major, 1 = B is N x K row-major               */
-  uint32_t flags;             /* 0, or SP_FLAG_DIE_PINNED | SP_FLAG_SERPENTINE | SP_FLAG_STREAM_K            */
+  uint32_t flags;             /* 0, or any of SP_FLAG_DIE_PINNED, _SERPENTINE, _STREAM_K, _OVERLAP            */
 } sp_params;
 
 /* One record per tile, written by sp_gemm_trace. */

@@ -257,7 +257,8 @@ static int get_die_map(DeviceState* ds) {
 
 // Device table for a table scheme; built by the device builder (or copied for SP_CUSTOM).
 static int get_table(DeviceState* ds, const Sched& c, const std::vector<int32_t>& host_perm, bool is_custom,
-                     cudaStream_t stream, const int32_t** out) {
+                     cudaStream_t stream, const int32_t** out, bool* built_now = nullptr) {
+  if (built_now) *built_now = false;
   const uint64_t h = is_custom ? fnv(host_perm.data(), c.T) : 0;
   for (auto& e : ds->tables)
     if (memcmp(&e.key, &c, sizeof c) == 0 && e.custom_hash == h) { e.stamp = ++g_stamp; *out = e.dev; return SP_OK; }
@@ -278,6 +279,7 @@ static int get_table(DeviceState* ds, const Sched& c, const std::vector<int32_t>
   } else {
     cudaError_t ce = launch_build_perm(c, e.dev, stream);
     if (ce != cudaSuccess) { cudaFree(e.dev); set_error("table build failed: %s", cudaGetErrorString(ce)); return SP_ERR_CUDA; }
+    if (built_now) *built_now = true;   // a kernel on `stream` is writing the table: the GEMM must be ordered after it
   }
   ds->tables.push_back(e);
   *out = e.dev;
@@ -342,9 +344,17 @@ static int gemm_common(const void* A, const void* B, void* C, int64_t M, int64_t
   call.trace_dev = want_trace ? trace : nullptr;
   call.stream = (cudaStream_t)stream;
   call.perm_dev = nullptr;
+  bool table_built_now = false;
   if (call.sched.use_table) {
-    rc = get_table(ds, call.sched, host_perm, scheme == kCustom, call.stream, &call.perm_dev);
+    rc = get_table(ds, call.sched, host_perm, scheme == kCustom, call.stream, &call.perm_dev, &table_built_now);
     if (rc != SP_OK) return rc;
+  }
+  if (params && (params->flags & SP_FLAG_OVERLAP)) {
+    if (want_trace || (params->flags & (SP_FLAG_DIE_PINNED | SP_FLAG_STREAM_K))) {
+      set_error("SP_FLAG_OVERLAP cannot be combined with tracing, SP_FLAG_DIE_PINNED or SP_FLAG_STREAM_K");
+      return SP_ERR_INVALID_ARG;
+    }
+    call.overlap = table_built_now ? 0 : 1;
   }
   if (params && (params->flags & SP_FLAG_DIE_PINNED)) {
     if (scheme != kDieSplit || call.sched.interleave) {

@@ -77,6 +77,7 @@ struct GemmArgs {
   float* sk_ws;                    // one fp32 partial tile per unit: [unit][cta of the unit][lane quarter][column][lane]
   int32_t* sk_flags;               // one word per (unit, cta, lane quarter): set to sk_epoch once that partial is complete
   int32_t sk_epoch;                // differs from launch to launch on one workspace, so the flags need no clearing
+  int overlap;                     // launched with programmatic stream serialisation (never waits for its predecessor)
   Sched sched;
 };
 
@@ -133,6 +134,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   const int T = args.sched.T, Tn = args.sched.Tn;
   const int KB = args.kblocks;
 
+  // A GEMM launched behind this one with SP_FLAG_OVERLAP may be scheduled from now on: its CTAs become resident as
+  // ours exit (shared memory admits one CTA per SM).  Without such a successor this is a no-op.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (threadIdx.x == 0) {
     for (int i = 0; i < S; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_empty + 8 * i, 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(bar_tfull + 8 * i, 1); mbar_init(bar_tempty + 8 * i, 4 * CG); }
@@ -594,6 +598,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   tcgen05_fence_before();
   unit_sync<CG>();
   if (warp == 1) tmem_dealloc<CG>(tmem_base, kTmemCols);
+  // An overlapped launch never waited for its predecessor; it must still not COMPLETE before it, or whatever follows
+  // on the stream (a copy of the predecessor's C, an event) could run too early.  One thread holds the CTA's exit
+  // until the predecessor grid has completed and its writes are visible; by now that is almost always the case.
+  if (args.overlap && threadIdx.x == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 // Self-test of the bounded wait: a barrier nobody arrives on.  The wait must give up after
@@ -738,13 +746,15 @@ static int launch_variant(const GemmCall& call, const CUtensorMap& tmA, const CU
   cfg.blockDim = dim3(C::kThreads);
   cfg.dynamicSmemBytes = C::kSmemBytes;
   cfg.stream = call.stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = CG;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = call.overlap ? 2 : 1;
   e = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmC, args);
   if (e != cudaSuccess) { set_error("kernel launch failed: %s", cudaGetErrorString(e)); return SP_ERR_CUDA; }
   return SP_OK;
@@ -816,6 +826,7 @@ int launch_gemm(const GemmCall& call) {
   args.sched = call.sched;
   args.sk = SkPlan{0, args.units, call.sched.T};   // no tail: every slot is a whole tile
   args.sk_ws = nullptr; args.sk_flags = nullptr; args.sk_epoch = 0;
+  args.overlap = call.overlap;
   if (call.stream_k) {
     // units are not capped by the tile count here: a problem smaller than a wave is spread over all of them
     const int all_units = gemm_units(call.tile_m, call.tile_n, kMaxTiles);

@@ -55,6 +55,7 @@ struct GemmCall {
   uint32_t die_mask[8];
   sp_trace_rec* trace_dev;  // nullptr unless tracing
   int stream_k;             // SP_FLAG_STREAM_K: split the tail wave along k
+  int overlap;              // SP_FLAG_OVERLAP: launch with programmatic stream serialisation, never wait for the predecessor
   int32_t* sk_flags_dev;    // kSkFlagBytes of flags, zero when allocated
   int32_t sk_epoch;         // value the flags take in this launch: 1, 2, ... per workspace
   float* sk_ws_dev;         // kSkWorkspaceBytes of partial tiles

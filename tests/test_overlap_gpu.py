@@ -1,0 +1,76 @@
+"""SP_FLAG_OVERLAP: launches declared independent of their predecessor start while it is still running.  The results
+must be those of ordinary launches, and whatever follows on the stream must still see both kernels complete."""
+
+import numpy as np
+import pytest
+
+import paper_2508_20258_b200 as sp
+from oracle import gemm as G
+from paper_2508_20258_b200 import synth
+
+pytestmark = pytest.mark.gpu
+torch = pytest.importorskip("torch")
+OV = sp.FLAG_OVERLAP
+
+
+def dev_bf16(bits):
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def test_chain_of_independent_gemms_matches_the_oracle():
+    shapes = [(1024, 1280, 768, (256, 256)), (640, 896, 1000, (128, 128)), (2304, 2560, 512, (256, 512)),
+              (512, 512, 512, (128, 256)), (1160, 600, 520, (256, 128))]
+    problems = []
+    for i, (M, N, K, tile) in enumerate(shapes):
+        A, B = synth.make_int_inputs(M, N, K, seed=40 + i)
+        problems.append((dev_bf16(A), dev_bf16(B), torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda"),
+                         tile, G.gemm_full(A, B)[0]))
+    orders = [(sp.HILBERT, {}), (sp.GROUP_M, dict(group=2)), (sp.ROW_MAJOR, {}), (sp.MORTON, {}), (sp.GROUP_N, dict(group=3))]
+    for rep in range(3):                                  # the first round builds tile tables, later rounds overlap fully
+        for (dA, dB, dC, tile, _), (scheme, kw) in zip(problems, orders):
+            if rep:
+                dC.fill_(float("nan"))
+        for (dA, dB, dC, tile, _), (scheme, kw) in zip(problems, orders):
+            sp.gemm(dA, dB, dC, scheme, sp.make_params(tile_m=tile[0], tile_n=tile[1], out_dtype=1, flags=OV, **kw))
+        assert sp.get_status() == 0
+        for (_, _, dC, _, ref) in problems:
+            assert np.array_equal(dC.cpu().numpy().astype(np.float64), ref)
+
+
+def test_a_copy_behind_a_short_overlapped_launch_still_sees_the_long_predecessor_complete():
+    w, A, B = synth.make_workload("cfg2")
+    dA, dB = dev_bf16(A), dev_bf16(B)
+    big = torch.empty((w.M, w.N), dtype=torch.bfloat16, device="cuda")
+    p = sp.make_params(tile_m=256, tile_n=256)
+    sp.gemm(dA, dB, big, sp.ROW_MAJOR, p)
+    want = big.cpu()
+    a2, b2 = synth.make_int_inputs(128, 128, 64, seed=3)
+    dA2, dB2 = dev_bf16(a2), dev_bf16(b2)
+    small = torch.empty((128, 128), dtype=torch.bfloat16, device="cuda")
+    host = torch.empty((w.M, w.N), dtype=torch.bfloat16).pin_memory()
+    for _ in range(5):
+        big.zero_()
+        torch.cuda.synchronize()
+        sp.gemm(dA, dB, big, sp.ROW_MAJOR, p)                                        # about 0.1 ms
+        sp.gemm(dA2, dB2, small, sp.ROW_MAJOR, sp.make_params(tile_m=128, tile_n=128, flags=OV))   # microseconds, overlapped
+        host.copy_(big, non_blocking=True)                                            # ordered behind both
+        torch.cuda.synchronize()
+        assert torch.equal(host.view(torch.int16), want.view(torch.int16))
+    assert sp.get_status() == 0
+
+
+def test_overlap_rejections():
+    A, B = synth.make_int_inputs(512, 512, 512, seed=1)
+    dA, dB = dev_bf16(A), dev_bf16(B)
+    dC = torch.zeros((512, 512), dtype=torch.bfloat16, device="cuda")
+    for bad in (OV | sp.FLAG_STREAM_K, OV | sp.FLAG_DIE_PINNED):
+        with pytest.raises(sp.SpError) as e:
+            sp.gemm(dA, dB, dC, sp.DIE_SPLIT, sp.make_params(tile_m=128, tile_n=128, inner_scheme=sp.ROW_MAJOR, flags=bad))
+        assert e.value.status == sp.ERR_INVALID_ARG
+    with pytest.raises(sp.SpError) as e:
+        sp.gemm_trace(dA, dB, dC, sp.ROW_MAJOR, sp.make_params(tile_m=128, tile_n=128, flags=OV))
+    assert e.value.status == sp.ERR_INVALID_ARG
+    with pytest.raises(sp.SpError) as e:
+        sp.gemm_noalloc(dA, dB, dC, sp.ROW_MAJOR, sp.make_params(tile_m=128, tile_n=128, flags=OV))
+    assert e.value.status == sp.ERR_INVALID_ARG
+    assert sp.get_status() == 0 and float(dC.float().abs().sum()) == 0.0
