@@ -157,7 +157,10 @@ int sp_tile_map_device(int64_t M, int64_t N, int32_t tileM, int32_t tileN, int s
  * Products are accumulated in fp32 on the tensor cores.  M and N need not be tile multiples.
  * Errors (all detected on the host, nothing launched): as sp_tile_map, plus SP_ERR_ALIGNMENT (A, B or C not
  * 16-byte aligned; K or N not a multiple of 8), SP_ERR_UNSUPPORTED (tile shape), SP_ERR_DEVICE, SP_ERR_CUDA.
- * The first call for a given (grid, scheme) may allocate a cached tile table; later calls allocate nothing.
+ * The first call for a given (grid, scheme) may allocate a cached tile table; later calls allocate nothing and
+ * issue only the kernel launch (plus one small memset node with SP_FLAG_DIE_PINNED), so after one warm-up call per
+ * (shape, scheme, params) further calls can be recorded into a CUDA graph by stream capture and replayed; the
+ * pointers and the order are then those of the recording.
  * A device-side wait that expires is reported by sp_get_status, not here. */
 int sp_gemm(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t K, int scheme,
             const sp_params* params, void* stream);

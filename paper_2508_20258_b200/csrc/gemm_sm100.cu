@@ -691,12 +691,12 @@ int make_map_plain(CUtensorMap* m, const void* base, int64_t rows, int64_t cols,
 // device can hold at once (asked of the occupancy calculator, cached per shape).
 template <int CG, int BN>
 static int max_units() {
-  static int cached = 0;
-  if (cached > 0) return cached;
+  static int cached[64] = {};      // per device
   using C = Cfg<CG, BN>;
   auto kern = gemm_kernel<CG, BN, false, false>;
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return -1;
+  if (cached[dev & 63] > 0) return cached[dev & 63];
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return -1;
   int units = sms / CG;
   if (CG == 2) {
@@ -713,7 +713,7 @@ static int max_units() {
     if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) == cudaSuccess && n > 0 && n < units) units = n;
     cudaGetLastError();
   }
-  cached = units;
+  cached[dev & 63] = units;
   return units;
 }
 
@@ -734,12 +734,11 @@ static int launch_variant(const GemmCall& call, const CUtensorMap& tmA, const CU
                           const GemmArgs& args) {
   using C = Cfg<CG, BN>;
   auto kern = gemm_kernel<CG, BN, B_NK, OUT_F32>;
-  static bool configured = false;  // per instantiation; attribute is per device but identical everywhere
+  static uint64_t configured = 0;  // per instantiation, one bit per device
   cudaError_t e = cudaSuccess;
-  if (!configured) {
+  if (first_use_on_this_device(configured)) {
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemBytes);
-    if (e != cudaSuccess) { set_error("cudaFuncSetAttribute(smem=%u) failed: %s", C::kSmemBytes, cudaGetErrorString(e)); return SP_ERR_CUDA; }
-    configured = true;
+    if (e != cudaSuccess) { configured = 0; set_error("cudaFuncSetAttribute(smem=%u) failed: %s", C::kSmemBytes, cudaGetErrorString(e)); return SP_ERR_CUDA; }
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(args.units * CG));

@@ -22,6 +22,17 @@ constexpr size_t kSkWorkspaceBytes = (size_t)148 * 128 * 256 * 4;
 
 void set_error(const char* fmt, ...);
 
+// Per-function set-up that CUDA keeps per device (cudaFuncSetAttribute): true the first time it is asked for the
+// current device with this mask.  A lost race only repeats a harmless call.
+inline bool first_use_on_this_device(uint64_t& done_mask) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return true;
+  const uint64_t bit = 1ull << (dev & 63);
+  if (done_mask & bit) return false;
+  done_mask |= bit;
+  return true;
+}
+
 // Validates sizes and parameters and fills `out`.  Returns an sp_status.
 int resolve_sched(int64_t M, int64_t N, int32_t tileM, int32_t tileN, int scheme, const sp_params* params, Sched* out);
 

@@ -156,12 +156,11 @@ int launch_stencil(const void* in, void* out, int64_t M, int64_t N, float c_cent
   CUtensorMap tmIn;
   int rc = make_map_plain(&tmIn, in, M, N, kStBoxRows, kStBoxCols);
   if (rc != SP_OK) return rc;
-  static bool configured = false;
+  static uint64_t configured = 0;   // one bit per device
   cudaError_t e;
-  if (!configured) {
+  if (first_use_on_this_device(configured)) {
     e = cudaFuncSetAttribute(stencil_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStSmem);
-    if (e != cudaSuccess) { set_error("cudaFuncSetAttribute failed: %s", cudaGetErrorString(e)); return SP_ERR_CUDA; }
-    configured = true;
+    if (e != cudaSuccess) { configured = 0; set_error("cudaFuncSetAttribute failed: %s", cudaGetErrorString(e)); return SP_ERR_CUDA; }
   }
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {

@@ -329,3 +329,31 @@ def test_small_host_gemm_and_shutdown_then_reuse():
     sp.gemm_host(A.view(np.int16), B.view(np.int16), hC, sp.DIE_SPLIT, sp.make_params(tile_m=128, tile_n=128, out_dtype=1,
                                                                                    inner_scheme=sp.MORTON))
     assert np.array_equal(hC.astype(np.float64), ref)
+
+
+def test_gemm_launches_replay_from_a_cuda_graph():
+    # warm caches first (tile table, status word), then capture three launches on a side stream and replay them
+    A, B = synth.make_int_inputs(768, 1024, 512, seed=23)
+    ref, _ = G.gemm_full(A, B)
+    dA, dB = dev_bf16(A), dev_bf16(B)
+    outs = [torch.zeros((768, 1024), dtype=torch.float32, device="cuda") for _ in range(3)]
+    cases = [(sp.HILBERT, sp.make_params(tile_m=128, tile_n=128, out_dtype=1)),
+             (sp.GROUP_M, sp.make_params(tile_m=256, tile_n=256, out_dtype=1, group=2)),
+             (sp.ROW_MAJOR, sp.make_params(tile_m=256, tile_n=512, out_dtype=1))]
+    for (scheme, p), o in zip(cases, outs):
+        sp.gemm(dA, dB, o, scheme, p)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            for (scheme, p), o in zip(cases, outs):
+                sp.gemm(dA, dB, o, scheme, p, side)
+    for rep in range(3):
+        for o in outs:
+            o.fill_(float("nan"))
+        graph.replay()
+        torch.cuda.synchronize()
+        for o in outs:
+            assert np.array_equal(o.cpu().numpy().astype(np.float64), ref)
+    assert sp.get_status() == 0
