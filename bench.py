@@ -33,7 +33,7 @@ L2_BYTES = 126 * 2 ** 20
 # DRAM bytes per launch of the GEMM kernel from the ncu captures summarised under profiles/
 # (dram__bytes_read.sum + dram__bytes_write.sum), keyed by (workload, tile, scheme spec); None = not captured.
 NCU_DRAM_BYTES = {
-    ("cfg3", "256x512", "group_n:8"): 0.970e9,   # profiles/gemm_kernel_cfg3_256x512_group_n8_full.md (mean of 2 launches)
+    ("cfg3", "256x512", "group_n:8"): 0.952e9,   # profiles/gemm_kernel_cfg3_256x512_group_n8_full.md (mean of 2 launches)
     ("cfg3", "256x256", "die_split:m:group_m:8:p"): 1.071e9,   # profiles/l2_hit_rate_per_scheme.md
     ("cfg5", "256x256", "die_split:m:group_m:8:p"): 1.247e9,
     ("cfg3", "256x256", "group_m:8"): 1.200e9,   # profiles/gemm_kernel_cfg3_group_m8_full.md (mean of 2 launches)

@@ -93,6 +93,13 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
          ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
 }
 
+// The same descriptor for another start address: `base` was built for address 0, `addr16` is the byte address >> 4
+// (below 2^14: shared memory ends at 227 KiB).  Only the low word changes: one 32-bit add per descriptor in the
+// issue loop instead of the full field arithmetic.
+__device__ __forceinline__ uint64_t desc_at(uint64_t base, uint32_t addr16) {
+  return ((uint64_t)(uint32_t)(base >> 32) << 32) | (uint64_t)((uint32_t)base + addr16);
+}
+
 // Instruction descriptor, kind::f16: D fp32, A and B bf16, A K-major, B K- or MN-major.
 __host__ __device__ constexpr uint32_t make_idesc(int m, int n, bool b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) |
@@ -253,6 +260,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     // Whole warp in the loop, one elected lane issues: descriptors stay warp-uniform values.
     if (rank == 0) {
       constexpr uint32_t idesc = make_idesc(TILE_M, C::kMmaN, !B_NK);
+      const uint64_t da0 = smem_desc(0, 16, 1024), db0 = smem_desc(0, args.b_lbo, args.b_sbo);
+      const uint32_t b_kstep16 = args.b_kstep >> 4;
       int stage = 0;
       uint32_t phase = 0;
       int it = 0;
@@ -301,8 +310,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                   const uint32_t sb = sa + C::kABytes + (uint32_t)(c * C::kMmaCols * kBK * 2);
 #pragma unroll
                   for (int k = 0; k < kBK / kUmmaK; ++k) {
-                    const uint64_t da = smem_desc(sa + k * (kUmmaK * 2), 16, 1024);
-                    const uint64_t db = smem_desc(sb + k * args.b_kstep, args.b_lbo, args.b_sbo);
+                    const uint64_t da = desc_at(da0, (sa >> 4) + k * (kUmmaK * 2 / 16));
+                    const uint64_t db = desc_at(db0, (sb >> 4) + k * b_kstep16);
                     umma_bf16<CG>(tmem_base + (uint32_t)(c * C::kMmaN), da, db, idesc, (uint32_t)(((kb + i) | k) != 0));
                   }
                 }
@@ -339,8 +348,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             if (elect_one()) {
 #pragma unroll
               for (int k = 0; k < kBK / kUmmaK; ++k) {
-                const uint64_t da = smem_desc(sa + k * (kUmmaK * 2), 16, 1024);
-                const uint64_t db = smem_desc(sb + c * (C::kMmaCols * kBK * 2) + k * args.b_kstep, args.b_lbo, args.b_sbo);
+                const uint64_t da = desc_at(da0, (sa >> 4) + k * (kUmmaK * 2 / 16));
+                const uint64_t db = desc_at(db0, ((sb + c * (C::kMmaCols * kBK * 2)) >> 4) + k * b_kstep16);
                 umma_bf16<CG>(d_tmem, da, db, idesc, (uint32_t)(kb > wk.k0 || k != 0));
               }
               if (kb == wk.k1 - 1) umma_commit<CG>(bar_tfull + 8 * part);   // this part is complete

@@ -70,12 +70,26 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
+// try_wait that lets the hardware keep the thread suspended for up to `ns` nanoseconds while the phase is incomplete
+// (it still resumes as soon as the phase completes): fewer trips round the polling loop for long waits.
+__device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity, uint32_t ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(ns)
+      : "memory");
+  return ok != 0;
+}
+
 // Bounded wait.  Returns false after kTimeoutNs or once the status word is set by anyone.
 static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, int32_t* status, int code,
                                             unsigned long long timeout_ns = kTimeoutNs) {
   const unsigned long long t0 = globaltimer();
   for (uint32_t i = 1;; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_try_wait_hint(bar, parity, 20000u)) return true;
     if ((i & 63u) == 0) {
       if (*(volatile int32_t*)status != 0) return false;
       if (globaltimer() - t0 > timeout_ns) {
