@@ -87,9 +87,11 @@ typedef enum {
 
 #define SP_FLAG_OVERLAP 16u   /* sp_gemm only.  The caller states that this launch is independent of the kernel before it on the
                                  stream: it reads nothing that kernel writes, and it may start writing C while that kernel is
-                                 still running.  The launch is then made with programmatic stream serialisation and never
-                                 waits for its predecessor; every GEMM launch of this library signals at its start that its
-                                 successor may be scheduled.  CTAs of the next GEMM then take over SMs as the CTAs of the
+                                 still running.  Every GEMM launch of this library is made with programmatic stream
+                                 serialisation and signals at its start that its successor may be scheduled; an ordinary
+                                 launch then waits, after its set-up and before it touches global memory, until the kernel
+                                 before it has completed and its writes are visible (so only launch latency and set-up
+                                 overlap, and the stream order is the usual one); a launch with this flag does not wait.  CTAs of the next GEMM then take over SMs as the CTAs of the
                                  previous one finish, which fills the partly empty last wave of back-to-back independent
                                  GEMMs.  The paper has no counterpart.  A launch that first has to build its tile table (first
                                  use of a non-arithmetic order) is made without the overlap.  Not with SP_FLAG_DIE_PINNED,

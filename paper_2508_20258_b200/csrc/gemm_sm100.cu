@@ -77,7 +77,7 @@ struct GemmArgs {
   float* sk_ws;                    // one fp32 partial tile per unit: [unit][cta of the unit][lane quarter][column][lane]
   int32_t* sk_flags;               // one word per (unit, cta, lane quarter): set to sk_epoch once that partial is complete
   int32_t sk_epoch;                // differs from launch to launch on one workspace, so the flags need no clearing
-  int overlap;                     // launched with programmatic stream serialisation (never waits for its predecessor)
+  int overlap;                     // 1: never waits for its predecessor before working (only before exiting)
   Sched sched;
 };
 
@@ -175,6 +175,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   unit_sync<CG>();
   tcgen05_fence_after();
   const uint32_t tmem_base = *tmem_slot_ptr;
+  // Every launch is made with programmatic stream serialisation: the set-up above may run while the kernel before
+  // this one on the stream is still finishing (its CTAs leaving free the SMs ours start on).  From here on global
+  // memory is touched, so an ordinary launch now waits until that kernel has completed and its writes are visible;
+  // a launch declared independent of it (SP_FLAG_OVERLAP) goes straight on and waits only before it exits.
+  if (!args.overlap) asm volatile("griddepcontrol.wait;" ::: "memory");
 
   // whole tiles of this unit: slots s_first, s_first + s_step, ... below s_end; then its segments of the stream-K tail
   int s_first = unit, s_step = args.units, s_end = args.sk.first_slot;
@@ -762,7 +767,7 @@ static int launch_variant(const GemmCall& call, const CUtensorMap& tmA, const CU
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = call.overlap ? 2 : 1;
+  cfg.numAttrs = 2;
   e = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmC, args);
   if (e != cudaSuccess) { set_error("kernel launch failed: %s", cudaGetErrorString(e)); return SP_ERR_CUDA; }
   return SP_OK;
