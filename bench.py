@@ -200,7 +200,7 @@ def run_ours(args) -> int:
     else:
         w = synth.WORKLOADS[args.workload]
         _, A, B = synth.make_workload(args.workload, b_is_nk=bool(b_nk))
-    if not args.tile and args.workload in DEFAULT_TILE and not (args.sweep or args.sweep_sustained or args.profile_sweep):
+    if not args.tile and args.workload in DEFAULT_TILE and not (args.sweep or args.sweep_sustained or args.profile_sweep or args.alternate):
         args.tile = DEFAULT_TILE[args.workload]
     tile_m, tile_n = (int(v) for v in args.tile.split("x")) if args.tile else (w.tile_m, w.tile_n)
     out_f32 = int(w.out_dtype == "fp32")
@@ -233,6 +233,8 @@ def run_ours(args) -> int:
 
     if args.sweep_sustained:
         return run_sweep_sustained(args, sp, w, dA, dB, dC, params_for, flops, stream)
+    if args.alternate:
+        return run_alternate(args, sp, w, dA, dB, dC, params_for, flops, stream)
     if args.sweep:
         return run_sweep(args, sp, w, dA, dB, dC, params_for, flops, stream)
     if args.profile_sweep:                     # one launch per scheme, in SWEEPS order: the command ncu wraps
@@ -444,6 +446,57 @@ def run_sweep_sustained(args, sp, w, dA, dB, dC, params_for, flops, stream) -> i
     return 0
 
 
+def run_alternate(args, sp, w, dA, dB, dC, params_for, flops, stream) -> int:
+    """The given schemes (and, with the pseudo-scheme 'cublas', torch.matmul on the same tensors) in alternating blocks of
+    --steps launches, --rounds rounds, median per arm: every arm sees the same thermal state.  JSON lines to stdout."""
+    import torch
+    arms = []
+    ref = None
+    for spec in args.alternate.split(","):
+        if spec == "cublas":
+            if args.b_layout != "kn" or dC.dtype != torch.bfloat16:
+                raise SystemExit("the cublas arm needs B stored K x N and bf16 output")
+            ref = torch.empty_like(dC)
+            arms.append((spec, lambda: torch.matmul(dA, dB, out=ref)))
+        else:
+            s, p = params_for(spec)
+            arms.append((spec, lambda s=s, p=p: sp.gemm(dA, dB, dC, s, p, stream)))
+    n = max(args.steps, 1)
+    for _, fn in arms:
+        for _ in range(n):
+            fn()
+    torch.cuda.synchronize()
+    times = {spec: [] for spec, _ in arms}
+    mhz = {spec: [] for spec, _ in arms}
+    sampler = benchutil.ClockSampler(0).start()
+    for _ in range(args.rounds):
+        for spec, fn in arms:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            t0 = time.perf_counter()
+            e0.record(stream)
+            for _ in range(n):
+                fn()
+            e1.record(stream)
+            e1.synchronize()
+            t1 = time.perf_counter()
+            times[spec].append(e0.elapsed_time(e1) / n)
+            # the host runs ahead of the GPU: only the second half of the block is sure to have the GPU busy with this arm
+            c = sampler.summary(0.5 * (t0 + t1), t1)
+            if c["sm_mhz"] is not None and c["samples"] >= 3 and "+-50" not in c["window"]:
+                mhz[spec].append(c["sm_mhz"])
+    sampler.stop()
+    assert sp.get_status() == 0
+    base = None
+    for spec, _ in arms:
+        ms = float(np.median(times[spec]))
+        base = base or ms
+        clk = float(np.median(mhz[spec])) if mhz[spec] else None
+        print(json.dumps({"alternate": w.name, "arm": spec, "ms": ms, "tflops": flops / ms / 1e9, "first_arm_over_this": base / ms,
+                          "block_launches": n, "rounds": args.rounds, "sm_mhz": clk,
+                          "sm_cycles_per_launch": None if clk is None else ms * 1e-3 * clk * 1e6}), flush=True)
+    return 0
+
+
 def run_sweep(args, sp, w, dA, dB, dC, params_for, flops, stream) -> int:
     """Every scheme of the workload, interleaved (ABAB) to share thermal state; JSON lines to stdout."""
     import torch
@@ -621,6 +674,9 @@ def main() -> int:
     ap.add_argument("--sweep", action="store_true", help="time every scheme of the workload")
     ap.add_argument("--sweep-sustained", action="store_true", help="time every scheme in its own back-to-back loop")
     ap.add_argument("--profile-sweep", action="store_true", help="launch each scheme once (for ncu counters)")
+    ap.add_argument("--alternate", default=None, metavar="SPEC,SPEC[,cublas]",
+                    help="time the given schemes in alternating blocks of --steps launches (--rounds rounds, median)")
+    ap.add_argument("--rounds", type=int, default=6)
     ap.add_argument("--b-layout", default="kn", choices=["kn", "nk"], help="B stored K x N (default) or N x K")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
