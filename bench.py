@@ -54,6 +54,10 @@ def parse_scheme(spec: str):
         scheme, kw = parse_scheme(spec[:-2])
         kw["flags"] = kw.get("flags", 0) | sp.FLAG_STREAM_K
         return scheme, kw
+    if spec.endswith("+c"):    # any order, slots handed out by cluster launch control instead of a fixed stride
+        scheme, kw = parse_scheme(spec[:-2])
+        kw["flags"] = kw.get("flags", 0) | sp.FLAG_CLC
+        return scheme, kw
     if spec.endswith("+o"):    # any order, launches declared independent of their predecessor (they overlap its tail)
         scheme, kw = parse_scheme(spec[:-2])
         kw["flags"] = kw.get("flags", 0) | sp.FLAG_OVERLAP

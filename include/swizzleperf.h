@@ -85,6 +85,15 @@ typedef enum {
                                  (SP_ERR_INVALID_ARG) nor for the 256x512 tile (SP_ERR_UNSUPPORTED).  In a trace the record
                                  of a split tile describes the piece that stored it. */
 
+#define SP_FLAG_CLC 32u       /* sp_gemm / sp_gemm_trace / sp_gemm_host: dynamic scheduling by cluster launch control.  The grid has
+                                 one cluster per tile instead of one per persistent unit; the clusters that get to run compute
+                                 the slot of their own index and then keep asking the hardware to cancel a cluster that has not
+                                 started yet and to hand them its index (clusterlaunchcontrol.try_cancel), until none is left.
+                                 Slots are then taken in the order the hardware starts and cancels clusters, first come first
+                                 served, not with a fixed stride; every tile still runs exactly once and C has the same bits.
+                                 The counterpart, on this hardware, of the paper's premise that the scheduler hands out
+                                 consecutive block ids in a fixed pattern.  Not with SP_FLAG_DIE_PINNED or SP_FLAG_STREAM_K
+                                 (SP_ERR_INVALID_ARG). */
 #define SP_FLAG_OVERLAP 16u   /* sp_gemm only.  The caller states that this launch is independent of the kernel before it on the
                                  stream: it reads nothing that kernel writes, and it may start writing C while that kernel is
                                  still running.  Every GEMM launch of this library is made with programmatic stream

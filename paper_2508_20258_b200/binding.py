@@ -288,7 +288,7 @@ def gemm_units(tile_m: int, tile_n: int, T: int) -> int:
     return int(lib().sp_gemm_units(tile_m, tile_n, T))
 
 
-FLAG_DIE_PINNED, FLAG_SERPENTINE, FLAG_STREAM_K, FLAG_OVERLAP = 2, 4, 8, 16
+FLAG_DIE_PINNED, FLAG_SERPENTINE, FLAG_STREAM_K, FLAG_OVERLAP, FLAG_CLC = 2, 4, 8, 16, 32
 STREAMK_MAX_SEGMENTS = 8
 WORK_FULL, WORK_CONTRIB, WORK_OWNER = 0, 1, 2
 

@@ -369,6 +369,13 @@ static int gemm_common(const void* A, const void* B, void* C, int64_t M, int64_t
     call.sms_on_die[0] = ds->sms_on_die[0]; call.sms_on_die[1] = ds->sms_on_die[1];
     for (int i = 0; i < 8; ++i) call.die_mask[i] = ds->die_mask[i];
   }
+  if (params && (params->flags & SP_FLAG_CLC)) {
+    if (params->flags & (SP_FLAG_DIE_PINNED | SP_FLAG_STREAM_K)) {
+      set_error("SP_FLAG_CLC cannot be combined with SP_FLAG_DIE_PINNED or SP_FLAG_STREAM_K");
+      return SP_ERR_INVALID_ARG;
+    }
+    call.clc = 1;
+  }
   if (params && (params->flags & SP_FLAG_STREAM_K)) {
     if (call.pinned) {
       set_error("SP_FLAG_STREAM_K cannot be combined with SP_FLAG_DIE_PINNED");

@@ -66,6 +66,10 @@ extern "C" int sp_gemm_noalloc(const void* A, const void* B, void* C, int64_t M,
     set_error("SP_FLAG_STREAM_K needs a workspace and is not available in sp_gemm_noalloc");
     return SP_ERR_INVALID_ARG;
   }
+  if (params && (params->flags & SP_FLAG_CLC)) {
+    set_error("SP_FLAG_CLC is not available in sp_gemm_noalloc");
+    return SP_ERR_INVALID_ARG;
+  }
   if (params && (params->flags & SP_FLAG_OVERLAP)) {
     set_error("SP_FLAG_OVERLAP is not available in sp_gemm_noalloc (its scratch is rewritten by every call)");
     return SP_ERR_INVALID_ARG;

@@ -38,6 +38,7 @@ constexpr int kUmmaK = 16;       // k extent of one tcgen05.mma with 16-bit inpu
 constexpr uint32_t kSmemLimit = 232448;  // 227 KiB opt-in maximum per CTA
 constexpr uint32_t kBarrierBytes = 1024;
 constexpr int kTmemCols = 512;
+constexpr int kClcDepth = 4;     // responses of cluster launch control in flight / not yet read by every role
 
 template <int CG, int BN>
 struct Cfg {
@@ -78,6 +79,8 @@ struct GemmArgs {
   int32_t* sk_flags;               // one word per (unit, cta, lane quarter): set to sk_epoch once that partial is complete
   int32_t sk_epoch;                // differs from launch to launch on one workspace, so the flags need no clearing
   int overlap;                     // 1: never waits for its predecessor before working (only before exiting)
+  int clc;                         // 1: one cluster per tile is launched; running clusters take over the slots of clusters
+                                   //    not yet started (cluster launch control) instead of striding through the slots
   Sched sched;
 };
 
@@ -133,6 +136,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   const uint32_t bar_tfull = bar_base + 16 * S;    // 2 barriers
   const uint32_t bar_tempty = bar_tfull + 16;      // 2 barriers
   const uint32_t tmem_slot = bar_tempty + 16;      // 4 bytes
+  const uint32_t clc_resp = bar_base + 256;        // kClcDepth responses of 16 bytes (cluster launch control)
+  const uint32_t clc_full = clc_resp + 16 * kClcDepth, clc_empty = clc_full + 8 * kClcDepth;
   volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -147,6 +152,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   if (threadIdx.x == 0) {
     for (int i = 0; i < S; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_empty + 8 * i, 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(bar_tfull + 8 * i, 1); mbar_init(bar_tempty + 8 * i, 4 * CG); }
+    // a response is read by the producer and the epilogue warps of every CTA of the unit and by the leader's MMA warp
+    for (int i = 0; i < kClcDepth; ++i) { mbar_init(clc_full + 8 * i, 1); mbar_init(clc_empty + 8 * i, CG * (1 + C::kEpiWarps) + 1); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -191,9 +198,27 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   }
   const int n_whole = s_first < s_end ? (s_end - s_first + s_step - 1) / s_step : 0;
   const int n_items = n_whole + sk_segments(args.sk, unit, KB);
-  auto work_at = [&](int i) -> Work {
-    if (i < n_whole) { Work w; w.slot = s_first + i * s_step; w.k0 = 0; w.k1 = KB; w.kind = kWorkFull; return w; }
-    return sk_segment(args.sk, unit, i - n_whole, KB);
+  // The i-th piece of work of this unit; slot < 0 when there is none.  Called by whole warps, every role with its own
+  // counter.  With cluster launch control the first tile is the cluster's own and every further one comes from a
+  // response the leader's producer warp asked for one tile earlier (ring of kClcDepth responses, written to every CTA
+  // of the unit by the hardware; a reader hands the entry back on the leader's barrier).
+  auto work_at = [&](int i, int wait_code) -> Work {
+    Work w; w.k0 = 0; w.k1 = KB; w.kind = kWorkFull; w.slot = -1;
+    if (args.clc) {
+      if (i == 0) { w.slot = unit; return w; }
+      const int e = (i - 1) % kClcDepth;
+      bool okc = mbar_wait(clc_full + 8 * e, (uint32_t)((i - 1) / kClcDepth) & 1u, args.status, wait_code);
+      okc = __all_sync(0xffffffffu, okc);
+      uint32_t valid = 0, first_cta = 0;
+      if (okc) clc_decode(clc_resp + 16 * e, valid, first_cta);
+      __syncwarp();
+      if (okc && elect_one()) mbar_arrive_cluster(CG == 1 ? clc_empty + 8 * e : mapa(clc_empty + 8 * e, 0));
+      if (okc && valid) w.slot = (int)(first_cta / CG);
+      return w;
+    }
+    if (i < n_whole) { w.slot = s_first + i * s_step; return w; }
+    if (i < n_items) return sk_segment(args.sk, unit, i - n_whole, KB);
+    return w;
   };
 
   if (warp == 0) {
@@ -204,9 +229,25 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int item = 0; item < n_items && ok; ++item) {
-        const Work wk = work_at(item);
+      for (int item = 0; ok; ++item) {
+        const Work wk = work_at(item, (kRoleProducer << 8) | 4);
+        if (wk.slot < 0) break;
         const int s = wk.slot;
+        if (args.clc) {
+          // ask for the tile after this one: every CTA arms its own barrier for the 16 bytes the hardware will write
+          // to it; the leader first makes sure every reader has handed the entry back, then issues the request
+          const int e = item % kClcDepth;
+          if (rank == 0 && item >= kClcDepth) {
+            ok = mbar_wait(clc_empty + 8 * e, (uint32_t)(item / kClcDepth - 1) & 1u, args.status, (kRoleProducer << 8) | 5);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+          }
+          if (elect_one()) {
+            mbar_arrive_expect_tx(clc_full + 8 * e, 16);
+            if (rank == 0) clc_try_cancel<CG>(clc_resp + 16 * e, clc_full + 8 * e);
+          }
+          __syncwarp();
+        }
         const int t = tile_of_slot(args, s);
         const int tm = t / Tn, tn = t - tm * Tn;
         const int row0 = tm * TILE_M + (int)rank * 128;
@@ -275,8 +316,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       // Two MMA tiles (BN = 512): two parts, each with its own pair of barriers, so the epilogue can drain the
       // first while the second is still being computed, and the next tile can start on the first part while the
       // second is being drained.
-      for (; it < n_items && ok; ++it) {
-        const Work wk = work_at(it);
+      for (; ok; ++it) {
+        const Work wk = work_at(it, (kRoleMma << 8) | 4);
+        if (wk.slot < 0) break;
         const int s = wk.slot;
         const int buf = it % C::kBufs;
         const uint32_t use = C::kNT == 1 ? ((uint32_t)(it / C::kBufs) & 1u) : ((uint32_t)it & 1u);
@@ -389,8 +431,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c * C::kMmaN);
       int it2 = 0;
       bool ok2 = true;
-      for (; it2 < n_items && ok2; ++it2) {
-        const int s = work_at(it2).slot;
+      for (; ok2; ++it2) {
+        const int s = work_at(it2, (kRoleEpilogue << 8) | 4).slot;
+        if (s < 0) break;
         const int t = tile_of_slot(args, s);
         const int tm = t / Tn, tn = t - tm * Tn;
         const uint32_t use = (uint32_t)it2 & 1u;
@@ -465,8 +508,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     int it = 0;
     int chunk = 0;                 // staging buffers alternate per stored chunk, across tiles
     bool ok = true;
-    for (; it < n_items && ok; ++it) {
-      const Work wk = work_at(it);
+    for (; ok; ++it) {
+      const Work wk = work_at(it, (kRoleEpilogue << 8) | 4);
+      if (wk.slot < 0) break;
       const int s = wk.slot;
       const int t = tile_of_slot(args, s);
       const int tm = t / Tn, tn = t - tm * Tn;
@@ -755,7 +799,7 @@ static int launch_variant(const GemmCall& call, const CUtensorMap& tmA, const CU
     if (e != cudaSuccess) { configured = 0; set_error("cudaFuncSetAttribute(smem=%u) failed: %s", C::kSmemBytes, cudaGetErrorString(e)); return SP_ERR_CUDA; }
   }
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(args.units * CG));
+  cfg.gridDim = dim3((unsigned)((args.clc ? args.sched.T : args.units) * CG));   // one cluster per tile, or per persistent unit
   cfg.blockDim = dim3(C::kThreads);
   cfg.dynamicSmemBytes = C::kSmemBytes;
   cfg.stream = call.stream;
@@ -840,6 +884,7 @@ int launch_gemm(const GemmCall& call) {
   args.sk = SkPlan{0, args.units, call.sched.T};   // no tail: every slot is a whole tile
   args.sk_ws = nullptr; args.sk_flags = nullptr; args.sk_epoch = 0;
   args.overlap = call.overlap;
+  args.clc = call.clc;
   if (call.stream_k) {
     // units are not capped by the tile count here: a problem smaller than a wave is spread over all of them
     const int all_units = gemm_units(call.tile_m, call.tile_n, kMaxTiles);

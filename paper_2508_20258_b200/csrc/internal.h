@@ -66,6 +66,7 @@ struct GemmCall {
   uint32_t die_mask[8];
   sp_trace_rec* trace_dev;  // nullptr unless tracing
   int stream_k;             // SP_FLAG_STREAM_K: split the tail wave along k
+  int clc;                  // SP_FLAG_CLC: one cluster per tile, tiles of unstarted clusters taken over by running ones
   int overlap;              // SP_FLAG_OVERLAP: launch with programmatic stream serialisation, never wait for the predecessor
   int32_t* sk_flags_dev;    // kSkFlagBytes of flags, zero when allocated
   int32_t sk_epoch;         // value the flags take in this launch: 1, 2, ... per workspace

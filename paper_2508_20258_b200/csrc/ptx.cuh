@@ -110,6 +110,40 @@ __device__ __forceinline__ int32_t ld_acquire_gpu(const int32_t* p) {
   return v;
 }
 
+// Cluster launch control: ask the hardware to cancel the launch of a cluster of this grid that has not started yet and
+// to hand its first CTA id to this cluster instead.  The 16-byte response is written to `resp` (same offset in every
+// CTA of the cluster when CG > 1) and completes 16 bytes on the mbarrier `bar` (same offset in every CTA).
+template <int CG>
+__device__ __forceinline__ void clc_try_cancel(uint32_t resp, uint32_t bar) {
+  if constexpr (CG == 1) {
+    asm volatile("clusterlaunchcontrol.try_cancel.async.shared::cta.mbarrier::complete_tx::bytes.b128 [%0], [%1];"
+                 ::"r"(resp), "r"(bar) : "memory");
+  } else {
+    asm volatile(
+        "clusterlaunchcontrol.try_cancel.async.shared::cta.mbarrier::complete_tx::bytes.multicast::cluster::all.b128 [%0], [%1];"
+        ::"r"(resp), "r"(bar) : "memory");
+  }
+}
+
+// Reads a response: valid = 1 and the x coordinate of the cancelled cluster's first CTA, or valid = 0 when nothing was
+// left to cancel.  The closing fence orders this read before the next asynchronous write to the same entry.
+__device__ __forceinline__ void clc_decode(uint32_t resp, uint32_t& valid, uint32_t& first_cta_x) {
+  uint32_t v, x;
+  asm volatile(
+      "{\n\t.reg .pred p1;\n\t.reg .b128 r;\n\t.reg .b32 ty, tz;\n\t"
+      "ld.shared.b128 r, [%2];\n\t"
+      "clusterlaunchcontrol.query_cancel.is_canceled.pred.b128 p1, r;\n\t"
+      "selp.u32 %1, 1, 0, p1;\n\t"
+      "mov.u32 %0, 0;\n\t"
+      "@p1 clusterlaunchcontrol.query_cancel.get_first_ctaid.v4.b32.b128 {%0, ty, tz, _}, r;\n\t}"
+      : "=r"(x), "=r"(v)
+      : "r"(resp)
+      : "memory");
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  valid = v;
+  first_cta_x = x;
+}
+
 // Bounded wait for a word in global memory to take the value `want` (written by another CTA with st_release_gpu).
 static __device__ __noinline__ bool flag_wait(const int32_t* flag, int32_t want, int32_t* status, int code,
                                               unsigned long long timeout_ns = kTimeoutNs) {
