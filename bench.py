@@ -33,17 +33,20 @@ L2_BYTES = 126 * 2 ** 20
 # DRAM bytes per launch of the GEMM kernel from the ncu captures summarised under profiles/
 # (dram__bytes_read.sum + dram__bytes_write.sum), keyed by (workload, tile, scheme spec); None = not captured.
 NCU_DRAM_BYTES = {
-    ("cfg3", "256x512", "group_n:8"): 0.952e9,   # profiles/gemm_kernel_cfg3_256x512_group_n8_full.md (mean of 2 launches)
-    ("cfg3", "256x256", "die_split:m:group_m:8:p"): 1.071e9,   # profiles/l2_hit_rate_per_scheme.md
-    ("cfg5", "256x256", "die_split:m:group_m:8:p"): 1.247e9,
-    ("cfg3", "256x256", "group_m:8"): 1.200e9,   # profiles/gemm_kernel_cfg3_group_m8_full.md (mean of 2 launches)
-    ("cfg3", "256x256", "row_major"): 2.341e9,   # profiles/l2_hit_rate_per_scheme.md
-    ("cfg3", "256x256", "group_n:8"): 1.228e9,
-    ("cfg3", "256x256", "hilbert"): 1.237e9,
-    ("cfg5", "256x256", "group_m:16"): 1.599e9,
-    ("cfg5", "256x256", "group_m:8"): 2.325e9,
-    ("cfg4", "256x256", "group_n:8"): 0.543e9,
-    ("cfg2", "128x256", "group_m:8"): 0.085e9,
+    ("cfg3", "256x512", "group_n:8"): 0.956e9,   # profiles/gemm_kernel_cfg3_256x512_group_n8_full.md (mean of 2 launches)
+    ("cfg3", "256x512", "die_split:m:group_m:8:p"): 0.971e9,   # this and the rest: profiles/l2_hit_rate_per_scheme.md
+    ("cfg3", "256x256", "die_split:m:group_m:8:p"): 1.229e9,
+    ("cfg3", "256x256", "group_m:8"): 1.216e9,
+    ("cfg3", "256x256", "row_major"): 2.363e9,
+    ("cfg3", "256x256", "group_n:8"): 1.245e9,
+    ("cfg3", "256x256", "hilbert"): 1.271e9,
+    ("cfg5", "256x512", "die_split:m:group_m:8:p"): 1.647e9,
+    ("cfg5", "256x256", "die_split:m:group_m:8:p"): 1.348e9,
+    ("cfg5", "256x256", "group_m:16"): 1.623e9,
+    ("cfg5", "256x256", "group_m:8"): 2.090e9,
+    ("cfg4", "256x256", "group_n:8"): 0.548e9,
+    ("cfg2", "128x256", "group_m:8"): 0.092e9,
+    ("cfg2", "128x256", "row_major"): 0.084e9,
 }
 
 
@@ -111,7 +114,8 @@ DEFAULT_SCHEME = {"cfg1": "group_m:2", "cfg2": "group_m:8", "cfg3": "die_split:m
 FALLBACK_SCHEME = {"cfg3": "group_m:8", "cfg5": "group_m:16"}   # if the topology probe finds no two-way L2 structure
 # 8192^3 is timed with two 256x256 2-CTA MMA tiles per scheduler tile (they share the A panel: a quarter less operand
 # traffic from L2); the plain 256x256 scheduler tile is timed beside it and reported in the same line.
-DEFAULT_TILE = {"cfg3": "256x512", "cfg2": "256x512"}   # 4096^3: A and B fit in L2, the order hardly matters, the wider tile does
+DEFAULT_TILE = {"cfg3": "256x512", "cfg2": "256x512",   # 4096^3: A and B fit in L2, the order hardly matters, the wider tile does
+                "cfg5": "256x512"}
 DEFAULT_SCHEME_BY_TILE = {("cfg3", "256x512"): "group_n:8", ("cfg5", "256x512"): "die_split:m:group_m:8:p",
                           ("cfg2", "256x512"): "row_major"}
 

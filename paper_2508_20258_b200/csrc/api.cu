@@ -494,6 +494,10 @@ int sp_gemm_host(const void* A_host, const void* B_host, void* C_host, int64_t M
     set_error("sp_params.struct_size is %u, expected %zu", params->struct_size, sizeof(sp_params));
     return SP_ERR_INVALID_ARG;
   }
+  if (params && (params->flags & SP_FLAG_OVERLAP)) {
+    set_error("SP_FLAG_OVERLAP is a statement about device buffers the caller manages; sp_gemm_host orders its own copies and kernels");
+    return SP_ERR_INVALID_ARG;
+  }
   const size_t out_elt = (params && params->out_dtype == 1) ? 4 : 2;
   auto pad = [](size_t b) { return (b + 255) & ~(size_t)255; };
   const size_t a_bytes = (size_t)M * (size_t)K * 2, b_bytes = (size_t)K * (size_t)N * 2, c_bytes = (size_t)M * (size_t)N * out_elt;

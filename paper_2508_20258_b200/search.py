@@ -55,6 +55,10 @@ def default_candidates(units: int) -> List[Tuple[str, int, Dict]]:
             c.append((f"die_split:{an}:group_m:{g}:p", sp.DIE_SPLIT,
                       dict(split_axis=axis, inner_scheme=sp.GROUP_M, inner_group=g, flags=2)))
         c.append((f"die_split:{an}:hilbert:p", sp.DIE_SPLIT, dict(split_axis=axis, inner_scheme=sp.HILBERT, flags=2)))
+    # variants of the schedule under one good order: slots handed out by cluster launch control; last wave split along k
+    # (the latter changes the rounding order of the split tiles, so the loop files it under "wrong" unless C is exact)
+    c.append(("group_m:8+clc", sp.GROUP_M, dict(group=8, flags=sp.FLAG_CLC)))
+    c.append(("group_n:8+clc", sp.GROUP_N, dict(group=8, flags=sp.FLAG_CLC)))
     return c
 
 

@@ -73,4 +73,8 @@ def test_overlap_rejections():
     with pytest.raises(sp.SpError) as e:
         sp.gemm_noalloc(dA, dB, dC, sp.ROW_MAJOR, sp.make_params(tile_m=128, tile_n=128, flags=OV))
     assert e.value.status == sp.ERR_INVALID_ARG
+    with pytest.raises(sp.SpError) as e:
+        sp.gemm_host(A.view(np.int16), B.view(np.int16), np.zeros((512, 512), dtype=np.int16), sp.ROW_MAJOR,
+                     sp.make_params(tile_m=128, tile_n=128, flags=OV))
+    assert e.value.status == sp.ERR_INVALID_ARG
     assert sp.get_status() == 0 and float(dC.float().abs().sum()) == 0.0
