@@ -398,6 +398,18 @@ def run_ours(args) -> int:
         cpu_baseline = {"value": 2.0 * rows * w.N * w.K / dt / 1e12, "unit": "TFLOP/s", "cores": G.threads(),
                         "kind": "oracle", "seconds": dt,
                         "sample": f"first {rows} rows of C ({rows}x{w.N}x{w.K}) of the {w.M}-row product"}
+        # the other half of the oracle: the enumerated remap of this workload's tile grid under the timed order
+        from oracle import remap as OR
+        kw_o = parse_scheme(spec)[1]
+        op = OR.Params(**{k: v for k, v in kw_o.items() if k in OR.Params.__dataclass_fields__})
+        t0 = time.perf_counter()
+        OR.tile_map(w.M, w.N, tile_m, tile_n, scheme, op)
+        cpu_baseline["remap_oracle_ms"] = (time.perf_counter() - t0) * 1e3
+        if w.M * w.N * w.K <= 2 ** 28:                      # small enough to also time on one core (512^3)
+            t0 = time.perf_counter()
+            G.gemm_rows(A, B, np.arange(w.M), nthreads=1)
+            cpu_baseline["single_thread_tflops"] = 2.0 * w.M * w.N * w.K / (time.perf_counter() - t0) / 1e12
+            G.gemm_rows(A, B, np.arange(1), nthreads=cpu_baseline["cores"])    # the thread count is sticky: put it back
 
     if rank == 0:
         line = {
