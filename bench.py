@@ -445,6 +445,16 @@ def run_sweep_sustained(args, sp, w, dA, dB, dC, params_for, flops, stream) -> i
         except sp.SpError as err:
             if err.status != sp.ERR_UNSUPPORTED:
                 raise
+    done = {}
+    if args.resume and os.path.exists(args.resume):     # an interrupted sweep picks up where it stopped
+        for l in open(args.resume):
+            try:
+                j = json.loads(l)
+                if j.get("sweep_sustained") == w.name and j.get("key") == args.resume_key:
+                    done[j["scheme"]] = j
+            except ValueError:
+                pass
+        specs = [s_ for s_ in specs if s_ not in done]
     acc = {spec: [] for spec in specs}
     for _ in range(2):
         for spec in specs:
@@ -457,12 +467,19 @@ def run_sweep_sustained(args, sp, w, dA, dB, dC, params_for, flops, stream) -> i
             acc[spec].append(time_steps(sp, dA, dB, dC, s, p, n, stream) / n)
     assert sp.get_status() == 0
     base = None
+    for j in done.values():
+        print(json.dumps(j), flush=True)
+        base = base or j["ms"]
     for spec in specs:
         ms = sum(acc[spec]) / len(acc[spec])
         if base is None:
             base = ms
-        print(json.dumps({"sweep_sustained": w.name, "scheme": spec, "ms": ms, "tflops": flops / ms / 1e9,
-                          "speedup_vs_first": base / ms, "passes_ms": acc[spec]}), flush=True)
+        line = {"sweep_sustained": w.name, "scheme": spec, "ms": ms, "tflops": flops / ms / 1e9,
+                "speedup_vs_first": base / ms, "passes_ms": acc[spec], "key": args.resume_key}
+        print(json.dumps(line), flush=True)
+        if args.resume:
+            with open(args.resume, "a") as fh:
+                fh.write(json.dumps(line) + "\n")
     return 0
 
 
@@ -697,12 +714,15 @@ def main() -> int:
     ap.add_argument("--alternate", default=None, metavar="SPEC,SPEC[,cublas]",
                     help="time the given schemes in alternating blocks of --steps launches (--rounds rounds, median)")
     ap.add_argument("--rounds", type=int, default=6)
+    ap.add_argument("--resume", default=None, metavar="FILE.jsonl",
+                    help="--sweep-sustained: append each scheme's line to FILE and skip schemes already in it")
     ap.add_argument("--b-layout", default="kn", choices=["kn", "nk"], help="B stored K x N (default) or N x K")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--transpose", default=None, metavar="MxN", help="time sp_transpose on an M x N 16-bit matrix instead")
     ap.add_argument("--stencil", default=None, metavar="MxN", help="time sp_stencil2d on an M x N fp32 grid instead")
     args = ap.parse_args()
+    args.resume_key = f"{args.workload}|{args.shape}|{args.tile}|{args.b_layout}"
     if args.transpose:
         return run_transpose(args)
     if args.stencil:

@@ -172,7 +172,9 @@ int sp_tile_map_device(int64_t M, int64_t N, int32_t tileM, int32_t tileN, int s
  * issue only the kernel launch (plus one small memset node with SP_FLAG_DIE_PINNED), so after one warm-up call per
  * (shape, scheme, params) further calls can be recorded into a CUDA graph by stream capture and replayed; the
  * pointers and the order are then those of the recording.
- * A device-side wait that expires is reported by sp_get_status, not here. */
+ * A device-side wait that expires is reported by sp_get_status, not here.
+ * With the environment variable SP_LOG set, every launch writes one line to stderr (shape, tile, variant, grid, pipeline
+ * depth, flags in effect); nothing is ever written to stdout. */
 int sp_gemm(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t K, int scheme,
             const sp_params* params, void* stream);
 

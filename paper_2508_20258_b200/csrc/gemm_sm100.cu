@@ -903,6 +903,15 @@ int launch_gemm(const GemmCall& call) {
     }
   }
 
+  if (getenv("SP_LOG")) {   // diagnostics on request: which variant runs, and how
+    const int stages = cg == 1 ? (call.tile_n == 128 ? Cfg<1, 128>::kStages : Cfg<1, 256>::kStages)
+                               : (call.tile_n == 128 ? Cfg<2, 128>::kStages : call.tile_n == 256 ? Cfg<2, 256>::kStages : Cfg<2, 512>::kStages);
+    fprintf(stderr, "[swizzleperf] gemm %dx%dx%d tile %dx%d (%d CTA%s per tile) scheme %d T=%d units=%d grid=%d stages=%d kblocks=%d "
+                    "b=%s out=%s table=%d pinned=%d split_tail=%d/%d clc=%d overlap=%d\n",
+            args.M, args.N, args.K, call.tile_m, call.tile_n, cg, cg > 1 ? "s" : "", call.sched.scheme, call.sched.T, args.units,
+            (args.clc ? call.sched.T : args.units) * cg, stages, args.kblocks, call.b_nk ? "NxK" : "KxN", call.out_f32 ? "fp32" : "bf16",
+            call.sched.use_table, args.pinned, args.sk.tiles, args.sk.units, args.clc, args.overlap);
+  }
   if (cg == 1) return call.tile_n == 128 ? launch_shape<1, 128>(call, tmA, tmB, tmC, args) : launch_shape<1, 256>(call, tmA, tmB, tmC, args);
   if (call.tile_n == 512) return launch_shape<2, 512>(call, tmA, tmB, tmC, args);
   return call.tile_n == 128 ? launch_shape<2, 128>(call, tmA, tmB, tmC, args) : launch_shape<2, 256>(call, tmA, tmB, tmC, args);
