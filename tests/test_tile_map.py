@@ -137,3 +137,28 @@ def test_die_pinned_rank_assignment_covers_every_rank_under_any_placement():
         for arrivals0 in range(0, n0 + n1 + 1):
             assert L.sp_selftest_pinned_tickets(n0, n1, arrivals0) == sp.OK, (n0, n1, arrivals0)
     assert L.sp_selftest_pinned_tickets(2, 2, 5) == sp.ERR_INVALID_ARG
+
+
+def test_largest_accepted_grids():
+    """The documented limits: 2^24 tiles, curve orders up to 4096 tiles per side.  At the limit the maps are still
+    bijections (checked with numpy; the enumerating oracle would take minutes), one tile beyond is refused."""
+    T = 1 << 24
+    for scheme, kw in [(sp.ROW_MAJOR, {}), (sp.GROUP_M, dict(group=5)), (sp.GROUP_N, dict(group=7)),
+                       (sp.XCD, dict(num_xcds=8, wave=148, xcd_balanced=1)),
+                       (sp.DIE_SPLIT, dict(split_axis=1, inner_scheme=sp.GROUP_M, inner_group=3, interleave=1))]:
+        perm = np.asarray(sp.tile_map(4096, 4096, 1, 1, scheme, sp.make_params(**kw)))
+        assert perm.shape == (T,)
+        seen = np.zeros(T, dtype=bool)
+        seen[perm] = True
+        assert seen.all(), scheme
+    h = np.asarray(sp.tile_map(4096, 4096, 1, 1, sp.HILBERT))
+    tm, tn = np.divmod(h, 4096)
+    assert (np.abs(np.diff(tm)) + np.abs(np.diff(tn)) == 1).all()          # a Hilbert walk moves one cell at a time
+    assert h[0] == 0 and np.array_equal(np.sort(h), np.arange(T))
+    with pytest.raises(sp.SpError) as e:
+        sp.tile_map(4097, 4096, 1, 1, sp.ROW_MAJOR)
+    assert e.value.status == sp.ERR_INVALID_ARG
+    with pytest.raises(sp.SpError) as e:
+        sp.tile_map(4097, 8, 1, 1, sp.HILBERT)
+    assert e.value.status == sp.ERR_UNSUPPORTED
+    assert sp.tile_count(1 << 40, 1 << 40, 1 << 30, 1 << 30) == 1 << 20
