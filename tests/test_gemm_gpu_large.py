@@ -112,3 +112,25 @@ def test_large_workload_sampled(name, tile, schemes):
             del Cf
         else:
             assert np.array_equal(bits, first_bits)      # same bits under every order
+
+
+def test_output_larger_than_4_gib_is_addressed_correctly():
+    """C of 49152 x 49152 bf16 is 4.8 GB: byte offsets beyond 2^32.  K is one k-block, so the product is cheap and the
+    oracle can check whole rows, among them the last ones."""
+    M = N = 49152
+    K = 64
+    A, B = synth.make_int_inputs(M, N, K, seed=77)
+    dA, dB = dev_bf16(A), dev_bf16(B)
+    dC = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    rows = [0, 1, 255, 256, 21845, 32767, 32768, 43690, 43691, M - 257, M - 2, M - 1]   # byte offsets up to 4.83e9
+    ref, _ = G.gemm_rows(A, B, rows)
+    want = G.bf16_bits_to_f64(synth.f32_to_bf16_bits(ref.astype(np.float32)))           # small integers: exact, then RNE
+    for scheme, kw, tile in [(sp.HILBERT, {}, (256, 512)), (sp.GROUP_M, dict(group=8), (256, 256)),
+                             (sp.ROW_MAJOR, dict(flags=sp.FLAG_CLC), (128, 256))]:
+        dC.fill_(float("nan"))
+        sp.gemm(dA, dB, dC, scheme, sp.make_params(tile_m=tile[0], tile_n=tile[1], **kw))
+        assert sp.get_status() == 0
+        got = G.bf16_bits_to_f64(dC[rows].view(torch.int16).cpu().numpy().view(np.uint16))
+        assert np.array_equal(got, want), (scheme, tile)
+        assert not bool(torch.isnan(dC[:, N - 1].float()).any()) and not bool(torch.isnan(dC[M - 1].float()).any())
+        assert not bool(torch.isnan(dC[::997].float()).any())

@@ -109,3 +109,18 @@ def test_stencil_rejections():
     assert L.sp_stencil2d(xw.data_ptr(), torch.zeros_like(xw).data_ptr(), 640, 128, 1.0, 0.0, sp.XCD, ctypes.byref(bad),
                           None) == sp.ERR_NOT_BIJECTIVE
     assert sp.get_status() == 0
+
+
+def test_grid_larger_than_4_gib_is_addressed_correctly():
+    M, N = 36864, 32768                                # 4.8 GB per fp32 grid: byte offsets beyond 2^32
+    g = torch.Generator(device="cuda").manual_seed(5)
+    dx = torch.randint(-8, 9, (M, N), device="cuda", generator=g, dtype=torch.int32).float()
+    out = torch.full_like(dx, float("nan"))
+    sp.stencil2d(dx, out, 0.5, 0.125, sp.HILBERT)
+    assert sp.get_status() == 0
+    for i in [0, 1, 63, 64, 16383, 16384, 32767, 32768, 32769, M - 65, M - 2, M - 1]:
+        lo, hi = max(i - 1, 0), min(i + 2, M)
+        x = dx[lo:hi].cpu().numpy()
+        ref = S.stencil2d(x, 0.5, 0.125)[i - lo] if 0 < i < M - 1 else x[i - lo].astype(np.float64)
+        assert np.array_equal(out[i].cpu().numpy().astype(np.float64), ref), i      # dyadic weights, small integers: exact
+    assert not bool(torch.isnan(out[:, N - 1]).any()) and not bool(torch.isnan(out[::1013]).any())

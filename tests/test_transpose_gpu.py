@@ -52,3 +52,16 @@ def test_transpose_rejections():
     assert L.sp_transpose(None, b.data_ptr(), 64, 64, sp.ROW_MAJOR, None, None) == sp.ERR_INVALID_ARG
     p = sp.make_params(num_xcds=8)          # 5 x 2 tiles, 8 chiplets: printed formula leaves the range
     assert L.sp_transpose(a.data_ptr(), b.data_ptr(), 320, 128, sp.XCD, ctypes.byref(p), None) == sp.ERR_NOT_BIJECTIVE
+
+
+def test_matrix_larger_than_4_gib_is_addressed_correctly():
+    M, N = 40960, 61440                                # 5 GB of 16-bit elements: byte offsets beyond 2^32
+    g = torch.Generator(device="cuda").manual_seed(9)
+    x = torch.randint(-32768, 32768, (M, N), device="cuda", generator=g, dtype=torch.int16)
+    out = torch.zeros((N, M), dtype=torch.int16, device="cuda")
+    sp.transpose(x, out, sp.DIE_SPLIT, sp.make_params(split_axis=0, inner_scheme=sp.HILBERT, interleave=1))
+    assert sp.get_status() == 0
+    for j in [0, 1, 63, 64, 30719, 30720, N - 65, N - 1]:            # rows of the output = columns of the input
+        assert torch.equal(out[j], x[:, j]), j
+    for i in [0, 4095, 20480, M - 1]:
+        assert torch.equal(out[:, i], x[i]), i
