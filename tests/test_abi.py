@@ -53,3 +53,20 @@ def test_gemm_rejects_bad_arguments_before_touching_a_device():
     assert sp.last_error() != ""
     smid = np.zeros(4, dtype=np.int32)
     assert L.sp_probe_dispatch(3, 2, smid.ctypes.data, smid.ctypes.data) == sp.ERR_INVALID_ARG
+
+
+def test_stencil_and_transpose_reject_bad_arguments_before_touching_a_device():
+    L = sp.lib()
+    a, b = 0x1000, 0x200000
+    assert L.sp_stencil2d(a, b, 64, 126, 1.0, 0.0, sp.ROW_MAJOR, None, None) == sp.ERR_ALIGNMENT
+    assert L.sp_stencil2d(a + 4, b, 64, 128, 1.0, 0.0, sp.ROW_MAJOR, None, None) == sp.ERR_ALIGNMENT
+    assert L.sp_stencil2d(a, a, 64, 128, 1.0, 0.0, sp.ROW_MAJOR, None, None) == sp.ERR_INVALID_ARG
+    assert L.sp_stencil2d(None, b, 64, 128, 1.0, 0.0, sp.ROW_MAJOR, None, None) == sp.ERR_INVALID_ARG
+    assert L.sp_stencil2d(a, b, -1, 128, 1.0, 0.0, sp.ROW_MAJOR, None, None) == sp.ERR_INVALID_ARG
+    assert L.sp_stencil2d(a, b, 64, 128, 1.0, float("nan"), sp.ROW_MAJOR, None, None) == sp.ERR_INVALID_ARG
+    bad = sp.make_params(num_xcds=4, xcd_balanced=0)      # 10 tiles: the printed formula with X = 4 leaves [0, 10)
+    assert L.sp_stencil2d(a, b, 640, 128, 1.0, 0.0, sp.XCD, ctypes.byref(bad), None) == sp.ERR_NOT_BIJECTIVE
+    assert L.sp_transpose(a, b, 64, 60, sp.ROW_MAJOR, None, None) == sp.ERR_ALIGNMENT
+    assert L.sp_transpose(a, a, 64, 64, sp.ROW_MAJOR, None, None) == sp.ERR_INVALID_ARG
+    first = ctypes.c_int32(0)
+    assert L.sp_streamk_plan(16, 4, 8, ctypes.byref(first), None) == sp.ERR_INVALID_ARG
