@@ -162,3 +162,50 @@ def test_largest_accepted_grids():
         sp.tile_map(4097, 8, 1, 1, sp.HILBERT)
     assert e.value.status == sp.ERR_UNSUPPORTED
     assert sp.tile_count(1 << 40, 1 << 40, 1 << 30, 1 << 30) == 1 << 20
+
+
+def test_the_papers_other_printed_remaps_meet_the_gate_as_caller_tables():
+    """The appendix prints a remap for each of its other kernels (with eight chiplets).  Restated here as functions of
+    the linear block id and handed to the library as SP_CUSTOM tables: the gate must accept exactly those that are
+    permutations, which is what the paper's loop needs from it (a broken remap is a failed attempt, not a launch)."""
+    X = 8
+
+    def chunked(p, n):            # layer-norm / softmax figures: chiplet from (p div X) mod X, position p mod X
+        return ((p // X) % X) * (-(-n // X)) + p % X
+
+    def floor_form(p, n):         # the hardware-aware transpose figure: the GEMM formula with floor for ceil
+        return p // X + (p % X) * (n // X)
+
+    def strided(p, n):            # the transpose figure: chiplet from (p div X) mod X, then p div X
+        return ((p // X) % X) * (n // X) + p // X
+
+    def collapsed(p, n, rows):    # the stencil figure: a whole chunk of `rows` ids lands on one id
+        return (p // (X * rows)) * X + (p // rows) % X
+
+    def gate(table, T):
+        seen = np.zeros(T, dtype=bool)
+        ok = all(0 <= t < T for t in table)
+        if ok:
+            seen[np.asarray(table)] = True
+        want = ok and bool(seen.all())
+        try:
+            got = list(sp.tile_map(T, 1, 1, 1, sp.CUSTOM, sp.make_params(custom_perm=list(table))))
+            assert got == list(table)
+            accepted = True
+        except sp.SpError as e:
+            assert e.status == sp.ERR_NOT_BIJECTIVE
+            accepted = False
+        assert accepted == want
+        return accepted
+
+    assert gate([chunked(p, 64) for p in range(64)], 64)                  # 64 blocks: the identity
+    assert not gate([chunked(p, 128) for p in range(128)], 128)           # beyond 64 blocks ids repeat (p and p + 64)
+    assert not gate([chunked(p, 40) for p in range(40)], 40)
+    for n in (64, 128, 1024):
+        assert gate([floor_form(p, n) for p in range(n)], n)              # X divides n: a transposition of the id space
+    for n in (20, 100, 148):
+        assert not gate([floor_form(p, n) for p in range(n)], n)          # it does not: ids collide
+    for n in (64, 256):
+        assert not gate([strided(p, n) for p in range(n)], n)             # both terms depend on p div X only: X ids share a target
+    assert not gate([collapsed(p, 64, 4) for p in range(64)], 64)         # four ids per target
+    assert gate([collapsed(p, 64, 1) for p in range(64)], 64)             # one row per chunk: the identity
