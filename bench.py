@@ -205,6 +205,11 @@ def run_ours(args) -> int:
         SWEEPS[w.name] = ["row_major", "group_m:4", "group_m:8", "group_m:16", "hilbert", "die_split:m:group_m:8:p"]
         DEFAULT_SCHEME[w.name] = "group_m:8"
         args.workload = w.name
+        if not (args.tile or args.scheme or args.sweep or args.sweep_sustained or args.profile_sweep or args.alternate):
+            rs, rp = sp.recommend(Ms, Ns, Ks, 0, b_nk)      # nothing asked for: the library's own suggestion for the shape
+            args.tile = f"{rp.tile_m}x{rp.tile_n}"
+            args.scheme = {sp.ROW_MAJOR: "row_major", sp.COL_MAJOR: "col_major", sp.GROUP_M: f"group_m:{rp.group}",
+                           sp.GROUP_N: f"group_n:{rp.group}"}[rs]
     else:
         w = synth.WORKLOADS[args.workload]
         _, A, B = synth.make_workload(args.workload, b_is_nk=bool(b_nk))

@@ -249,6 +249,19 @@ int sp_transpose(const void* in, void* out, int64_t M, int64_t N, int scheme, co
 int sp_stencil2d(const void* in, void* out, int64_t M, int64_t N, float c_center, float c_neighbor, int scheme,
                  const sp_params* params, void* stream);
 
+/* A starting configuration for sp_gemm on this hardware: tile shape, order and its parameters for a given problem.
+ * The paper arrives at a remap by searching with measurements in the loop; this is the short table that this
+ * library's own sweeps on B200 distil to (no counterpart in the paper, and no substitute for measuring: the search
+ * loop of the Python package does that).  Rule: among the supported tiles, the one with the least estimated time
+ * waves x tile area / (CTAs per tile x relative efficiency of the tile shape), waves = ceil(T / units), units = 74 CTA
+ * pairs or 148 CTAs; row-major when A and B together are at most 64 MiB (they stay in L2) or the tile grid is at most
+ * ten tiles wide, column-major when it is at most ten tiles tall, else bands of 8 tile columns (256x512 tile) or 8
+ * tile rows (other tiles).  Host only; no GPU needed.
+ *   params : HOST, receives a complete sp_params (struct_size, tile_m, tile_n, group, out_dtype, b_layout set; the
+ *            rest zero).   scheme : HOST, receives the sp_scheme.
+ * Errors: SP_ERR_INVALID_ARG (NULL, sizes <= 0, bad out_dtype / b_layout). */
+int sp_recommend(int64_t M, int64_t N, int64_t K, int32_t out_dtype, int32_t b_layout, sp_params* params, int* scheme);
+
 /* Number of persistent CTAs (tile 128xN) or CTA pairs (tile 256xN) sp_gemm launches for T tiles;
  * slot s is run by unit s % units in round s / units.  Returns -1 on error. */
 int sp_gemm_units(int32_t tile_m, int32_t tile_n, int64_t T);

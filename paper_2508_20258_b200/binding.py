@@ -57,7 +57,7 @@ TRACE_DTYPE = np.dtype([("slot", "<i4"), ("tile", "<i4"), ("smid", "<i4"), ("uni
                         ("mma_wait_acc", "<u4"), ("load_wait_stage", "<u4"), ("epi_wait_acc", "<u4")])
 
 EXPORTS = ["sp_tile_count", "sp_tile_map", "sp_tile_map_device", "sp_gemm", "sp_gemm_trace", "sp_gemm_host",
-           "sp_gemm_noalloc", "sp_transpose", "sp_stencil2d", "sp_gemm_units", "sp_streamk_plan",
+           "sp_gemm_noalloc", "sp_transpose", "sp_stencil2d", "sp_gemm_units", "sp_streamk_plan", "sp_recommend",
            "sp_probe_dispatch", "sp_probe_topology", "sp_probe_l2_capacity", "sp_selftest_timeout", "sp_selftest_pinned_tickets", "sp_get_status", "sp_last_error", "sp_shutdown"]
 
 
@@ -99,6 +99,8 @@ def lib() -> ctypes.CDLL:
         L.sp_stencil2d.argtypes = [vp, vp, i64, i64, ctypes.c_float, ctypes.c_float, ctypes.c_int, pp, vp]
         L.sp_gemm_units.restype = ctypes.c_int
         L.sp_gemm_units.argtypes = [i32, i32, i64]
+        L.sp_recommend.restype = ctypes.c_int
+        L.sp_recommend.argtypes = [i64, i64, i64, i32, i32, pp, ctypes.POINTER(ctypes.c_int)]
         L.sp_streamk_plan.restype = ctypes.c_int
         L.sp_streamk_plan.argtypes = [i64, i32, i32, ctypes.POINTER(ctypes.c_int32), vp]
         L.sp_probe_dispatch.restype = ctypes.c_int
@@ -291,6 +293,14 @@ def gemm_units(tile_m: int, tile_n: int, T: int) -> int:
 FLAG_DIE_PINNED, FLAG_SERPENTINE, FLAG_STREAM_K, FLAG_OVERLAP, FLAG_CLC = 2, 4, 8, 16, 32
 STREAMK_MAX_SEGMENTS = 8
 WORK_FULL, WORK_CONTRIB, WORK_OWNER = 0, 1, 2
+
+
+def recommend(M: int, N: int, K: int, out_dtype: int = 0, b_layout: int = 0):
+    """(scheme, params) the library suggests for this problem on B200: a table distilled from its own sweeps."""
+    p = SpParams()
+    scheme = ctypes.c_int(0)
+    _check(lib().sp_recommend(M, N, K, out_dtype, b_layout, ctypes.byref(p), ctypes.byref(scheme)))
+    return int(scheme.value), p
 
 
 def streamk_plan(T: int, units: int, kblocks: int):

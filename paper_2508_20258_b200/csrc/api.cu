@@ -639,6 +639,43 @@ int sp_stencil2d(const void* in, void* out, int64_t M, int64_t N, float c_center
   return launch_stencil(in, out, M, N, c_center, c_neighbor, sched, perm_dev, ds->status, (cudaStream_t)stream);
 }
 
+int sp_recommend(int64_t M, int64_t N, int64_t K, int32_t out_dtype, int32_t b_layout, sp_params* params, int* scheme) {
+  if (!params || !scheme) { set_error("params and scheme must not be NULL"); return SP_ERR_INVALID_ARG; }
+  if (M <= 0 || N <= 0 || K <= 0) { set_error("M, N, K must be positive"); return SP_ERR_INVALID_ARG; }
+  if ((out_dtype != 0 && out_dtype != 1) || (b_layout != 0 && b_layout != 1)) { set_error("bad out_dtype / b_layout"); return SP_ERR_INVALID_ARG; }
+  // relative throughput of the tile shapes at equal work, from the sustained sweeps at 4096^3 and 8192^3
+  static const struct { int tm, tn; double eff; } kTiles[] = {
+      {256, 512, 1.00}, {256, 256, 0.97}, {128, 256, 0.89}, {256, 128, 0.75}, {128, 128, 0.67}};
+  int best = 0;
+  double best_cost = 0;
+  for (int i = 0; i < 5; ++i) {
+    const int64_t T = ((M + kTiles[i].tm - 1) / kTiles[i].tm) * ((N + kTiles[i].tn - 1) / kTiles[i].tn);
+    const int cg = kTiles[i].tm / 128, units = 148 / cg;
+    const double waves = (double)((T + units - 1) / units);
+    const double cost = waves * kTiles[i].tm * kTiles[i].tn / (cg * kTiles[i].eff);
+    if (i == 0 || cost < best_cost) { best = i; best_cost = cost; }   // ties keep the larger tile (listed first)
+  }
+  memset(params, 0, sizeof *params);
+  params->struct_size = sizeof(sp_params);
+  params->tile_m = kTiles[best].tm; params->tile_n = kTiles[best].tn;
+  params->out_dtype = out_dtype; params->b_layout = b_layout;
+  params->group = 1;
+  // Order: a wave of U tiles should cover a block of C that is about as tall as it is wide, so that it needs the
+  // fewest rows of A and columns of B.  When the operands fit in L2 anyway, or the grid is at most ten tiles wide
+  // (tall), plain row-major (column-major) already does that; else bands of eight.
+  const double operands = 2.0 * ((double)M * (double)K + (double)K * (double)N);
+  const int64_t Tm = (M + params->tile_m - 1) / params->tile_m, Tn = (N + params->tile_n - 1) / params->tile_n;
+  if (operands <= 64.0 * 1048576.0 || Tn <= 10) {
+    *scheme = SP_ROW_MAJOR;
+  } else if (Tm <= 10) {
+    *scheme = SP_COL_MAJOR;
+  } else {
+    *scheme = params->tile_n == 512 ? SP_GROUP_N : SP_GROUP_M;
+    params->group = 8;
+  }
+  return SP_OK;
+}
+
 int sp_gemm_units(int32_t tile_m, int32_t tile_n, int64_t T) {
   int dev = 0;
   if (current_device(&dev) != SP_OK) return -1;

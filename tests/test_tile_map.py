@@ -209,3 +209,27 @@ def test_the_papers_other_printed_remaps_meet_the_gate_as_caller_tables():
         assert not gate([strided(p, n) for p in range(n)], n)             # both terms depend on p div X only: X ids share a target
     assert not gate([collapsed(p, 64, 4) for p in range(64)], 64)         # four ids per target
     assert gate([collapsed(p, 64, 1) for p in range(64)], 64)             # one row per chunk: the identity
+
+
+def test_recommendation_is_valid_and_matches_what_the_sweeps_found():
+    found = {  # (M, N, K) -> (tile, scheme, group): the fastest (or within noise of it) in this repository's sweeps on B200
+        (4096, 4096, 4096): ((256, 512), sp.ROW_MAJOR, 1),
+        (8192, 8192, 8192): ((256, 512), sp.GROUP_N, 8),
+        (16384, 2048, 8192): ((256, 256), sp.ROW_MAJOR, 1),
+        (16384, 16384, 4096): ((256, 512), sp.GROUP_N, 8),
+        (2048, 2048, 2048): ((256, 256), sp.ROW_MAJOR, 1),
+    }
+    for (M, N, K), (tile, scheme, group) in found.items():
+        s, p = sp.recommend(M, N, K)
+        assert (p.tile_m, p.tile_n) == tile and s == scheme and p.group == group, (M, N, K)
+    rng = np.random.default_rng(0)
+    for _ in range(200):                                  # always a supported tile and a bijective order
+        M, N, K = (int(rng.integers(1, 40000)), int(rng.integers(1, 5000)) * 8, int(rng.integers(1, 3000)) * 8)
+        s, p = sp.recommend(M, N, K, out_dtype=int(rng.integers(2)), b_layout=int(rng.integers(2)))
+        assert (p.tile_m, p.tile_n) in [(128, 128), (128, 256), (256, 128), (256, 256), (256, 512)]
+        perm = np.asarray(sp.tile_map(M, N, p.tile_m, p.tile_n, s, p))
+        assert np.array_equal(np.sort(perm), np.arange(len(perm)))
+    with pytest.raises(sp.SpError):
+        sp.recommend(0, 8, 8)
+    with pytest.raises(sp.SpError):
+        sp.recommend(8, 8, 8, out_dtype=3)
