@@ -118,14 +118,16 @@ def gemm_block(A: np.ndarray, B: np.ndarray, r0: int, r1: int, c0: int, c1: int,
 PHI = 2.0 ** -10
 
 
-def compare(got: np.ndarray, ref: np.ndarray, S: np.ndarray, phi: float = PHI) -> Dict[str, float]:
+def compare(got: np.ndarray, ref: np.ndarray, S: np.ndarray, phi: float = PHI, K: int = 0, bf16_out: bool = True) -> Dict[str, float]:
     """Element-wise error of a GPU result against the oracle.
 
     err_ij = |got - ref| / max(|ref|, phi * S).  With zero-mean inputs a few outputs
     cancel to |ref| far below the rounding noise of ANY fp32 accumulation (which scales
     with S, not with ref), so the relative error is floored at phi * S; a dropped term
     or k-block is still orders of magnitude above 1e-2 * phi * S.
-    Returns the gated figure (``max_err``) and diagnostics.
+    Returns the gated figure (``max_err``) and diagnostics.  With ``K`` given, also counts (never gates) the elements
+    outside the strict tier |got - ref| <= 2^-8 |ref| + 2 K 2^-24 S for bf16 output (half an ulp of the rounding to
+    bf16 plus a worst-case fp32 accumulation) or <= 2 K 2^-24 S for fp32 output: ``strict_violations``.
     """
     got = np.asarray(got, dtype=np.float64)
     diff = np.abs(got - ref)
@@ -135,7 +137,12 @@ def compare(got: np.ndarray, ref: np.ndarray, S: np.ndarray, phi: float = PHI) -
     err = diff / den
     unfloored = np.abs(ref) >= floor
     fro = float(np.sqrt((diff ** 2).sum()) / max(np.sqrt((ref ** 2).sum()), 1e-300))
+    strict = None
+    if K > 0:
+        bound = 2.0 * K * 2.0 ** -24 * S + (2.0 ** -8 * np.abs(ref) if bf16_out else 0.0)
+        strict = int((diff > bound).sum())
     return {
+        "strict_violations": strict,
         "max_err": float(err.max()) if err.size else 0.0,
         "max_err_unfloored": float(err[unfloored].max()) if unfloored.any() else 0.0,
         "n_floored": int((~unfloored).sum()),

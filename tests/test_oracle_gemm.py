@@ -120,3 +120,21 @@ def test_input_recipe_is_deterministic_and_a_is_drawn_first():
     assert vals.min() >= -1.0 and vals.max() <= 1.0
     w = synth.WORKLOADS["cfg5"]
     assert (w.M, w.N, w.K, w.std, w.seed) == (16384, 16384, 4096, 0.5, 4)
+
+
+def test_strict_tier_is_a_diagnostic_that_honest_rounding_passes_and_a_dropped_term_fails():
+    rng = np.random.default_rng(11)
+    M, N, K = 24, 40, 512
+    a = rng.standard_normal((M, K)).astype(np.float32)
+    b = rng.standard_normal((K, N)).astype(np.float32)
+    A = (a.view(np.uint32) >> 16).astype(np.uint16)              # truncation to bf16 bits: any bf16 values will do
+    B = (b.view(np.uint32) >> 16).astype(np.uint16)
+    ref, S = G.gemm_full(A, B)
+    honest = G.bf16_bits_to_f64(((ref.astype(np.float32).view(np.uint32) + 0x8000) >> 16).astype(np.uint16))
+    r = G.compare(honest, ref, S, K=K)
+    assert r["strict_violations"] == 0 and r["max_err"] <= 1e-2
+    broken = honest.copy()
+    broken[3, 5] -= G.bf16_bits_to_f64(A[3:4, 7:8])[0, 0] * G.bf16_bits_to_f64(B[7:8, 5:6])[0, 0] + 0.5
+    assert G.compare(broken, ref, S, K=K)["strict_violations"] >= 1
+    assert G.compare(ref, ref, S, K=K, bf16_out=False)["strict_violations"] == 0
+    assert G.compare(ref, ref, S)["strict_violations"] is None
