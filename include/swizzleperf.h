@@ -169,7 +169,7 @@ int sp_tile_map_device(int64_t M, int64_t N, int32_t tileM, int32_t tileN, int s
  * Errors (all detected on the host, nothing launched): as sp_tile_map, plus SP_ERR_ALIGNMENT (A, B or C not
  * 16-byte aligned; K or N not a multiple of 8), SP_ERR_UNSUPPORTED (tile shape), SP_ERR_DEVICE, SP_ERR_CUDA.
  * The first call for a given (grid, scheme) may allocate a cached tile table; later calls allocate nothing and
- * issue only the kernel launch (plus one small memset node with SP_FLAG_DIE_PINNED), so after one warm-up call per
+ * issue only the kernel launch, so after one warm-up call per
  * (shape, scheme, params) further calls can be recorded into a CUDA graph by stream capture and replayed; the
  * pointers and the order are then those of the recording.
  * A device-side wait that expires is reported by sp_get_status, not here.

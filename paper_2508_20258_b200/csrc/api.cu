@@ -223,9 +223,10 @@ static int current_device(int* dev) {
 
 static int get_status_word(DeviceState* ds) {
   if (!ds->status) {
-    // status word, then kDiePairs pairs of arrival counters handed to die-pinned launches in rotation
-    SP_CUDA(cudaMalloc(&ds->status, (2 + 2 * kDiePairs) * sizeof(int32_t)));
-    SP_CUDA(cudaMemset(ds->status, 0, (2 + 2 * kDiePairs) * sizeof(int32_t)));
+    // status word, then kDiePairs counter sets (arrivals on half 0, arrivals on half 1, units finished) handed to
+    // die-pinned launches in rotation; the last unit of a launch to finish puts its set back to zero
+    SP_CUDA(cudaMalloc(&ds->status, (2 + 3 * kDiePairs) * sizeof(int32_t)));
+    SP_CUDA(cudaMemset(ds->status, 0, (2 + 3 * kDiePairs) * sizeof(int32_t)));
   }
   return SP_OK;
 }
@@ -364,7 +365,7 @@ static int gemm_common(const void* A, const void* B, void* C, int64_t M, int64_t
     rc = get_die_map(ds);
     if (rc != SP_OK) return rc;
     call.pinned = 1;
-    call.die_count_dev = ds->status + 2 + 2 * (int)(ds->die_pair_next++ % kDiePairs);
+    call.die_count_dev = ds->status + 2 + 3 * (int)(ds->die_pair_next++ % kDiePairs);
     call.half0 = die_split_half0(call.sched);
     call.sms_on_die[0] = ds->sms_on_die[0]; call.sms_on_die[1] = ds->sms_on_die[1];
     for (int i = 0; i < 8; ++i) call.die_mask[i] = ds->die_mask[i];
@@ -756,7 +757,8 @@ int sp_get_status(void* stream, int32_t* detail) {
   int32_t word = 0;
   if (ds->status) {
     SP_CUDA(cudaMemcpy(&word, ds->status, sizeof word, cudaMemcpyDeviceToHost));
-    if (word != 0) SP_CUDA(cudaMemset(ds->status, 0, sizeof word));
+    // after an expired wait a die-pinned launch may have left its counters behind: everything back to zero
+    if (word != 0) SP_CUDA(cudaMemset(ds->status, 0, (2 + 3 * kDiePairs) * sizeof(int32_t)));
   }
   if (detail) *detail = word;
   if (word != 0) { set_error("a device-side wait expired (status word 0x%x)", word); return SP_ERR_TIMEOUT; }

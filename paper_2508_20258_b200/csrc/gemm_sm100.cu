@@ -71,7 +71,7 @@ struct GemmArgs {
   int pinned;                      // 0: slot s runs on unit s % units
   int half0;                       // number of slots in half 0 (queue boundary)
   int units_on_die[2];             // persistent units per die (all SMs host one CTA each)
-  int32_t* die_count;              // two device counters, zero at launch: arrival rank of a unit on its die
+  int32_t* die_count;              // three device counters, zero at launch: arrivals on half 0, on half 1, units finished
   uint32_t die_mask[8];            // bit smid = die of that SM (from the topology probe)
   // Stream-K tail (SP_FLAG_STREAM_K): the last sk.tiles slots are split along k over sk.units units.
   SkPlan sk;
@@ -656,6 +656,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   tcgen05_fence_before();
   unit_sync<CG>();
   if (warp == 1) tmem_dealloc<CG>(tmem_base, kTmemCols);
+  if (args.pinned && rank == 0 && threadIdx.x == 0) {
+    // every unit took its rank at start-up; the last one to get here hands the counters back at zero, so the next
+    // launch that is given this set needs no clearing in between (and keeps its place right behind this kernel)
+    __threadfence();
+    if (atomicAdd(args.die_count + 2, 1) == args.units - 1) {
+      args.die_count[0] = 0; args.die_count[1] = 0; args.die_count[2] = 0;
+      __threadfence();
+    }
+  }
   // An overlapped launch never waited for its predecessor; it must still not COMPLETE before it, or whatever follows
   // on the stream (a copy of the predecessor's C, an event) could run too early.  One thread holds the CTA's exit
   // until the predecessor grid has completed and its writes are visible; by now that is almost always the case.
@@ -877,8 +886,6 @@ int launch_gemm(const GemmCall& call) {
     // (the same rule that covers uneven placement), so both halves finish together.
     args.units_on_die[0] = (args.units + 1) / 2;
     args.units_on_die[1] = args.units / 2;
-    cudaError_t ce = cudaMemsetAsync(args.die_count, 0, 2 * sizeof(int32_t), call.stream);
-    if (ce != cudaSuccess) { set_error("clearing the die counters failed: %s", cudaGetErrorString(ce)); return SP_ERR_CUDA; }
   }
   args.sched = call.sched;
   args.sk = SkPlan{0, args.units, call.sched.T};   // no tail: every slot is a whole tile

@@ -59,7 +59,7 @@ struct GemmCall {
   Sched sched;
   const int32_t* perm_dev;  // table for non-arithmetic schemes, else nullptr
   int32_t* status_dev;      // device status word
-  int32_t* die_count_dev;   // die-pinned launches: a pair of device counters nobody else uses while this launch runs
+  int32_t* die_count_dev;   // die-pinned launches: a set of three device counters nobody else uses while this launch runs
   int pinned;               // die-pinned scheduling (SP_DIE_SPLIT + SP_FLAG_DIE_PINNED)
   int half0;                // slots in half 0
   int sms_on_die[2];
