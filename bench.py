@@ -79,6 +79,8 @@ def parse_scheme(spec: str):
         return sp.MORTON, {}
     if name == "hilbert":
         return sp.HILBERT, {}
+    if name == "hilbert_rect":
+        return sp.HILBERT_RECT, {}
     if name == "xcd":      # xcd:X[:W]  (balanced form)
         return sp.XCD, dict(num_xcds=int(a[1]), wave=int(a[2]) if len(a) > 2 else 0, xcd_balanced=1)
     if name == "die_split":  # die_split:{m|n}:inner[:G][:i][:p][:s]

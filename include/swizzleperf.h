@@ -55,7 +55,11 @@ typedef enum {
   SP_DIE_SPLIT = 7, /* tile space cut in two halves along split_axis (half 0 gets the ceil), each half a    */
                     /*   grid of its own ordered by inner_scheme; perm = half 0 then half 1, or alternating */
                     /*   (slot parity = half, the paper's formula with two chiplets) when interleave = 1    */
-  SP_CUSTOM = 8     /* caller-supplied table                                                                */
+  SP_CUSTOM = 8,    /* caller-supplied table                                                                */
+  SP_HILBERT_RECT = 9 /* generalised Hilbert curve laid directly over the Tm x Tn rectangle (the published         */
+                    /*   construction for arbitrary rectangles): no cell outside the grid is visited, consecutive   */
+                    /*   slots are adjacent tiles (at most one diagonal step); on 2^k squares it is a Hilbert curve. */
+                    /*   Not in the paper.  Not available as inner order of SP_DIE_SPLIT.                            */
 } sp_scheme;
 
 /* sp_params.flags */

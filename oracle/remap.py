@@ -20,7 +20,7 @@ from dataclasses import dataclass, field
 from typing import List, Optional, Sequence, Tuple
 
 # scheme numbers: the values of the C enum the library's header declares
-ROW_MAJOR, COL_MAJOR, GROUP_M, GROUP_N, MORTON, HILBERT, XCD, DIE_SPLIT, CUSTOM = range(9)
+ROW_MAJOR, COL_MAJOR, GROUP_M, GROUP_N, MORTON, HILBERT, XCD, DIE_SPLIT, CUSTOM, HILBERT_RECT = range(10)
 
 
 class NotBijective(ValueError):
@@ -161,6 +161,55 @@ def morton(Tm: int, Tn: int) -> List[int]:
 # ----------------------------------------------------------------------------------
 # the paper's formula (appendix listing for GEMM): chiplet-aware transposition
 # ----------------------------------------------------------------------------------
+def hilbert_rect_cells(width: int, height: int) -> List[Tuple[int, int]]:
+    """Generalised Hilbert curve over a width x height rectangle, by the published recursive construction (not in the
+    paper): a rectangle spanned by a major vector a and a minor vector b is walked directly when one cell thick, cut in
+    two along a when 2|a| > 3|b|, else cut into three parts walked along b, along a, and back.  Returns the cells
+    (x, y) in visiting order."""
+    out: List[Tuple[int, int]] = []
+
+    def sgn(v: int) -> int:
+        return (v > 0) - (v < 0)
+
+    def gen(x: int, y: int, ax: int, ay: int, bx: int, by: int) -> None:
+        w, h = abs(ax + ay), abs(bx + by)
+        dax, day, dbx, dby = sgn(ax), sgn(ay), sgn(bx), sgn(by)
+        if h == 1:
+            for _ in range(w):
+                out.append((x, y))
+                x, y = x + dax, y + day
+            return
+        if w == 1:
+            for _ in range(h):
+                out.append((x, y))
+                x, y = x + dbx, y + dby
+            return
+        ax2, ay2, bx2, by2 = ax // 2, ay // 2, bx // 2, by // 2     # floor division, also for negative vectors
+        w2, h2 = abs(ax2 + ay2), abs(bx2 + by2)
+        if 2 * w > 3 * h:
+            if w2 % 2 and w > 2:
+                ax2, ay2 = ax2 + dax, ay2 + day                     # prefer even steps
+            gen(x, y, ax2, ay2, bx, by)
+            gen(x + ax2, y + ay2, ax - ax2, ay - ay2, bx, by)
+        else:
+            if h2 % 2 and h > 2:
+                bx2, by2 = bx2 + dbx, by2 + dby
+            gen(x, y, bx2, by2, ax2, ay2)
+            gen(x + bx2, y + by2, ax, ay, bx - bx2, by - by2)
+            gen(x + (ax - dax) + (bx2 - dbx), y + (ay - day) + (by2 - dby), -bx2, -by2, -(ax - ax2), -(ay - ay2))
+
+    if width >= height:
+        gen(0, 0, width, 0, 0, height)
+    else:
+        gen(0, 0, 0, height, width, 0)
+    return out
+
+
+def hilbert_rect(Tm: int, Tn: int) -> List[int]:
+    """x runs along the tile columns, y along the tile rows."""
+    return [y * Tn + x for (x, y) in hilbert_rect_cells(Tn, Tm)]
+
+
 def xcd_window(n: int, X: int, balanced: bool) -> List[int]:
     """Image of the local ids 0..n-1 of one window under the paper's swizzle.
 
@@ -313,6 +362,8 @@ def tile_map(M: int, N: int, tile_m: int, tile_n: int, scheme: int, p: Optional[
         out = xcd(T, p.num_xcds, p.wave, bool(p.xcd_balanced))
     elif scheme == DIE_SPLIT:
         out = die_split(Tm, Tn, p.split_axis, p.inner_scheme, p.inner_group, bool(p.interleave), bool(p.flags & 4))
+    elif scheme == HILBERT_RECT:
+        out = hilbert_rect(Tm, Tn)
     elif scheme == CUSTOM:
         if p.custom_perm is None:
             raise ValueError("custom scheme needs a table")

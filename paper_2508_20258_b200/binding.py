@@ -21,8 +21,8 @@ LIB_PATH = os.environ.get("SWIZZLEPERF_LIB") or os.path.join(_HERE, "libswizzlep
 # sp_status
 OK, ERR_INVALID_ARG, ERR_NOT_BIJECTIVE, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_CUDA, ERR_TIMEOUT, ERR_DEVICE = range(8)
 # sp_scheme
-ROW_MAJOR, COL_MAJOR, GROUP_M, GROUP_N, MORTON, HILBERT, XCD, DIE_SPLIT, CUSTOM = range(9)
-SCHEME_NAMES = ["row_major", "col_major", "group_m", "group_n", "morton", "hilbert", "xcd", "die_split", "custom"]
+ROW_MAJOR, COL_MAJOR, GROUP_M, GROUP_N, MORTON, HILBERT, XCD, DIE_SPLIT, CUSTOM, HILBERT_RECT = range(10)
+SCHEME_NAMES = ["row_major", "col_major", "group_m", "group_n", "morton", "hilbert", "xcd", "die_split", "custom", "hilbert_rect"]
 
 
 class SpParams(ctypes.Structure):

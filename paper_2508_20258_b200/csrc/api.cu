@@ -42,7 +42,7 @@ int resolve_sched(int64_t M, int64_t N, int32_t tileM, int32_t tileN, int scheme
   c.Tm = (int)Tm; c.Tn = (int)Tn; c.T = (int)(Tm * Tn);
   c.group = 1; c.X = 1; c.W = c.T; c.inner_group = 1;
   switch (scheme) {
-    case kRow: case kCol: case kMorton: case kHilbert: break;
+    case kRow: case kCol: case kMorton: case kHilbert: case kHilbertRect: break;
     case kGroupM: case kGroupN:
       if (!p || p->group < 1) { set_error("group must be >= 1"); return SP_ERR_INVALID_ARG; }
       c.group = p->group;
@@ -73,13 +73,19 @@ int resolve_sched(int64_t M, int64_t N, int32_t tileM, int32_t tileN, int scheme
       set_error("unknown scheme %d", scheme);
       return SP_ERR_INVALID_ARG;
   }
+  if (scheme == kHilbertRect && ((int64_t)c.Tm > 32768 || (int64_t)c.Tn > 32768)) {
+    set_error("SP_HILBERT_RECT supports grids up to 32768 tiles per side");
+    return SP_ERR_UNSUPPORTED;
+  }
   const bool curve = scheme == kMorton || scheme == kHilbert ||
                      (scheme == kDieSplit && (c.inner == kMorton || c.inner == kHilbert));
   if (curve && (c.Tm > kMaxCurveSide || c.Tn > kMaxCurveSide)) {
     set_error("curve orders support grids up to %d tiles per side", kMaxCurveSide);
     return SP_ERR_UNSUPPORTED;
   }
-  c.use_table = arithmetic_scheme(c) ? 0 : 1;
+  // The generalised Hilbert curve is arithmetic (no rank among skipped cells is needed) but costs a few hundred
+  // instructions per cell: kernels read it from a table, which the device builder fills with the same function.
+  c.use_table = (arithmetic_scheme(c) && scheme != kHilbertRect) ? 0 : 1;
   *out = c;
   return SP_OK;
 }

@@ -19,7 +19,7 @@
 namespace sp {
 
 enum : int { kRow = 0, kCol = 1, kGroupM = 2, kGroupN = 3, kMorton = 4, kHilbert = 5, kXcd = 6, kDieSplit = 7,
-             kCustom = 8 };
+             kCustom = 8, kHilbertRect = 9 };
 
 struct Sched {
   int scheme;        // sp_scheme
@@ -50,6 +50,49 @@ SP_HD void hilbert_decode(int k, uint32_t d, int& x, int& y) {
     px = nx; py = ny;
   }
   x = px; y = py;
+}
+
+SP_HD int isgn(int v) { return (v > 0) - (v < 0); }
+SP_HD int iabs(int v) { return v < 0 ? -v : v; }
+SP_HD int floor_half(int v) { return v >= 0 ? v / 2 : -((-v + 1) / 2); }
+
+// Cell number d of the generalised Hilbert curve over a rectangle of `width` x `height` cells (the published recursive
+// construction for arbitrary rectangles: a rectangle spanned by a major vector a and a minor vector b is cut in two
+// along a when it is long, else into three parts walked b-wise, a-wise and back).  Instead of generating the whole
+// curve, this descends into the part that holds index d: O(log) steps, no table.  The curve starts at (0, 0) and
+// moves one cell at a time (one diagonal step can occur when the sides' parities force it).
+SP_HD void hilbert_rect_cell(int width, int height, int d, int& cx, int& cy) {
+  int x = 0, y = 0, ax, ay, bx, by;
+  if (width >= height) { ax = width; ay = 0; bx = 0; by = height; } else { ax = 0; ay = height; bx = width; by = 0; }
+  for (;;) {
+    const int w = iabs(ax + ay), h = iabs(bx + by);
+    const int dax = isgn(ax), day = isgn(ay), dbx = isgn(bx), dby = isgn(by);
+    if (h == 1) { cx = x + dax * d; cy = y + day * d; return; }
+    if (w == 1) { cx = x + dbx * d; cy = y + dby * d; return; }
+    int ax2 = floor_half(ax), ay2 = floor_half(ay), bx2 = floor_half(bx), by2 = floor_half(by);
+    const int w2 = iabs(ax2 + ay2), h2 = iabs(bx2 + by2);
+    if (2 * w > 3 * h) {                                   // long: two parts along a
+      if ((w2 & 1) && w > 2) { ax2 += dax; ay2 += day; }
+      const int n1 = iabs(ax2 + ay2) * h;
+      if (d < n1) { ax = ax2; ay = ay2; }
+      else { d -= n1; x += ax2; y += ay2; ax -= ax2; ay -= ay2; }
+    } else {                                               // three parts
+      if ((h2 & 1) && h > 2) { bx2 += dbx; by2 += dby; }
+      const int hb = iabs(bx2 + by2);
+      const int n1 = hb * iabs(ax2 + ay2), n2 = w * (h - hb);
+      if (d < n1) {
+        const int tx = ax2, ty = ay2;
+        ax = bx2; ay = by2; bx = tx; by = ty;
+      } else if (d < n1 + n2) {
+        d -= n1; x += bx2; y += by2; bx -= bx2; by -= by2;
+      } else {
+        d -= n1 + n2;
+        x += (ax - dax) + (bx2 - dbx); y += (ay - day) + (by2 - dby);
+        const int nax = -bx2, nay = -by2, nbx = -(ax - ax2), nby = -(ay - ay2);
+        ax = nax; ay = nay; bx = nbx; by = nby;
+      }
+    }
+  }
 }
 
 SP_HD uint32_t compact_even_bits(uint32_t v) {
@@ -156,7 +199,7 @@ SP_HD bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
 // True when slot_to_tile needs no table for this configuration.
 SP_HD bool arithmetic_scheme(const Sched& c) {
   switch (c.scheme) {
-    case kRow: case kCol: case kGroupM: case kGroupN: case kXcd: return true;
+    case kRow: case kCol: case kGroupM: case kGroupN: case kXcd: case kHilbertRect: return true;
     case kMorton: case kHilbert: return c.Tm == c.Tn && is_pow2(c.Tm);
     case kDieSplit: return c.inner <= kGroupN;
     default: return false;
@@ -172,6 +215,11 @@ SP_HD int slot_to_tile(const Sched& c, int s) {
       int tm, tn;
       curve_cell(c.scheme, curve_order(c.Tm, c.Tn), c.Tm, c.Tn, (uint32_t)s, tm, tn);
       return tm * c.Tn + tn;
+    }
+    case kHilbertRect: {
+      int x, y;
+      hilbert_rect_cell(c.Tn, c.Tm, s, x, y);
+      return y * c.Tn + x;
     }
     case kXcd: {
       const int base = (s / c.W) * c.W;

@@ -45,7 +45,7 @@ def default_candidates(units: int) -> List[Tuple[str, int, Dict]]:
     for g in (2, 4, 8, 16, 32):
         c.append((f"group_m:{g}", sp.GROUP_M, dict(group=g)))
         c.append((f"group_n:{g}", sp.GROUP_N, dict(group=g)))
-    c += [("morton", sp.MORTON, {}), ("hilbert", sp.HILBERT, {})]
+    c += [("morton", sp.MORTON, {}), ("hilbert", sp.HILBERT, {}), ("hilbert_rect", sp.HILBERT_RECT, {})]
     # the paper's formula as printed (may be rejected) and its balanced form, per wave of resident units
     c.append((f"xcd:2:{units}:literal", sp.XCD, dict(num_xcds=2, wave=units, xcd_balanced=0)))
     c.append((f"xcd:8:{units}:literal", sp.XCD, dict(num_xcds=8, wave=units, xcd_balanced=0)))

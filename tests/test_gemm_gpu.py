@@ -44,7 +44,7 @@ def run_gemm(A, B, scheme=sp.ROW_MAJOR, tile=(256, 256), out="bf16", b_is_nk=Fal
                                         (128 * 37, 128 * 5, 128, 128), (128, 128 * 300, 128, 128)])
 def test_device_remap_matches_oracle(M, N, tm, tn):
     cases = [(sp.ROW_MAJOR, {}), (sp.COL_MAJOR, {}), (sp.GROUP_M, dict(group=8)), (sp.GROUP_M, dict(group=3)),
-             (sp.GROUP_N, dict(group=4)), (sp.MORTON, {}), (sp.HILBERT, {}),
+             (sp.GROUP_N, dict(group=4)), (sp.MORTON, {}), (sp.HILBERT, {}), (sp.HILBERT_RECT, {}),
              (sp.XCD, dict(num_xcds=2, wave=74, xcd_balanced=1)), (sp.XCD, dict(num_xcds=8, xcd_balanced=1)),
              (sp.DIE_SPLIT, dict(split_axis=0, inner_scheme=sp.HILBERT)),
              (sp.DIE_SPLIT, dict(split_axis=1, inner_scheme=sp.GROUP_M, inner_group=8, interleave=1)),
@@ -119,7 +119,7 @@ def test_ragged_sizes_full(M, N, K, tile, out, b_is_nk):
     """Several tiles, ragged M / N tails, K not a multiple of the 64-wide k-block."""
     A, B = synth.make_inputs(M, N, K, "normal", 1.0, seed=M)
     ref, S = G.gemm_full(A, B)
-    for scheme, kw in [(sp.HILBERT, {}), (sp.XCD, dict(num_xcds=2, xcd_balanced=1))]:
+    for scheme, kw in [(sp.HILBERT, {}), (sp.HILBERT_RECT, {}), (sp.XCD, dict(num_xcds=2, xcd_balanced=1))]:
         got, _ = run_gemm(A, B, scheme, tile, out, b_is_nk, **kw)
         r = G.compare(got, ref, S)
         assert r["max_err"] <= TOL, (scheme, r)
@@ -182,7 +182,7 @@ def test_output_bits_do_not_depend_on_the_scheme():
     A, B = synth.make_inputs(2048, 2304, 1024, "normal", 1.0, 12)
     ref = None
     table = np.random.default_rng(1).permutation(8 * 9).astype(np.int32)
-    for scheme, kw in [(sp.ROW_MAJOR, {}), (sp.COL_MAJOR, {}), (sp.GROUP_N, dict(group=3)), (sp.MORTON, {}),
+    for scheme, kw in [(sp.ROW_MAJOR, {}), (sp.COL_MAJOR, {}), (sp.GROUP_N, dict(group=3)), (sp.MORTON, {}), (sp.HILBERT_RECT, {}),
                        (sp.XCD, dict(num_xcds=4, wave=16, xcd_balanced=1)), (sp.CUSTOM, dict(custom_perm=table)),
                        (sp.DIE_SPLIT, dict(split_axis=1, inner_scheme=sp.HILBERT))]:
         _, dC = run_gemm(A, B, scheme, (256, 256), "bf16", **kw)
@@ -280,7 +280,7 @@ def test_device_remap_matches_oracle_on_random_grids():
         inner = int(rng.choice([sp.ROW_MAJOR, sp.COL_MAJOR, sp.GROUP_M, sp.GROUP_N, sp.MORTON, sp.HILBERT]))
         axis, inter, serp = int(rng.integers(2)), int(rng.integers(2)), int(rng.integers(2)) * 4
         for scheme, kw in [(sp.GROUP_M, dict(group=G, flags=serp)), (sp.GROUP_N, dict(group=G, flags=serp)),
-                           (sp.MORTON, {}), (sp.HILBERT, {}), (sp.XCD, dict(num_xcds=X, wave=W, xcd_balanced=1)),
+                           (sp.MORTON, {}), (sp.HILBERT, {}), (sp.HILBERT_RECT, {}), (sp.XCD, dict(num_xcds=X, wave=W, xcd_balanced=1)),
                            (sp.DIE_SPLIT, dict(split_axis=axis, inner_scheme=inner, inner_group=G, interleave=inter, flags=serp))]:
             want = R.tile_map(Tm * 64, Tn * 64, 64, 64, scheme, R.Params(**kw))
             got = sp.tile_map_device(Tm * 64, Tn * 64, 64, 64, scheme, sp.make_params(**kw)).cpu().numpy().tolist()

@@ -299,3 +299,36 @@ def test_exactly_when_the_printed_formula_is_a_bijection():
         for X in range(1, 25):
             bij = R.is_bijection(R.xcd_window(n, X, False), n)
             assert bij == (X > n or n % X in (0, X - 1)), (n, X)
+
+
+# ------------------------------------------------- generalised Hilbert curve over a rectangle (not in the paper)
+def test_hilbert_rect_hand_derived_examples():
+    # 4 wide, 2 high: long case, two 2 x 2 blocks each walked down, along, up
+    assert R.hilbert_rect_cells(4, 2) == [(0, 0), (0, 1), (1, 1), (1, 0), (2, 0), (2, 1), (3, 1), (3, 0)]
+    assert R.hilbert_rect(2, 4) == [0, 4, 5, 1, 2, 6, 7, 3]
+    # 2 wide, 3 high: major axis along y; one cell, then a column of three, then back up the first column
+    assert R.hilbert_rect_cells(2, 3) == [(0, 0), (1, 0), (1, 1), (1, 2), (0, 2), (0, 1)]
+    assert R.hilbert_rect(3, 2) == [0, 1, 3, 5, 4, 2]
+    assert R.hilbert_rect(1, 5) == [0, 1, 2, 3, 4] and R.hilbert_rect(5, 1) == [0, 1, 2, 3, 4]
+
+
+def test_hilbert_rect_on_power_of_two_squares_is_a_hilbert_curve():
+    for k in range(1, 6):
+        n = 1 << k
+        cells = R.hilbert_rect_cells(n, n)
+        h = R.hilbert_cells(k)                               # the independent construction pinned above
+        assert cells == h or cells == [(y, x) for (x, y) in h]
+
+
+def test_hilbert_rect_visits_every_cell_once_in_unit_steps():
+    for W in range(1, 26):
+        for H in range(1, 26):
+            cells = R.hilbert_rect_cells(W, H)
+            assert len(cells) == W * H and len(set(cells)) == W * H
+            assert all(0 <= x < W and 0 <= y < H for (x, y) in cells)
+            assert cells[0] == (0, 0)
+            steps = [abs(a[0] - b[0]) + abs(a[1] - b[1]) for a, b in zip(cells, cells[1:])]
+            diagonal = [s for s in steps if s != 1]
+            assert all(s == 2 for s in diagonal) and len(diagonal) <= 1      # at most one diagonal step, never a jump
+            if W % 2 == 0 and H % 2 == 0:
+                assert not diagonal

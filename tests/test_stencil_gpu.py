@@ -11,7 +11,7 @@ pytestmark = pytest.mark.gpu
 torch = pytest.importorskip("torch")
 
 ORDERS = [(sp.ROW_MAJOR, {}), (sp.COL_MAJOR, {}), (sp.GROUP_M, dict(group=3)), (sp.GROUP_N, dict(group=2)), (sp.MORTON, {}),
-          (sp.HILBERT, {}), (sp.XCD, dict(num_xcds=8, xcd_balanced=1)),
+          (sp.HILBERT, {}), (sp.HILBERT_RECT, {}), (sp.XCD, dict(num_xcds=8, xcd_balanced=1)),
           (sp.DIE_SPLIT, dict(split_axis=0, inner_scheme=sp.GROUP_M, inner_group=2, interleave=1))]
 
 

@@ -233,3 +233,16 @@ def test_recommendation_is_valid_and_matches_what_the_sweeps_found():
         sp.recommend(0, 8, 8)
     with pytest.raises(sp.SpError):
         sp.recommend(8, 8, 8, out_dtype=3)
+
+
+def test_hilbert_rect_index_descent_matches_the_recursive_construction():
+    """The library finds cell s by descending into the part of the rectangle that holds it; the oracle generates the
+    whole curve recursively.  Every grid up to 40 x 40, the five workload grids, and some long thin ones."""
+    grids = [(a, b) for a in range(1, 41) for b in range(1, 41)]
+    grids += [(4, 4), (32, 16), (32, 32), (64, 8), (64, 64), (32, 64), (1, 300), (300, 1), (3, 1000), (1000, 3), (127, 255)]
+    for Tm, Tn in grids:
+        got = list(sp.tile_map(Tm, Tn, 1, 1, sp.HILBERT_RECT))
+        assert got == R.hilbert_rect(Tm, Tn), (Tm, Tn)
+    with pytest.raises(sp.SpError) as e:                  # not available inside DIE_SPLIT
+        sp.tile_map(8, 8, 1, 1, sp.DIE_SPLIT, sp.make_params(inner_scheme=sp.HILBERT_RECT))
+    assert e.value.status == sp.ERR_INVALID_ARG

@@ -28,7 +28,7 @@ def test_transpose_is_bit_exact_under_every_order(M, N):
     want = T.transpose(x)
     Tm, Tn = -(-M // 64), -(-N // 64)
     table = np.random.default_rng(5).permutation(Tm * Tn).astype(np.int32)
-    for scheme, kw in [(sp.ROW_MAJOR, {}), (sp.COL_MAJOR, {}), (sp.GROUP_M, dict(group=8)), (sp.HILBERT, {}),
+    for scheme, kw in [(sp.ROW_MAJOR, {}), (sp.COL_MAJOR, {}), (sp.GROUP_M, dict(group=8)), (sp.HILBERT, {}), (sp.HILBERT_RECT, {}),
                        (sp.XCD, dict(num_xcds=8, xcd_balanced=1)), (sp.CUSTOM, dict(custom_perm=table)),
                        (sp.DIE_SPLIT, dict(split_axis=1, inner_scheme=sp.GROUP_N, inner_group=4, interleave=1))]:
         assert np.array_equal(run(x, scheme, **kw), want), (scheme, kw)
