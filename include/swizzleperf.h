@@ -3,6 +3,8 @@
  * A tiled dense bf16 GEMM for NVIDIA B200 (sm_100a) whose block-to-output-tile mapping
  * is a programmable "swizzle": a bijective remap of tile ids, as in the GEMM case study
  * of the SwizzlePerf paper (arXiv 2508.20258, appendix "Case Study: GEMM Swizzling").
+ * Two memory-bound workloads of the paper's suite, a tiled transpose and a 2-D stencil, run
+ * under the same remaps (sp_transpose, sp_stencil2d).
  *
  * Vocabulary.  C (M x N) = A (M x K) . B (K x N) is cut into Tm x Tn output tiles,
  * Tm = ceil(M / tileM), Tn = ceil(N / tileN), T = Tm * Tn.  The logical id of tile
@@ -16,7 +18,8 @@
  * Conventions.  Every function returns an sp_status (0 = success) and never throws,
  * aborts or prints.  "host" / "device" below says where a pointer must point.  The
  * caller owns every buffer it passes; the library owns only its internal caches (tile
- * tables, a status word), released by sp_shutdown().  All device work is enqueued on the
+ * tables, a status word with scheduling counters, staging for the host entry point, the
+ * workspace of SP_FLAG_STREAM_K), released by sp_shutdown().  All device work is enqueued on the
  * caller's stream; nothing synchronises unless stated.
  */
 #ifndef SWIZZLEPERF_H_
