@@ -55,3 +55,25 @@ def test_scheme_specs_parse():
     for name, specs in bench.SWEEPS.items():
         for s in specs:
             bench.parse_scheme(s)
+
+
+def test_scheme_specs_parse_to_library_parameters():
+    import bench
+    import paper_2508_20258_b200 as sp
+    assert bench.parse_scheme("row_major") == (sp.ROW_MAJOR, {})
+    assert bench.parse_scheme("hilbert_rect") == (sp.HILBERT_RECT, {})
+    assert bench.parse_scheme("group_n:8:s") == (sp.GROUP_N, dict(group=8, flags=sp.FLAG_SERPENTINE))
+    assert bench.parse_scheme("xcd:8:148") == (sp.XCD, dict(num_xcds=8, wave=148, xcd_balanced=1))
+    s, kw = bench.parse_scheme("die_split:n:group_m:4:i:p")
+    assert s == sp.DIE_SPLIT and kw == dict(split_axis=1, inner_scheme=sp.GROUP_M, inner_group=4, interleave=1, flags=sp.FLAG_DIE_PINNED)
+    for suffix, flag in (("+k", sp.FLAG_STREAM_K), ("+o", sp.FLAG_OVERLAP), ("+c", sp.FLAG_CLC)):
+        s, kw = bench.parse_scheme("group_m:8" + suffix)
+        assert s == sp.GROUP_M and kw == dict(group=8, flags=flag)
+    # every spec of every sweep list is understood and, on its workload's grid, a bijection (or refused as documented)
+    from paper_2508_20258_b200 import synth
+    for name, specs in bench.SWEEPS.items():
+        w = synth.WORKLOADS[name]
+        for spec in specs:
+            s, kw = bench.parse_scheme(spec)
+            perm = sp.tile_map(w.M, w.N, w.tile_m, w.tile_n, s, sp.make_params(**kw))
+            assert sorted(perm) == list(range(len(perm))), (name, spec)
