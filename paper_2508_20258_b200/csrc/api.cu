@@ -218,6 +218,9 @@ static int current_device(int* dev) {
     return SP_ERR_DEVICE;
   }
   SP_CUDA(cudaGetDevice(dev));
+  // A host thread that has made no runtime call yet has no context bound, and the tensor maps are encoded through the
+  // driver API, which needs one: selecting the device it already has binds the primary context to this thread.
+  SP_CUDA(cudaSetDevice(*dev));
   int major = 0;
   SP_CUDA(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, *dev));
   if (major != 10) {

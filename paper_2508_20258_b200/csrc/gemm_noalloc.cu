@@ -90,6 +90,7 @@ extern "C" int sp_gemm_noalloc(const void* A, const void* B, void* C, int64_t M,
   int ndev = 0, dev = 0;
   if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) { cudaGetLastError(); set_error("no CUDA device"); return SP_ERR_DEVICE; }
   if (cudaGetDevice(&dev) != cudaSuccess) { set_error("cudaGetDevice failed"); return SP_ERR_CUDA; }
+  if (cudaSetDevice(dev) != cudaSuccess) { set_error("cudaSetDevice failed"); return SP_ERR_CUDA; }   // binds the context to this thread (no allocation)
   int32_t* scratch = nullptr;
   rc = noalloc_scratch(dev, &scratch);
   if (rc != SP_OK) return rc;

@@ -357,3 +357,40 @@ def test_gemm_launches_replay_from_a_cuda_graph():
         for o in outs:
             assert np.array_equal(o.cpu().numpy().astype(np.float64), ref)
     assert sp.get_status() == 0
+
+
+def test_host_threads_on_separate_streams():
+    """Four host threads, each with its own stream and problem, call the library at the same time (plain, table-based,
+    die-pinned when available, k-split and cluster-launch-control launches mixed): every result is exact."""
+    import threading
+    jobs = []
+    flags = [0, sp.FLAG_STREAM_K, sp.FLAG_CLC, 0]
+    schemes = [(sp.HILBERT, {}), (sp.GROUP_M, dict(group=4)), (sp.ROW_MAJOR, {}), (sp.DIE_SPLIT, dict(inner_scheme=sp.GROUP_M, inner_group=2))]
+    shapes = [(1024, 1280, 512), (2304, 2560, 1024), (1160, 600, 520), (2048, 2304, 256)]
+    for i in range(4):
+        M, N, K = shapes[i]
+        A, B = synth.make_int_inputs(M, N, K, seed=60 + i)
+        jobs.append(dict(dA=dev_bf16(A), dB=dev_bf16(B), ref=G.gemm_full(A, B)[0],
+                         out=[torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda") for _ in range(6)],
+                         stream=torch.cuda.Stream(), scheme=schemes[i][0],
+                         p=sp.make_params(tile_m=256 if i % 2 else 128, tile_n=256, out_dtype=1, flags=flags[i], **schemes[i][1])))
+    torch.cuda.synchronize()
+    errors = []
+
+    def work(j):
+        try:
+            for o in j["out"]:
+                sp.gemm(j["dA"], j["dB"], o, j["scheme"], j["p"], j["stream"])
+        except Exception as e:      # noqa: BLE001
+            errors.append(e)
+    threads = [threading.Thread(target=work, args=(j,)) for j in jobs]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    torch.cuda.synchronize()
+    assert sp.get_status() == 0
+    for j in jobs:
+        for o in j["out"]:
+            assert np.array_equal(o.cpu().numpy().astype(np.float64), j["ref"])
