@@ -78,3 +78,45 @@ def test_overlap_rejections():
                      sp.make_params(tile_m=128, tile_n=128, flags=OV))
     assert e.value.status == sp.ERR_INVALID_ARG
     assert sp.get_status() == 0 and float(dC.float().abs().sum()) == 0.0
+
+
+def test_dependent_gemms_back_to_back_see_each_others_results():
+    """Ordinary launches are programmatic too (their set-up overlaps the predecessor's tail), so the wait that orders them
+    is checked where it matters: a chain in which every GEMM reads, as its A operand, what the GEMM before it wrote.
+    The GEMMs are large enough for the GPU, not the host, to set the pace, and every other one walks its tiles in reverse,
+    so that its first tiles need what its predecessor writes last (with SP_FLAG_OVERLAP set against its contract, this
+    very chain comes out wrong every time; with ordinary launches it must be exact)."""
+    M = N = K = 4096
+    rng = np.random.default_rng(3)
+    a0 = rng.integers(-3, 4, size=(M, K)).astype(np.float32)
+    A0 = synth.f32_to_bf16_bits(a0)
+    want = a0.astype(np.float64)
+    dPs = []
+    for seed in range(6):                                # right factors: signed permutation matrices, products stay small integers
+        r = np.random.default_rng(seed)
+        j, sg = r.permutation(N), r.choice([-1.0, 1.0], size=K).astype(np.float32)
+        P = np.zeros((K, N), dtype=np.float32)
+        P[np.arange(K), j] = sg
+        dPs.append(dev_bf16(synth.f32_to_bf16_bits(P)))
+        nxt = np.zeros_like(want)
+        nxt[:, j] = want * sg
+        want = nxt
+    for tile, kw in [((256, 256), {}), ((256, 512), {}), ((128, 256), {}), ((256, 256), dict(flags=sp.FLAG_CLC)),
+                     ((256, 256), dict(flags=sp.FLAG_STREAM_K))]:
+        T = sp.tile_count(M, N, tile[0], tile[1])
+        fwd = sp.make_params(tile_m=tile[0], tile_n=tile[1], **kw)
+        rev = sp.make_params(tile_m=tile[0], tile_n=tile[1], custom_perm=np.arange(T - 1, -1, -1, dtype=np.int32), **kw)
+        bufs = [dev_bf16(A0), torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")]
+        sp.gemm(bufs[0], dPs[0], bufs[1], sp.CUSTOM, rev)                 # uploads the table once, outside the chain
+        torch.cuda.synchronize()
+        bufs[1].zero_()
+        src = 0
+        for i, dP in enumerate(dPs):                     # no synchronisation anywhere in the chain
+            if i % 2 == 0:
+                sp.gemm(bufs[src], dP, bufs[1 - src], sp.ROW_MAJOR, fwd)
+            else:
+                sp.gemm(bufs[src], dP, bufs[1 - src], sp.CUSTOM, rev)
+            src = 1 - src
+        assert sp.get_status() == 0
+        got = G.bf16_bits_to_f64(bufs[src].view(torch.int16).cpu().numpy().view(np.uint16))
+        assert np.array_equal(got, want), (tile, kw)
