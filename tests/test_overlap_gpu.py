@@ -120,3 +120,29 @@ def test_dependent_gemms_back_to_back_see_each_others_results():
         assert sp.get_status() == 0
         got = G.bf16_bits_to_f64(bufs[src].view(torch.int16).cpu().numpy().view(np.uint16))
         assert np.array_equal(got, want), (tile, kw)
+
+
+def test_other_kernels_behind_a_gemm_wait_for_all_of_it():
+    """A GEMM tells the hardware at its start that a programmatic successor may be scheduled; a kernel launched the
+    ordinary way behind it (here the transpose, walking its tiles from the end) must still see all of C."""
+    M = N = K = 4096
+    A, B = synth.make_int_inputs(M, N, K, seed=12)
+    dA, dB = dev_bf16(A), dev_bf16(B)
+    dC = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    dT = torch.zeros((N, M), dtype=torch.bfloat16, device="cuda")
+    p = sp.make_params(tile_m=256, tile_n=512)
+    sp.gemm(dA, dB, dC, sp.ROW_MAJOR, p)
+    torch.cuda.synchronize()
+    want = dC.t().contiguous()
+    Tt = sp.tile_count(M, N, 64, 64)
+    rev = sp.make_params(custom_perm=np.arange(Tt - 1, -1, -1, dtype=np.int32))
+    sp.transpose(dC.view(torch.int16), dT.view(torch.int16), sp.CUSTOM, rev)          # uploads the table
+    for _ in range(5):
+        dC.zero_()
+        dT.zero_()
+        torch.cuda.synchronize()
+        sp.gemm(dA, dB, dC, sp.ROW_MAJOR, p)
+        sp.transpose(dC.view(torch.int16), dT.view(torch.int16), sp.CUSTOM, rev)      # starts with the tiles C gets last
+        torch.cuda.synchronize()
+        assert torch.equal(dT.view(torch.int16), want.view(torch.int16))
+    assert sp.get_status() == 0
