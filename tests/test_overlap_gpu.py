@@ -146,3 +146,32 @@ def test_other_kernels_behind_a_gemm_wait_for_all_of_it():
         torch.cuda.synchronize()
         assert torch.equal(dT.view(torch.int16), want.view(torch.int16))
     assert sp.get_status() == 0
+
+
+def test_gemm_behind_a_library_kernel_reads_its_complete_output():
+    """The producer of A is another library's GEMM (which may itself release its programmatic successors early): our
+    launch, walking its tiles from the end, must still read all of it."""
+    M = N = K = 4096
+    rng = np.random.default_rng(8)
+    x = torch.from_numpy(rng.integers(-2, 3, size=(M, K)).astype(np.float32)).cuda().bfloat16()
+    j = torch.from_numpy(rng.permutation(K)).cuda()
+    P = torch.zeros((K, K), dtype=torch.bfloat16, device="cuda")
+    P[torch.arange(K, device="cuda"), j] = 1.0                      # permutation matrix: x @ P is exact
+    E = torch.zeros((K, N), dtype=torch.bfloat16, device="cuda")
+    E[torch.arange(K, device="cuda"), torch.arange(K, device="cuda").flip(0)] = -1.0
+    mid = torch.zeros((M, K), dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    want = -(x.float()[:, torch.argsort(j)]).flip(1)                 # (x P) E, both factors signed permutations
+    T = sp.tile_count(M, N, 256, 256)
+    rev = sp.make_params(tile_m=256, tile_n=256, custom_perm=np.arange(T - 1, -1, -1, dtype=np.int32))
+    sp.gemm(mid, E, out, sp.CUSTOM, rev)
+    torch.cuda.synchronize()
+    for _ in range(5):
+        mid.zero_()
+        out.zero_()
+        torch.cuda.synchronize()
+        torch.matmul(x, P, out=mid)
+        sp.gemm(mid, E, out, sp.CUSTOM, rev)
+        torch.cuda.synchronize()
+        assert torch.equal(out.float(), want)
+    assert sp.get_status() == 0
