@@ -146,3 +146,26 @@ def test_split_through_the_host_entry_point():
     sp.gemm_host(A.view(np.int16), B.view(np.int16), hC, sp.GROUP_M,
                  sp.make_params(tile_m=256, tile_n=256, out_dtype=1, group=2, flags=SK))
     assert np.array_equal(hC.astype(np.float64), ref)
+
+
+def test_split_launches_of_different_shapes_back_to_back_and_on_two_streams():
+    """The workspace and its flags are reused from launch to launch on a stream (a launch counter tells the flags of one
+    launch from the next) and are separate per stream: different split shapes queued back to back on two streams at once."""
+    shapes = [(2304, 2560, 1024, (256, 256)), (512, 512, 2304, (128, 128)), (4096, 4096, 512, (256, 256)),
+              (128 * 13, 256 * 12, 64 * 12, (128, 256)), (2300, 1096, 840, (256, 128))]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    work = []
+    for i, (M, N, K, tile) in enumerate(shapes):
+        A, B = synth.make_int_inputs(M, N, K, seed=90 + i)
+        work.append((dev_bf16(A), dev_bf16(B), G.gemm_full(A, B)[0], tile,
+                     [torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda") for _ in range(4)]))
+    torch.cuda.synchronize()
+    for rep in range(2):
+        for k, st in enumerate(streams):
+            for (dA, dB, _, tile, outs) in work:
+                sp.gemm(dA, dB, outs[2 * rep + k], sp.GROUP_M, sp.make_params(tile_m=tile[0], tile_n=tile[1], out_dtype=1, group=2, flags=SK), st)
+    torch.cuda.synchronize()
+    assert sp.get_status() == 0
+    for (_, _, ref, _, outs) in work:
+        for o in outs:
+            assert np.array_equal(o.cpu().numpy().astype(np.float64), ref)
