@@ -406,3 +406,30 @@ def test_very_long_k():
         assert np.array_equal(got, ref), tile
     got, _ = run_gemm(A, B, sp.ROW_MAJOR, (128, 128), "fp32", flags=sp.FLAG_STREAM_K)     # 8 tiles on 148 units: 18 pieces each
     assert np.array_equal(got, ref)
+
+
+def test_die_pinned_launches_on_two_streams_at_once():
+    """Each die-pinned launch takes its ranks from its own set of counters; two such launches sharing the GPU land on
+    whatever SMs are free, and the overflow rule must still hand out every (half, rank) pair of each launch exactly once."""
+    M, N, K = 4096, 4608, 512
+    A, B = synth.make_int_inputs(M, N, K, seed=31)
+    ref, _ = G.gemm_full(A, B)
+    dA, dB = dev_bf16(A), dev_bf16(B)
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    outs = [[torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda") for _ in range(6)] for _ in streams]
+    p = sp.make_params(tile_m=256, tile_n=256, out_dtype=1, split_axis=0, inner_scheme=sp.GROUP_M, inner_group=4, flags=sp.FLAG_DIE_PINNED)
+    try:
+        sp.gemm(dA, dB, outs[0][0], sp.DIE_SPLIT, p)
+    except sp.SpError as e:
+        if e.status == sp.ERR_UNSUPPORTED:
+            pytest.skip("no two-way L2 structure measured on this device")
+        raise
+    torch.cuda.synchronize()
+    for i in range(6):
+        for k, st in enumerate(streams):
+            sp.gemm(dA, dB, outs[k][i], sp.DIE_SPLIT, p, st)
+    torch.cuda.synchronize()
+    assert sp.get_status() == 0
+    for k in range(2):
+        for o in outs[k]:
+            assert np.array_equal(o.cpu().numpy().astype(np.float64), ref)
