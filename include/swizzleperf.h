@@ -195,7 +195,8 @@ int sp_gemm_trace(const void* A, const void* B, void* C, int64_t M, int64_t N, i
  * runs sp_gemm, copies C back, and synchronises `stream`; C_host is valid on return.  With 4096 rows or more (and
  * neither a caller table nor SP_FLAG_DIE_PINNED) M is split into row blocks of at least 2048 rows, each computed by its
  * own sp_gemm under the same scheme applied to the block's tile grid, so that copies in both directions overlap the
- * compute; the result is the same.  One call at a time per device (the staging area is shared).  Adds SP_ERR_TIMEOUT
+ * compute; the result is the same.  The staging area is shared: calls from several host threads are served one after
+ * the other (the function holds a lock for its whole duration).  Adds SP_ERR_TIMEOUT
  * to sp_gemm's errors. */
 int sp_gemm_host(const void* A_host, const void* B_host, void* C_host, int64_t M, int64_t N, int64_t K, int scheme,
                  const sp_params* params, void* stream);

@@ -508,6 +508,10 @@ int sp_gemm_host(const void* A_host, const void* B_host, void* C_host, int64_t M
     set_error("SP_FLAG_OVERLAP is a statement about device buffers the caller manages; sp_gemm_host orders its own copies and kernels");
     return SP_ERR_INVALID_ARG;
   }
+  // One call at a time: the staging area, the two copy streams and their events are shared, and the call ends with a
+  // synchronisation anyway.  Calls from several host threads queue up here.
+  static std::mutex host_call_mu;
+  std::lock_guard<std::mutex> host_call_lock(host_call_mu);
   const size_t out_elt = (params && params->out_dtype == 1) ? 4 : 2;
   auto pad = [](size_t b) { return (b + 255) & ~(size_t)255; };
   const size_t a_bytes = (size_t)M * (size_t)K * 2, b_bytes = (size_t)K * (size_t)N * 2, c_bytes = (size_t)M * (size_t)N * out_elt;

@@ -433,3 +433,30 @@ def test_die_pinned_launches_on_two_streams_at_once():
     for k in range(2):
         for o in outs[k]:
             assert np.array_equal(o.cpu().numpy().astype(np.float64), ref)
+
+
+def test_host_entry_point_from_two_threads():
+    import threading
+    jobs = []
+    for i, (M, N, K) in enumerate([(4608, 1024, 512), (1024, 768, 256)]):
+        A, B = synth.make_int_inputs(M, N, K, seed=70 + i)
+        jobs.append((A, B, G.gemm_full(A, B)[0], [np.zeros((M, N), dtype=np.float32) for _ in range(3)]))
+    errors = []
+
+    def work(j):
+        A, B, _, outs = j
+        try:
+            for o in outs:
+                sp.gemm_host(A.view(np.int16), B.view(np.int16), o, sp.GROUP_M, sp.make_params(tile_m=128, tile_n=256, out_dtype=1, group=2),
+                             torch.cuda.Stream())
+        except Exception as e:      # noqa: BLE001
+            errors.append(e)
+    threads = [threading.Thread(target=work, args=(j,)) for j in jobs]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    for (_, _, ref, outs) in jobs:
+        for o in outs:
+            assert np.array_equal(o.astype(np.float64), ref)
