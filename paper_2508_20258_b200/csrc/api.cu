@@ -211,6 +211,13 @@ static uint64_t fnv(const int32_t* v, int n) {
   } while (0)
 
 static int current_device(int* dev) {
+  // the checks below are per (host thread, device): once passed, a call costs one cudaGetDevice
+  static thread_local int checked_dev = -1;
+  if (checked_dev >= 0) {
+    int d = -1;
+    if (cudaGetDevice(&d) == cudaSuccess && d == checked_dev) { *dev = d; return SP_OK; }
+    checked_dev = -1;
+  }
   int n = 0;
   if (cudaGetDeviceCount(&n) != cudaSuccess || n == 0) {
     cudaGetLastError();
@@ -227,6 +234,7 @@ static int current_device(int* dev) {
     set_error("device %d has compute capability %d.x; this library is sm_100a only", *dev, major);
     return SP_ERR_DEVICE;
   }
+  checked_dev = *dev;
   return SP_OK;
 }
 

@@ -177,6 +177,11 @@ __device__ __forceinline__ bool mbar_wait_timed(uint32_t bar, uint32_t parity, i
   return ok;
 }
 
+// Start fetching a tensor map (kernel parameter space) into the TMA unit's descriptor cache before its first use.
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
 template <int CG>
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
   if constexpr (CG == 1) {
