@@ -211,7 +211,7 @@ def run_ours(args) -> int:
             rs, rp = sp.recommend(Ms, Ns, Ks, 0, b_nk)      # nothing asked for: the library's own suggestion for the shape
             args.tile = f"{rp.tile_m}x{rp.tile_n}"
             args.scheme = {sp.ROW_MAJOR: "row_major", sp.COL_MAJOR: "col_major", sp.GROUP_M: f"group_m:{rp.group}",
-                           sp.GROUP_N: f"group_n:{rp.group}"}[rs]
+                           sp.GROUP_N: f"group_n:{rp.group}"}[rs] + ("+k" if rp.flags & sp.FLAG_STREAM_K else "")
     else:
         w = synth.WORKLOADS[args.workload]
         _, A, B = synth.make_workload(args.workload, b_is_nk=bool(b_nk))

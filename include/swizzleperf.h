@@ -79,7 +79,7 @@ typedef enum {
 #define SP_FLAG_STREAM_K 8u   /* sp_gemm / sp_gemm_trace / sp_gemm_host, tiles up to 256x256: wave quantisation.  The paper's
                                  remap picks the tile of a slot and has no counterpart for this.  When the persistent units U
                                  do not divide the tile count T, the last R = T mod U slots of the order are split along k:
-                                 each of their tiles goes to f = min(U / R, kblocks / 4) units, piece i taking k-blocks
+                                 each of their tiles goes to f = min(U / R, kblocks / 4, 8) units, piece i taking k-blocks
                                  [i * kblocks / f, (i + 1) * kblocks / f) (sp_streamk_plan lists the pieces); nothing is
                                  split when f < 2.  Pieces with the same i walk k in step, so they still share operand
                                  panels in L2.  A unit whose piece ends before the tile's last k-block writes an fp32 partial
@@ -264,7 +264,8 @@ int sp_stencil2d(const void* in, void* out, int64_t M, int64_t N, float c_center
  * waves x tile area / (CTAs per tile x relative efficiency of the tile shape), waves = ceil(T / units), units = 74 CTA
  * pairs or 148 CTAs; row-major when A and B together are at most 64 MiB (they stay in L2) or the tile grid is at most
  * ten tiles wide, column-major when it is at most ten tiles tall, else bands of 8 tile columns (256x512 tile) or 8
- * tile rows (other tiles).  Host only; no GPU needed.
+ * tile rows (other tiles); SP_FLAG_STREAM_K is set when the tiles fill at most half of the units and K is at least
+ * 2048 (C then differs in rounding order from a launch without the flag).  Host only; no GPU needed.
  *   params : HOST, receives a complete sp_params (struct_size, tile_m, tile_n, group, out_dtype, b_layout set; the
  *            rest zero).   scheme : HOST, receives the sp_scheme.
  * Errors: SP_ERR_INVALID_ARG (NULL, sizes <= 0, bad out_dtype / b_layout). */

@@ -12,15 +12,16 @@ from typing import List, Tuple
 
 FULL, CONTRIB, OWNER = 0, 1, 2
 MIN_RANGE = 4   # a unit's range is at least this many k-blocks, else fewer units share the tail
+MAX_PIECES = 8  # pieces per tile: the storing unit adds the others one after the other
 
 
 def tail(T: int, units: int, kblocks: int) -> Tuple[int, int]:
     """(number of tail slots, units sharing them): the remainder R = T mod units, each of its tiles cut into
-    f = units // R equal pieces (at least MIN_RANGE k-blocks each); nothing when f < 2."""
+    f = units // R equal pieces (at least MIN_RANGE k-blocks each, at most MAX_PIECES); nothing when f < 2."""
     R = T % units
     if R == 0:
         return 0, units
-    f = min(units // R, kblocks // MIN_RANGE)
+    f = min(units // R, kblocks // MIN_RANGE, MAX_PIECES)
     if f < 2:
         return 0, units
     return R, R * f

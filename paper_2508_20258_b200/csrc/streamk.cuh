@@ -81,18 +81,20 @@ SP_SK_HD int sk_contributors(const SkPlan& p, int unit, int slot, int KB) {
 
 // Host policy: which slots form the tail for T tiles on `units` units with KB k-blocks per tile.
 // Only the remainder R = T mod units is split, and only into equal pieces: each of its tiles goes to f = units / R
-// units (f >= 2, pieces of at least kMinRange k-blocks), piece i covering k-blocks [i * KB / f, (i + 1) * KB / f).
+// units (2 <= f <= kMaxPieces, pieces of at least kMinRange k-blocks), piece i covering k-blocks [i * KB / f, (i + 1) * KB / f).
 // Pieces with the same i run side by side and walk k in step, as the tiles of a full wave do, so the A and B panels
 // they share are still read from L2 by all of them at the same time.  (Ranges of unequal phase -- the general
 // stream-K cut, also over an extra full wave -- were measured: every unit then streams its operands alone, the tail
 // turns DRAM-bound and takes longer than the partly empty wave it replaces.)
 inline SkPlan sk_plan(int64_t T, int units, int KB) {
   constexpr int kMinRange = 4;
+  constexpr int kMaxPieces = 8;
   SkPlan p = {0, units, (int)T};
   const int64_t R = T % units;
   if (R == 0) return p;
   int64_t f = units / R;
   if (f > KB / kMinRange) f = KB / kMinRange;
+  if (f > kMaxPieces) f = kMaxPieces;      // the unit that stores a tile adds the other pieces one after the other
   if (f < 2) return p;
   p.tiles = (int)R;
   p.units = (int)(R * f);

@@ -397,14 +397,14 @@ def test_host_threads_on_separate_streams():
 
 
 def test_very_long_k():
-    """One tile, 1024 k-blocks: the ring, the phase bits and the accumulation run far longer than in any workload."""
+    """Eight tiles at most, 1024 k-blocks: the ring, the phase bits and the accumulation run far longer than in any workload."""
     M, N, K = 256, 512, 65536
     A, B = synth.make_int_inputs(M, N, K, seed=9)
     ref, _ = G.gemm_full(A, B)
     for tile in [(256, 512), (256, 256), (128, 128)]:
         got, _ = run_gemm(A, B, sp.ROW_MAJOR, tile, "fp32")
         assert np.array_equal(got, ref), tile
-    got, _ = run_gemm(A, B, sp.ROW_MAJOR, (128, 128), "fp32", flags=sp.FLAG_STREAM_K)     # 8 tiles on 148 units: 18 pieces each
+    got, _ = run_gemm(A, B, sp.ROW_MAJOR, (128, 128), "fp32", flags=sp.FLAG_STREAM_K)     # 8 tiles on 148 units: 8 pieces each
     assert np.array_equal(got, ref)
 
 

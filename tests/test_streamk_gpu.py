@@ -44,7 +44,7 @@ SPLIT_SHAPES = [
     ((256, 256), 4096, 4096, 512),     # 256 tiles: 34 left, 2 pieces
     ((256, 128), 2300, 1096, 840),     # ragged in M, N and K: 81 tiles, 7 left, 3 pieces
     ((128, 256), 128 * 13, 256 * 12, 64 * 12),   # 156 tiles on 148 units: 8 left, 3 pieces of 4 k-blocks
-    ((128, 128), 512, 512, 2304),      # smaller than a wave: 16 tiles, 9 pieces each
+    ((128, 128), 512, 512, 2304),      # smaller than a wave: 16 tiles, 8 pieces each (the cap)
     ((128, 128), 1024, 1280, 768),     # 80 tiles on 148 units: no split (f = 1)
 ]
 
@@ -64,7 +64,7 @@ def test_split_tail_is_exact_on_integer_inputs(tile, M, N, K, b_is_nk):
 
 
 def test_the_shapes_above_do_split():
-    expect = {0: 64, 1: 68, 3: 24, 4: 144, 5: 0}    # units holding a piece (256x128 case depends on raggedness: skipped)
+    expect = {0: 64, 1: 68, 3: 24, 4: 128, 5: 0}    # units holding a piece (256x128 case depends on raggedness: skipped)
     for i, n in expect.items():
         tile, M, N, K = SPLIT_SHAPES[i]
         if sp.gemm_units(tile[0], tile[1], 1 << 24) != (74 if tile[0] == 256 else 148):

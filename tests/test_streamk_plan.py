@@ -13,7 +13,7 @@ CASES = [
     (1024, 74, 128),    # 8192^3: 13 full waves + 62: more than half a wave, nothing is split
     (512, 148, 64),     # 4096^3 with 128x256 tiles: 68 left, cut in two
     (16, 148, 8),       # smaller than a wave: pieces of 4 k-blocks (two per tile) although nine units per tile are free
-    (16, 148, 64),      # ... nine pieces per tile
+    (16, 148, 64),      # ... eight pieces per tile (nine units per tile are free, eight is the cap)
     (16, 148, 2),       # ... too few k-blocks to split
     (3, 74, 64), (75, 74, 5), (75, 74, 64), (147, 74, 3), (149, 148, 16), (100, 7, 13), (101, 7, 13), (5, 4, 256),
     (9, 4, 1),
@@ -33,7 +33,7 @@ def test_plan_matches_enumeration(T, units, kb):
 def test_plan_properties(T, units, kb):
     first, segs = sp.streamk_plan(T, units, kb)
     R = T % units
-    f = min(units // R, kb // 4) if R else 0
+    f = min(units // R, kb // 4, 8) if R else 0
     if f < 2:
         assert first == T and all(s == [] for s in segs)
         return
