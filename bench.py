@@ -30,24 +30,18 @@ from paper_2508_20258_b200 import benchutil, synth  # noqa: E402
 
 L2_BYTES = 126 * 2 ** 20
 
-# DRAM bytes per launch of the GEMM kernel from the ncu captures summarised under profiles/
-# (dram__bytes_read.sum + dram__bytes_write.sum), keyed by (workload, tile, scheme spec); None = not captured.
-NCU_DRAM_BYTES = {
-    ("cfg3", "256x512", "group_n:8"): 0.956e9,   # profiles/gemm_kernel_cfg3_256x512_group_n8_full.md (mean of 2 launches)
-    ("cfg3", "256x512", "die_split:m:group_m:8:p"): 0.971e9,   # this and the rest: profiles/l2_hit_rate_per_scheme.md
-    ("cfg3", "256x256", "die_split:m:group_m:8:p"): 1.229e9,
-    ("cfg3", "256x256", "group_m:8"): 1.216e9,
-    ("cfg3", "256x256", "row_major"): 2.363e9,
-    ("cfg3", "256x256", "group_n:8"): 1.245e9,
-    ("cfg3", "256x256", "hilbert"): 1.271e9,
-    ("cfg5", "256x512", "die_split:m:group_m:8:p"): 1.647e9,
-    ("cfg5", "256x256", "die_split:m:group_m:8:p"): 1.348e9,
-    ("cfg5", "256x256", "group_m:16"): 1.623e9,
-    ("cfg5", "256x256", "group_m:8"): 2.090e9,
-    ("cfg4", "256x256", "group_n:8"): 0.548e9,
-    ("cfg2", "128x256", "group_m:8"): 0.092e9,
-    ("cfg2", "128x256", "row_major"): 0.084e9,
-}
+
+
+def captured_traffic(workload: str, tile: str, spec: str):
+    """DRAM bytes per launch of the GEMM kernel for (workload, tile, order), from the table of profiler captures kept
+    beside the package (written by `python -m paper_2508_20258_b200.ncuparse --traffic`); None when that combination
+    was never captured."""
+    path = os.path.join(ROOT, "paper_2508_20258_b200", "ncu_traffic.json")
+    with open(path) as fh:
+        for rec in json.load(fh)["captures"]:
+            if (rec["workload"], rec["tile"], rec["scheme"]) == (workload, tile, spec):
+                return rec
+    return None
 
 
 def parse_scheme(spec: str):
@@ -173,6 +167,114 @@ def run_reference(args) -> int:
     return 0
 
 
+def sustained_leg(fn, flops, stream, gpu_index, seconds=4.0):
+    """`fn` launched back to back for at least `seconds` (how the pool's sustained peak was taken): mean TFLOP/s over
+    the whole stretch, the SM clock sampled through it, and time x clock = SM cycles per launch, which separates what
+    the kernel needs from what the power limiter grants."""
+    import math
+    import torch
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for _ in range(3):
+        fn()
+    e0.record(stream)
+    for _ in range(10):
+        fn()
+    e1.record(stream)
+    e1.synchronize()
+    one = e0.elapsed_time(e1) / 10
+    n = int(math.ceil(seconds * 1e3 / one * 1.06))           # launches get slower as the clock settles: aim a little high
+    sampler = benchutil.ClockSampler(gpu_index, period_s=0.02).start()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    e0.record(stream)
+    for _ in range(n):
+        fn()
+    e1.record(stream)
+    e1.synchronize()
+    t1 = time.perf_counter()
+    sampler.stop()
+    ms = e0.elapsed_time(e1)
+    c = sampler.summary(t0, t1)
+    inside = [x[1] for x in sampler.samples if t0 <= x[0] <= t1]
+    return {"launches": n, "seconds": ms / 1e3, "ms_per_launch": ms / n, "tflops": flops * n / ms / 1e9,
+            "clocks": c, "sm_mhz_min": min(inside) if inside else None, "sm_mhz_max": max(inside) if inside else None,
+            "sm_cycles_per_launch": None if not c.get("sm_mhz") else ms / n * 1e3 * c["sm_mhz"]}
+
+
+def workloads_block(sp, names, peaks, stream):
+    """The other named workloads, each timed briefly in the same process: the fastest known (tile, order) for it beside
+    row-major on the same tile (alternating blocks, median of three), and the workload's nominal tile when that is another
+    one.  For the launch-bound 512^3 also what a call costs on the host and how long one launch takes from call to
+    completion."""
+    import torch
+    out = {}
+    for name in names:
+        w, A, B = synth.make_workload(name)
+        out_f32 = int(w.out_dtype == "fp32")
+        dA = torch.from_numpy(A.view(np.int16)).cuda().view(torch.bfloat16)
+        dB = torch.from_numpy(B.view(np.int16)).cuda().view(torch.bfloat16)
+        dC = torch.empty((w.M, w.N), dtype=torch.float32 if out_f32 else torch.bfloat16, device="cuda")
+        flops = 2.0 * w.M * w.N * w.K
+        tile = DEFAULT_TILE.get(name) or f"{w.tile_m}x{w.tile_n}"
+        spec = DEFAULT_SCHEME_BY_TILE.get((name, tile)) or DEFAULT_SCHEME[name]
+
+        def arm(tile_s, spec_s):
+            tm, tn = (int(v) for v in tile_s.split("x"))
+            scheme, kw = parse_scheme(spec_s)
+            return scheme, sp.make_params(tile_m=tm, tile_n=tn, out_dtype=out_f32, **kw)
+
+        def usable(tile_s, spec_s):
+            try:
+                sp.gemm(dA, dB, dC, *arm(tile_s, spec_s), stream)
+                return True
+            except sp.SpError as err:
+                if err.status != sp.ERR_UNSUPPORTED:
+                    raise
+                return False
+        if not usable(tile, spec):
+            spec = FALLBACK_SCHEME.get(name, "row_major")
+        arms = [("best", tile, spec), ("row_major", tile, "row_major")]
+        nominal_tile = f"{w.tile_m}x{w.tile_n}"
+        if nominal_tile != tile:
+            nspec = DEFAULT_SCHEME[name] if usable(nominal_tile, DEFAULT_SCHEME[name]) else FALLBACK_SCHEME.get(name, "row_major")
+            arms.append(("nominal_tile", nominal_tile, nspec))
+        for _, t_, s_ in arms:
+            for _ in range(3):
+                sp.gemm(dA, dB, dC, *arm(t_, s_), stream)
+        est = time_steps(sp, dA, dB, dC, *arm(tile, spec), 5, stream) / 5
+        n = int(max(10, min(2000, 40.0 / est)))
+        ms = {k: [] for k, _, _ in arms}
+        for _ in range(3):
+            for k, t_, s_ in arms:
+                ms[k].append(time_steps(sp, dA, dB, dC, *arm(t_, s_), n, stream) / n)
+        med = {k: sorted(v)[1] for k, v in ms.items()}
+        rec = {"shape": [w.M, w.N, w.K], "out": w.out_dtype, "tile": tile, "scheme": spec, "launches_per_block": n,
+               "ms": med["best"], "tflops": flops / med["best"] / 1e9, "frac_of_burst_peak": flops / med["best"] / 1e9 / peaks["bf16_tflops"],
+               "row_major_tflops": flops / med["row_major"] / 1e9, "speedup_over_row_major": med["row_major"] / med["best"]}
+        if "nominal_tile" in med:
+            rec["nominal_tile"] = {"tile": nominal_tile, "scheme": arms[2][2], "tflops": flops / med["nominal_tile"] / 1e9}
+        if flops < 1e9:      # launch-bound: what a call costs
+            scheme, p = arm(tile, spec)
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            for _ in range(200):     # few enough for the launch queue never to fill: pure host cost of the call
+                sp.gemm(dA, dB, dC, scheme, p, stream)
+            rec["host_us_per_call"] = (time.perf_counter() - t0) / 200 * 1e6
+            torch.cuda.synchronize()
+            lat = []
+            for _ in range(20):
+                t0 = time.perf_counter()
+                sp.gemm(dA, dB, dC, scheme, p, stream)
+                torch.cuda.synchronize()
+                lat.append((time.perf_counter() - t0) * 1e6)
+            rec["call_to_completion_us"] = min(lat)
+            rec["device_us_per_launch_back_to_back"] = med["best"] * 1e3
+        assert sp.get_status() == 0
+        out[name] = rec
+        del dA, dB, dC
+    return out
+
+
 # ---------------------------------------------------------------------------------- our arm
 def time_steps(sp, dA, dB, dC, scheme, p, steps, stream):
     import torch
@@ -270,6 +372,14 @@ def run_ours(args) -> int:
             raise
         spec = FALLBACK_SCHEME[args.workload]
         scheme, p = params_for(spec)
+    tile_s = f"{tile_m}x{tile_n}"
+    traffic = None
+    if not (args.kernel_only or args.no_traffic):
+        traffic = captured_traffic(w.name, tile_s, spec)
+        if traffic is None:
+            raise SystemExit(f"no profiler capture of DRAM traffic for ({w.name}, {tile_s}, {spec}): capture it (ncu over "
+                             f"`bench.py --profile-sweep`, then `python -m paper_2508_20258_b200.ncuparse --sweep ... --traffic`) "
+                             f"or pass --no-traffic to report roofline.traffic as null")
     for _ in range(max(args.warmup, 3)):
         sp.gemm(dA, dB, dC, scheme, p, stream)
     torch.cuda.synchronize()
@@ -280,7 +390,7 @@ def run_ours(args) -> int:
                           "ms_per_step": ms / args.steps, "tflops": flops * args.steps / ms / 1e9}), flush=True)
         return 0
 
-    sampler = benchutil.ClockSampler(local_rank).start()
+    sampler = benchutil.ClockSampler(local_rank, period_s=0.002).start()
     barrier()
     t_host0 = time.perf_counter()
     ms_total = time_steps(sp, dA, dB, dC, scheme, p, args.steps, stream)
@@ -380,6 +490,28 @@ def run_ours(args) -> int:
         cublas["ours_burst_alternating_tflops"] = flops / min(b_ours) / 1e9
         del ref
 
+    # the same launches back to back for four seconds, against the pool's sustained peak, with the clocks
+    sustained = None
+    if not args.no_sustained:
+        sustained = sustained_leg(lambda: sp.gemm(dA, dB, dC, scheme, p, stream), flops, stream, local_rank, args.sustained_seconds)
+        sustained["peak"] = benchutil.measured_peaks(ROOT)["bf16_tflops_sustained"]
+        sustained["frac"] = sustained["tflops"] / sustained["peak"]
+        sustained["protocol"] = f"launches back to back for >= {args.sustained_seconds:g} s, mean over the whole stretch; clock sampled every 20 ms"
+        if cublas is not None:
+            time.sleep(1.0)
+            ref = torch.empty_like(dC)
+            lib = sustained_leg(lambda: torch.matmul(dA, dB, out=ref), flops, stream, local_rank, args.sustained_seconds)
+            cublas["sustained"] = {k: lib[k] for k in ("tflops", "seconds", "sm_cycles_per_launch")}
+            cublas["sustained"]["sm_mhz"] = lib["clocks"]["sm_mhz"]
+            sustained["over_cublas_same_run"] = sustained["tflops"] / lib["tflops"]
+            del ref
+    assert sp.get_status() == 0
+
+    workloads = None
+    if rank == 0 and not args.no_workloads and not args.shape:
+        workloads = workloads_block(sp, [n_ for n_ in ("cfg1", "cfg2", "cfg4", "cfg5") if n_ != args.workload],
+                                    benchutil.measured_peaks(ROOT), stream)
+
     # end to end through the C ABI with host buffers (pinned): H2D of A and B, kernel, D2H of C, every step
     e2e = None
     if not args.no_e2e:
@@ -398,19 +530,63 @@ def run_ours(args) -> int:
         e2e = {"value": eagg["units"] / eagg["ms"] / 1e9, "unit": "TFLOP/s", "h2d_bytes_per_step": int(A.nbytes + B.nbytes),
                "d2h_bytes_per_step": int(hC.numel() * hC.element_size()), "steps": e2e_steps,
                "ms_per_step": eagg["ms"] / e2e_steps, "api": "sp_gemm_host (pinned host buffers)"}
+        # the floor the copies alone set on this machine: the same bytes over PCIe with nothing else going on, each direction
+        # on its own and both at once (what the pipelined call does); floor = the slower direction
+        dAB = torch.empty(A.nbytes + B.nbytes, dtype=torch.uint8, device="cuda")
+        hAB = torch.empty(A.nbytes + B.nbytes, dtype=torch.uint8).pin_memory()
+        hCb = hC.view(torch.uint8).reshape(-1)
+        dCb = dC.view(torch.uint8).reshape(-1)
+        s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+
+        def copies(h2d, d2h):
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            if h2d:
+                with torch.cuda.stream(s_in):
+                    dAB.copy_(hAB, non_blocking=True)
+            if d2h:
+                with torch.cuda.stream(s_out):
+                    hCb.copy_(dCb, non_blocking=True)
+            torch.cuda.synchronize()
+            return (time.perf_counter() - t0) * 1e3
+        copies(True, True)
+        h2d_ms = min(copies(True, False) for _ in range(3))
+        d2h_ms = min(copies(False, True) for _ in range(3))
+        both_ms = min(copies(True, True) for _ in range(3))
+        e2e["pcie_floor"] = {"h2d_GBps": dAB.numel() / h2d_ms / 1e6, "d2h_GBps": dCb.numel() / d2h_ms / 1e6, "h2d_ms": h2d_ms,
+                             "d2h_ms": d2h_ms, "both_directions_at_once_ms": both_ms, "floor_ms": max(h2d_ms, d2h_ms),
+                             "e2e_over_floor": e2e["ms_per_step"] / max(h2d_ms, d2h_ms),
+                             "note": "pinned host memory, one copy per direction, best of 3; rank 0's box"}
+        del dAB, hAB
         del hA, hB, hC
 
     peaks = benchutil.measured_peaks(ROOT)
     launch_ms = ms_total / args.steps
     achieved = flops / launch_ms / 1e9
+    # Which measured peak the timed region is compared with follows from its length: the pool's burst figure was taken on
+    # single launches, its sustained figure on launches back to back for 4 s (the chip then sits at its power limit and
+    # the clock has settled).  A timed region of under a second has not settled: it is a burst and is divided by the burst
+    # peak.  The `sustained` record below repeats the measurement the other way.
+    is_burst = ms_total < 1000.0
+    peak = peaks["bf16_tflops"] if is_burst else peaks["bf16_tflops_sustained"]
+    out_bytes = 4 if out_f32 else 2
+    algorithmic_bytes = 2.0 * (w.M * w.K + w.K * w.N) + out_bytes * w.M * w.N
     roofline = {
-        "bound": "tensor", "kernel": f"gemm_kernel<CG={tile_m // 128},BN={tile_n}>" + (" (two 256x256 2-CTA MMA tiles sharing A)" if tile_n == 512 else ""), "achieved": achieved,
-        "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops_sustained"],
-        "peak_kind": f"cuBLAS bf16 sustained, {peaks['source']}; launches are timed back to back inside the step loop",
-        "traffic": NCU_DRAM_BYTES.get((w.name, f"{tile_m}x{tile_n}", spec)),
+        "bound": "tensor", "kernel": f"gemm_kernel<CG={tile_m // 128},BN={tile_n}>" + (" (two 256x256 2-CTA MMA tiles sharing A)" if tile_n == 512 else ""),
+        "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+        "peak_kind": (f"cuBLAS bf16 {'burst (best single launch)' if is_burst else 'sustained (4 s back to back)'}, {peaks['source']}; "
+                      f"the timed region lasted {ms_total:.1f} ms"),
+        "traffic": None if traffic is None else traffic["dram_bytes"],
+        "traffic_source": None if traffic is None else {"captured": traffic["captured"], "command": traffic["command"],
+                                                        "dram_read_bytes": traffic["dram_read_bytes"],
+                                                        "dram_write_bytes": traffic["dram_write_bytes"]},
+        "algorithmic_bytes": algorithmic_bytes,
+        "traffic_over_algorithmic": None if traffic is None else traffic["dram_bytes"] / algorithmic_bytes,
         "algorithmic_flops_per_launch": flops,
+        "sm_cycles_per_launch": None if not clocks.get("sm_mhz") else launch_ms * 1e3 * clocks["sm_mhz"],
         "burst": {"achieved": flops / burst_ms / 1e9, "peak": peaks["bf16_tflops"],
                   "frac": flops / burst_ms / 1e9 / peaks["bf16_tflops"], "protocol": "best of 10 single launches, each queued behind one untimed launch"},
+        "sustained": sustained,
         "frac_of_nominal_2250": achieved / 2250.0,
     }
 
@@ -449,6 +625,7 @@ def run_ours(args) -> int:
                        "parallelism": "replicas only" if world > 1 else "1 GPU"},
             "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": args.steps,
             "clocks": clocks,
+            "workloads": workloads,
             "nominal_tile": nominal, "cublas_context": cublas, "overlapped_launches": overlapped,
             "row_major": {"ms_per_step": row_ms, "tflops": flops / row_ms / 1e9, "speedup_of_scheme": row_ms / launch_ms},
         }
@@ -744,6 +921,10 @@ def main() -> int:
                     help="--sweep-sustained: append each scheme's line to FILE and skip schemes already in it")
     ap.add_argument("--b-layout", default="kn", choices=["kn", "nk"], help="B stored K x N (default) or N x K")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the four-second back-to-back leg")
+    ap.add_argument("--sustained-seconds", type=float, default=4.0)
+    ap.add_argument("--no-workloads", action="store_true", help="skip the brief timings of the other named workloads")
+    ap.add_argument("--no-traffic", action="store_true", help="report roofline.traffic as null when no capture exists")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--transpose", default=None, metavar="MxN", help="time sp_transpose on an M x N 16-bit matrix instead")
     ap.add_argument("--stencil", default=None, metavar="MxN", help="time sp_stencil2d on an M x N fp32 grid instead")

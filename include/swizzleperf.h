@@ -109,8 +109,7 @@ typedef enum {
                                  before it has completed and its writes are visible (so only launch latency and set-up
                                  overlap, and the stream order is the usual one); a launch with this flag does not wait.  CTAs of the next GEMM then take over SMs as the CTAs of the
                                  previous one finish, which fills the partly empty last wave of back-to-back independent
-                                 GEMMs.  The paper has no counterpart.  A launch that first has to build its tile table (first
-                                 use of a non-arithmetic order) is made without the overlap.  Not with SP_FLAG_DIE_PINNED,
+                                 GEMMs.  The paper has no counterpart.  Not with SP_FLAG_DIE_PINNED,
                                  SP_FLAG_STREAM_K or tracing (SP_ERR_INVALID_ARG).  It still completes after its predecessor, so the
                                  stream order seen by everything else (copies, events, other kernels) is unchanged. */
 
@@ -130,7 +129,7 @@ typedef struct {
                               /*   the A panel); 0,0 = 256x256.  Ignored by sp_tile_map*.                    */
   int32_t out_dtype;          /* sp_gemm*: 0 = C is bf16 (round to nearest even), 1 = C is fp32             */
   int32_t b_layout;           /* sp_gemm*: 0 = B is K x N row-major, 1 = B is N x K row-major               */
-  uint32_t flags;             /* 0, or any of SP_FLAG_DIE_PINNED, _SERPENTINE, _STREAM_K, _OVERLAP            */
+  uint32_t flags;             /* 0, or any of SP_FLAG_DIE_PINNED, _SERPENTINE, _STREAM_K, _OVERLAP, _CLC      */
 } sp_params;
 
 /* One record per tile, written by sp_gemm_trace. */
@@ -175,12 +174,14 @@ int sp_tile_map_device(int64_t M, int64_t N, int32_t tileM, int32_t tileN, int s
  * Products are accumulated in fp32 on the tensor cores.  M and N need not be tile multiples.
  * Errors (all detected on the host, nothing launched): as sp_tile_map, plus SP_ERR_ALIGNMENT (A, B or C not
  * 16-byte aligned; K or N not a multiple of 8), SP_ERR_UNSUPPORTED (tile shape), SP_ERR_DEVICE, SP_ERR_CUDA.
- * The first call for a given (grid, scheme) may allocate a cached tile table; later calls allocate nothing and
- * issue only the kernel launch, so after one warm-up call per
+ * The first call for a given (grid, scheme) may allocate a cached tile table, fills it on `stream` and synchronises
+ * `stream` once before the table becomes visible to other calls (so a call on any other stream or host thread that
+ * finds it may launch at once); later calls allocate nothing, synchronise nothing and
+ * issue only the kernel launch (tensor maps of recently used matrices are kept per host thread), so after one warm-up call per
  * (shape, scheme, params) further calls can be recorded into a CUDA graph by stream capture and replayed; the
  * pointers and the order are then those of the recording.
  * A device-side wait that expires is reported by sp_get_status, not here.
- * With the environment variable SP_LOG set, every launch writes one line to stderr (shape, tile, variant, grid, pipeline
+ * With the environment variable SP_LOG set when the library is first used, every launch writes one line to stderr (shape, tile, variant, grid, pipeline
  * depth, flags in effect); nothing is ever written to stdout. */
 int sp_gemm(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t K, int scheme,
             const sp_params* params, void* stream);
@@ -193,9 +194,10 @@ int sp_gemm_trace(const void* A, const void* B, void* C, int64_t M, int64_t N, i
 /* sp_gemm for callers whose matrices live in HOST memory (pinned or pageable), same layouts and dtypes:
  * copies A and B to a device staging area owned by the library (grown on demand, kept until sp_shutdown),
  * runs sp_gemm, copies C back, and synchronises `stream`; C_host is valid on return.  With 4096 rows or more (and
- * neither a caller table nor SP_FLAG_DIE_PINNED) M is split into row blocks of at least 2048 rows, each computed by its
- * own sp_gemm under the same scheme applied to the block's tile grid, so that copies in both directions overlap the
- * compute; the result is the same.  The staging area is shared: calls from several host threads are served one after
+ * neither a caller table nor SP_FLAG_DIE_PINNED) M is split into row blocks (2048 rows or more, the last one cut
+ * further into halves down to 256 rows so that little work is left once the last byte of A has arrived), each computed
+ * by its own sp_gemm under the same scheme applied to the block's tile grid, so that copies in both directions overlap
+ * the compute; the result is the same.  The staging area is shared: calls from several host threads are served one after
  * the other (the function holds a lock for its whole duration).  Adds SP_ERR_TIMEOUT
  * to sp_gemm's errors. */
 int sp_gemm_host(const void* A_host, const void* B_host, void* C_host, int64_t M, int64_t N, int64_t K, int scheme,
@@ -210,7 +212,10 @@ int sp_gemm_host(const void* A_host, const void* B_host, void* C_host, int64_t M
  * a tile table for non-arithmetic orders and a status word; here both live in a fixed array inside the
  * library image, so this call performs no cudaMalloc, cudaFree or other allocating call.
  *
- *   A, B, C, M, N, K, scheme, params, stream : exactly as sp_gemm (DEVICE buffers owned by the caller).
+ *   A, B, C, M, N, K, scheme, params, stream : as sp_gemm (DEVICE buffers owned by the caller), except that of the
+ *                 flags only SP_FLAG_SERPENTINE is accepted: SP_FLAG_DIE_PINNED and SP_FLAG_STREAM_K need memory that
+ *                 sp_gemm allocates, SP_FLAG_OVERLAP and SP_FLAG_CLC launches could run beside their predecessor and
+ *                 find the shared array rewritten under them (each returns SP_ERR_INVALID_ARG here).
  *   status_host : HOST, may be NULL.  NULL: the call is asynchronous and an expired device-side wait goes
  *                 unreported.  Non-NULL: the call synchronises `stream`, stores the raw status word there and
  *                 returns SP_ERR_TIMEOUT if it is non-zero.
@@ -218,8 +223,11 @@ int sp_gemm_host(const void* A_host, const void* B_host, void* C_host, int64_t M
  *   - at most 65536 tiles (ceil(M/tile_m) * ceil(N/tile_n)); more returns SP_ERR_UNSUPPORTED.  The array
  *     (about 257 KiB) is held by every GPU context that loads the library until the process exits.
  *   - every call on a device uses the same array, and the array keeps the previous call's contents: each call
- *     clears the status word and rewrites the table it needs, on `stream`, before its kernel.  Two calls that
- *     overlap on the GPU (different streams, or several host threads) race on it; serialise them.
+ *     clears the status word and, unless the array already holds exactly the table it needs (same grid, order and
+ *     parameters, or the same caller table, as the call before), rewrites the table, on `stream`, before its kernel.
+ *     Two calls that overlap on the GPU (different streams, or several host threads) race on it; serialise them.
+ *   - a new SP_CUSTOM table is uploaded from pageable host memory: that call synchronises `stream` once, whatever
+ *     status_host is; repeating the same table does not.
  *   - the first call on each device looks up the array's device address (with that device current);
  *     make that first call outside any stream capture.
  * Errors: as sp_gemm, plus SP_ERR_UNSUPPORTED for too many tiles. */
@@ -261,11 +269,11 @@ int sp_stencil2d(const void* in, void* out, int64_t M, int64_t N, float c_center
  * The paper arrives at a remap by searching with measurements in the loop; this is the short table that this
  * library's own sweeps on B200 distil to (no counterpart in the paper, and no substitute for measuring: the search
  * loop of the Python package does that).  Rule: among the supported tiles, the one with the least estimated time
- * waves x tile area / (CTAs per tile x relative efficiency of the tile shape), waves = ceil(T / units), units = 74 CTA
- * pairs or 148 CTAs; row-major when A and B together are at most 64 MiB (they stay in L2) or the tile grid is at most
+ * waves x tile area / (CTAs per tile x relative efficiency of the tile shape), waves = ceil(T / units), units = what
+ * sp_gemm_units reports on the current device, or, with no device present, 74 CTA pairs / 148 CTAs; row-major when A and B together are at most 64 MiB (they stay in L2) or the tile grid is at most
  * ten tiles wide, column-major when it is at most ten tiles tall, else bands of 8 tile columns (256x512 tile) or 8
  * tile rows (other tiles); SP_FLAG_STREAM_K is set when the tiles fill at most half of the units and K is at least
- * 2048 (C then differs in rounding order from a launch without the flag).  Host only; no GPU needed.
+ * 2048 (C then differs in rounding order from a launch without the flag).  Host code; no GPU needed.
  *   params : HOST, receives a complete sp_params (struct_size, tile_m, tile_n, group, out_dtype, b_layout set; the
  *            rest zero).   scheme : HOST, receives the sp_scheme.
  * Errors: SP_ERR_INVALID_ARG (NULL, sizes <= 0, bad out_dtype / b_layout). */

@@ -16,7 +16,7 @@ from typing import Optional, Sequence
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.environ.get("SWIZZLEPERF_LIB") or os.path.join(_HERE, "libswizzleperf.so")
+LIB_PATH = os.path.join(_HERE, "libswizzleperf.so")
 
 # sp_status
 OK, ERR_INVALID_ARG, ERR_NOT_BIJECTIVE, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_CUDA, ERR_TIMEOUT, ERR_DEVICE = range(8)

@@ -27,15 +27,14 @@ def _stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False, defines=(), out: str = LIB) -> str:
-    """Compile the library if it is missing or older than its sources; returns its path.
-    `defines` / `out` build a variant (kernel experiments) beside the default library."""
-    if out == LIB and not force and not _stale():
+def build(force: bool = False, verbose: bool = False) -> str:
+    """Compile the library if it is missing or older than its sources; returns its path."""
+    if not force and not _stale():
         return LIB
+    out = LIB
     tmp = out + f".tmp{os.getpid()}"
     cmd = [_nvcc(), "-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
            "-Xcompiler", "-fPIC", "-shared", "-cudart", "static", "-o", tmp]
-    cmd += [f"-D{d}" for d in defines]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += [os.path.join(CSRC, s) for s in SOURCES]

@@ -3,6 +3,7 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <deque>
 #include <mutex>
 #include <vector>
 
@@ -167,7 +168,7 @@ struct DeviceState {
 };
 
 static std::mutex g_mu;
-static std::vector<DeviceState> g_devs;
+static std::deque<DeviceState> g_devs;   // a deque: entries keep their address when another device is added
 static uint64_t g_stamp = 0;
 constexpr size_t kMaxTables = 64;
 
@@ -176,13 +177,13 @@ constexpr int kDiePairs = 64;   // die-pinned launches that may be in flight at 
 static std::mutex g_valid_mu;
 static std::vector<Sched> g_validated;
 
-static bool already_validated(const Sched& c) {
+bool already_validated(const Sched& c) {
   std::lock_guard<std::mutex> lock(g_valid_mu);
   for (const Sched& v : g_validated) if (memcmp(&v, &c, sizeof c) == 0) return true;
   return false;
 }
 
-static void remember_validated(const Sched& c) {
+void remember_validated(const Sched& c) {
   std::lock_guard<std::mutex> lock(g_valid_mu);
   if (g_validated.size() >= 256) g_validated.erase(g_validated.begin());
   g_validated.push_back(c);
@@ -210,7 +211,7 @@ static uint64_t fnv(const int32_t* v, int n) {
     }                                                                             \
   } while (0)
 
-static int current_device(int* dev) {
+int current_device(int* dev) {
   // the checks below are per (host thread, device): once passed, a call costs one cudaGetDevice
   static thread_local int checked_dev = -1;
   if (checked_dev >= 0) {
@@ -273,10 +274,11 @@ static int get_die_map(DeviceState* ds) {
   return SP_OK;
 }
 
-// Device table for a table scheme; built by the device builder (or copied for SP_CUSTOM).
+// Device table for a table scheme; built by the device builder (or copied for SP_CUSTOM).  The build runs once per
+// table and is complete when this returns: an entry is published in the cache only after the stream that filled it
+// has been synchronised, so a later call on any stream or host thread that finds it may launch at once.
 static int get_table(DeviceState* ds, const Sched& c, const std::vector<int32_t>& host_perm, bool is_custom,
-                     cudaStream_t stream, const int32_t** out, bool* built_now = nullptr) {
-  if (built_now) *built_now = false;
+                     cudaStream_t stream, const int32_t** out) {
   const uint64_t h = is_custom ? fnv(host_perm.data(), c.T) : 0;
   for (auto& e : ds->tables)
     if (memcmp(&e.key, &c, sizeof c) == 0 && e.custom_hash == h) { e.stamp = ++g_stamp; *out = e.dev; return SP_OK; }
@@ -289,16 +291,13 @@ static int get_table(DeviceState* ds, const Sched& c, const std::vector<int32_t>
   TableEntry e;
   e.key = c; e.custom_hash = h; e.stamp = ++g_stamp; e.dev = nullptr;
   SP_CUDA(cudaMalloc(&e.dev, sizeof(int32_t) * (size_t)c.T));
-  if (is_custom) {
-    // pageable source: the copy has been staged when the call returns, so host_perm may die
-    cudaError_t ce = cudaMemcpyAsync(e.dev, host_perm.data(), sizeof(int32_t) * (size_t)c.T, cudaMemcpyHostToDevice, stream);
-    if (ce == cudaSuccess) ce = cudaStreamSynchronize(stream);
-    if (ce != cudaSuccess) { cudaFree(e.dev); set_error("table upload failed: %s", cudaGetErrorString(ce)); return SP_ERR_CUDA; }
-  } else {
-    cudaError_t ce = launch_build_perm(c, e.dev, stream);
-    if (ce != cudaSuccess) { cudaFree(e.dev); set_error("table build failed: %s", cudaGetErrorString(ce)); return SP_ERR_CUDA; }
-    if (built_now) *built_now = true;   // a kernel on `stream` is writing the table: the GEMM must be ordered after it
-  }
+  cudaError_t ce;
+  if (is_custom)   // pageable source: the copy has been staged when the call returns, so host_perm may die
+    ce = cudaMemcpyAsync(e.dev, host_perm.data(), sizeof(int32_t) * (size_t)c.T, cudaMemcpyHostToDevice, stream);
+  else
+    ce = launch_build_perm(c, e.dev, stream);
+  if (ce == cudaSuccess) ce = cudaStreamSynchronize(stream);
+  if (ce != cudaSuccess) { cudaFree(e.dev); set_error("filling the tile table failed: %s", cudaGetErrorString(ce)); return SP_ERR_CUDA; }
   ds->tables.push_back(e);
   *out = e.dev;
   return SP_OK;
@@ -362,9 +361,8 @@ static int gemm_common(const void* A, const void* B, void* C, int64_t M, int64_t
   call.trace_dev = want_trace ? trace : nullptr;
   call.stream = (cudaStream_t)stream;
   call.perm_dev = nullptr;
-  bool table_built_now = false;
   if (call.sched.use_table) {
-    rc = get_table(ds, call.sched, host_perm, scheme == kCustom, call.stream, &call.perm_dev, &table_built_now);
+    rc = get_table(ds, call.sched, host_perm, scheme == kCustom, call.stream, &call.perm_dev);
     if (rc != SP_OK) return rc;
   }
   if (params && (params->flags & SP_FLAG_OVERLAP)) {
@@ -372,7 +370,7 @@ static int gemm_common(const void* A, const void* B, void* C, int64_t M, int64_t
       set_error("SP_FLAG_OVERLAP cannot be combined with tracing, SP_FLAG_DIE_PINNED or SP_FLAG_STREAM_K");
       return SP_ERR_INVALID_ARG;
     }
-    call.overlap = table_built_now ? 0 : 1;
+    call.overlap = 1;
   }
   if (params && (params->flags & SP_FLAG_DIE_PINNED)) {
     if (scheme != kDieSplit || call.sched.interleave) {
@@ -541,12 +539,28 @@ int sp_gemm_host(const void* A_host, const void* B_host, void* C_host, int64_t M
   }
   cudaStream_t st = (cudaStream_t)stream;
   // Row blocks of C are independent: with at least two of them the copy of the next block of A and the copy-out of the
-  // previous block of C overlap the compute of the current one (both PCIe directions busy at once).  Caller tables and
+  // previous block of C overlap the compute of the current one (both PCIe directions busy at once).  The copies in
+  // are the long pole (A and B together are twice the bytes of C), so what counts is how soon after the last byte of A
+  // has landed the last byte of C leaves: the last block is cut into ever smaller ones (halves, down to 256 rows), so
+  // that only a sliver of compute and of copy-out is left behind the end of the copies in.  Caller tables and
   // die-pinned orders describe the whole grid, so they take the unsplit path.
-  int64_t rows = 2048;
-  while ((M + rows - 1) / rows > kHostChunks) rows *= 2;
-  const int n_chunks = (int)((M + rows - 1) / rows);
-  const bool split = n_chunks >= 2 && scheme != kCustom && !(params && (params->flags & SP_FLAG_DIE_PINNED));
+  int64_t blk = 2048;
+  while ((M + blk - 1) / blk > kHostChunks - 3) blk *= 2;
+  int64_t row_start[kHostChunks + 1];
+  int n_chunks = 0;
+  {
+    int64_t r = 0;
+    while (M - r > blk) { row_start[n_chunks++] = r; r += blk; }
+    int64_t rem = M - r;                                   // the last block, at most blk rows
+    while (rem > 256 && n_chunks < kHostChunks - 1) {
+      const int64_t h = ((rem + 1) / 2 + 255) / 256 * 256;
+      if (h >= rem) break;
+      row_start[n_chunks++] = r; r += h; rem -= h;
+    }
+    row_start[n_chunks++] = r;
+    row_start[n_chunks] = M;
+  }
+  const bool split = M >= 4096 && scheme != kCustom && !(params && (params->flags & SP_FLAG_DIE_PINNED));
   if (!split) {
     SP_CUDA(cudaMemcpyAsync(dA, A_host, a_bytes, cudaMemcpyHostToDevice, st));
     SP_CUDA(cudaMemcpyAsync(dB, B_host, b_bytes, cudaMemcpyHostToDevice, st));
@@ -574,14 +588,14 @@ int sp_gemm_host(const void* A_host, const void* B_host, void* C_host, int64_t M
   SP_CUDA(cudaMemcpyAsync(dB, B_host, b_bytes, cudaMemcpyHostToDevice, cin));
   SP_CUDA(cudaEventRecord(ev_b, cin));
   for (int i = 0; i < n_chunks; ++i) {
-    const int64_t r0 = (int64_t)i * rows, nr = (M - r0 < rows) ? M - r0 : rows;
+    const int64_t r0 = row_start[i], nr = row_start[i + 1] - r0;
     SP_CUDA(cudaMemcpyAsync(dA + (size_t)r0 * K * 2, (const char*)A_host + (size_t)r0 * K * 2, (size_t)nr * K * 2,
                             cudaMemcpyHostToDevice, cin));
     SP_CUDA(cudaEventRecord(ev[i], cin));
   }
   SP_CUDA(cudaStreamWaitEvent(st, ev_b, 0));
   for (int i = 0; i < n_chunks; ++i) {
-    const int64_t r0 = (int64_t)i * rows, nr = (M - r0 < rows) ? M - r0 : rows;
+    const int64_t r0 = row_start[i], nr = row_start[i + 1] - r0;
     SP_CUDA(cudaStreamWaitEvent(st, ev[i], 0));
     rc = gemm_common(dA + (size_t)r0 * K * 2, dB, dC + (size_t)r0 * N * out_elt, nr, N, K, scheme, params, stream, nullptr, false);
     if (rc != SP_OK) break;
@@ -661,6 +675,21 @@ int sp_stencil2d(const void* in, void* out, int64_t M, int64_t N, float c_center
   return launch_stencil(in, out, M, N, c_center, c_neighbor, sched, perm_dev, ds->status, (cudaStream_t)stream);
 }
 
+// Persistent units sp_gemm would launch for a tile shape: asked of the current device when there is one (parts of
+// the pool have SMs fused off), else those of a full B200 (148 SMs, one CTA each).
+static int units_or_nominal(int tile_m, int tile_n) {
+  int n = 0, dev = 0;
+  if (cudaGetDeviceCount(&n) == cudaSuccess && n > 0) {
+    if (current_device(&dev) == SP_OK) {
+      const int u = gemm_units(tile_m, tile_n, kMaxTiles);
+      if (u > 0) return u;
+    }
+  } else {
+    cudaGetLastError();
+  }
+  return 148 / (tile_m / 128);
+}
+
 int sp_recommend(int64_t M, int64_t N, int64_t K, int32_t out_dtype, int32_t b_layout, sp_params* params, int* scheme) {
   if (!params || !scheme) { set_error("params and scheme must not be NULL"); return SP_ERR_INVALID_ARG; }
   if (M <= 0 || N <= 0 || K <= 0) { set_error("M, N, K must be positive"); return SP_ERR_INVALID_ARG; }
@@ -672,7 +701,7 @@ int sp_recommend(int64_t M, int64_t N, int64_t K, int32_t out_dtype, int32_t b_l
   double best_cost = 0;
   for (int i = 0; i < 5; ++i) {
     const int64_t T = ((M + kTiles[i].tm - 1) / kTiles[i].tm) * ((N + kTiles[i].tn - 1) / kTiles[i].tn);
-    const int cg = kTiles[i].tm / 128, units = 148 / cg;
+    const int cg = kTiles[i].tm / 128, units = units_or_nominal(kTiles[i].tm, kTiles[i].tn);
     const double waves = (double)((T + units - 1) / units);
     const double cost = waves * kTiles[i].tm * kTiles[i].tn / (cg * kTiles[i].eff);
     if (i == 0 || cost < best_cost) { best = i; best_cost = cost; }   // ties keep the larger tile (listed first)
@@ -697,7 +726,7 @@ int sp_recommend(int64_t M, int64_t N, int64_t K, int32_t out_dtype, int32_t b_l
   }
   // Fewer tiles than half the units and a long k extent: the k-split puts the idle units to work (measured 1.5x at
   // 1024x1024x8192).  The sum is then taken in a different order than without the flag.
-  const int cg = params->tile_m / 128, units = 148 / cg;
+  const int units = units_or_nominal(params->tile_m, params->tile_n);
   const int64_t kblocks = (K + 63) / 64;
   if (params->tile_n <= 256 && Tm * Tn * 2 <= units && kblocks >= 32) params->flags |= SP_FLAG_STREAM_K;
   return SP_OK;

@@ -35,6 +35,18 @@ constexpr int kMaxDevices = 64;
 static std::mutex g_noalloc_mu;
 static int32_t* g_noalloc_ptr[kMaxDevices] = {};
 
+// What the table part of the array holds on each device: a call that needs the same table again (the same order on the
+// same grid, or the same caller table) neither rebuilds nor re-uploads it.  Valid under this entry point's contract
+// that calls on one device do not overlap.
+struct NoAllocTable { bool valid; Sched key; uint64_t custom_hash; };
+static NoAllocTable g_noalloc_table[kMaxDevices] = {};
+
+static uint64_t table_hash(const int32_t* v, int n) {
+  uint64_t h = 1469598103934665603ull;
+  for (int i = 0; i < n; ++i) { h ^= (uint32_t)v[i]; h *= 1099511628211ull; }
+  return h;
+}
+
 // Device address of the scratch array on the current device; looked up on first use.
 static int noalloc_scratch(int dev, int32_t** out) {
   if (dev < 0 || dev >= kMaxDevices) { set_error("device index %d out of range", dev); return SP_ERR_DEVICE; }
@@ -62,16 +74,10 @@ extern "C" int sp_gemm_noalloc(const void* A, const void* B, void* C, int64_t M,
   int rc = validate_gemm_args(A, B, C, M, N, K, params, &tile_m, &tile_n, &out_f32, &b_nk);
   if (rc != SP_OK) return rc;
 
-  if (params && (params->flags & SP_FLAG_STREAM_K)) {
-    set_error("SP_FLAG_STREAM_K needs a workspace and is not available in sp_gemm_noalloc");
-    return SP_ERR_INVALID_ARG;
-  }
-  if (params && (params->flags & SP_FLAG_CLC)) {
-    set_error("SP_FLAG_CLC is not available in sp_gemm_noalloc");
-    return SP_ERR_INVALID_ARG;
-  }
-  if (params && (params->flags & SP_FLAG_OVERLAP)) {
-    set_error("SP_FLAG_OVERLAP is not available in sp_gemm_noalloc (its scratch is rewritten by every call)");
+  if (params && (params->flags & (SP_FLAG_STREAM_K | SP_FLAG_CLC | SP_FLAG_OVERLAP | SP_FLAG_DIE_PINNED))) {
+    // STREAM_K needs a workspace and DIE_PINNED its counters (both allocated by sp_gemm); OVERLAP and CLC launches may
+    // run beside the call before them, which would rewrite the shared array under a running kernel
+    set_error("sp_gemm_noalloc accepts no flag other than SP_FLAG_SERPENTINE (got 0x%x)", params->flags);
     return SP_ERR_INVALID_ARG;
   }
   GemmCall call;
@@ -83,14 +89,18 @@ extern "C" int sp_gemm_noalloc(const void* A, const void* B, void* C, int64_t M,
               kNoAllocMaxTiles, call.sched.T);
     return SP_ERR_UNSUPPORTED;
   }
-  std::vector<int32_t> host_perm;   // host memory only; the bijectivity gate of every entry point
-  rc = build_perm_host(call.sched, params ? params->custom_perm : nullptr, host_perm);
-  if (rc != SP_OK) return rc;
+  // The bijectivity gate of every entry point, in host memory only.  An order that passed once on this grid is
+  // remembered; a caller table is checked on every call (its contents may have changed).
+  std::vector<int32_t> host_perm;
+  if (scheme == kCustom || !already_validated(call.sched)) {
+    rc = build_perm_host(call.sched, params ? params->custom_perm : nullptr, host_perm);
+    if (rc != SP_OK) return rc;
+    if (scheme != kCustom) remember_validated(call.sched);
+  }
 
-  int ndev = 0, dev = 0;
-  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) { cudaGetLastError(); set_error("no CUDA device"); return SP_ERR_DEVICE; }
-  if (cudaGetDevice(&dev) != cudaSuccess) { set_error("cudaGetDevice failed"); return SP_ERR_CUDA; }
-  if (cudaSetDevice(dev) != cudaSuccess) { set_error("cudaSetDevice failed"); return SP_ERR_CUDA; }   // binds the context to this thread (no allocation)
+  int dev = 0;
+  rc = current_device(&dev);   // device present, sm_100, context bound to this thread: no allocation
+  if (rc != SP_OK) return rc;
   int32_t* scratch = nullptr;
   rc = noalloc_scratch(dev, &scratch);
   if (rc != SP_OK) return rc;
@@ -104,13 +114,27 @@ extern "C" int sp_gemm_noalloc(const void* A, const void* B, void* C, int64_t M,
   if (e != cudaSuccess) { set_error("clearing the status word failed: %s", cudaGetErrorString(e)); return SP_ERR_CUDA; }
   call.perm_dev = nullptr;
   if (call.sched.use_table) {
-    if (scheme == kCustom) {
-      e = cudaMemcpyAsync(table_dev, host_perm.data(), sizeof(int32_t) * (size_t)call.sched.T, cudaMemcpyHostToDevice, st);
-      if (e == cudaSuccess) e = cudaStreamSynchronize(st);   // host_perm is pageable and dies with this call
-    } else {
-      e = launch_build_perm(call.sched, table_dev, st);
+    const uint64_t h = scheme == kCustom ? table_hash(host_perm.data(), call.sched.T) : 0;
+    bool have;
+    {
+      std::lock_guard<std::mutex> lock(g_noalloc_mu);
+      const NoAllocTable& t = g_noalloc_table[dev];
+      have = t.valid && memcmp(&t.key, &call.sched, sizeof(Sched)) == 0 && t.custom_hash == h;
+      g_noalloc_table[dev].valid = false;   // until the new contents are queued
     }
-    if (e != cudaSuccess) { set_error("filling the tile table failed: %s", cudaGetErrorString(e)); return SP_ERR_CUDA; }
+    if (!have) {
+      if (scheme == kCustom) {
+        e = cudaMemcpyAsync(table_dev, host_perm.data(), sizeof(int32_t) * (size_t)call.sched.T, cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(st);   // host_perm is pageable and dies with this call
+      } else {
+        e = launch_build_perm(call.sched, table_dev, st);
+      }
+      if (e != cudaSuccess) { set_error("filling the tile table failed: %s", cudaGetErrorString(e)); return SP_ERR_CUDA; }
+    }
+    {
+      std::lock_guard<std::mutex> lock(g_noalloc_mu);
+      g_noalloc_table[dev].key = call.sched; g_noalloc_table[dev].custom_hash = h; g_noalloc_table[dev].valid = true;
+    }
     call.perm_dev = table_dev;
   }
   call.A = A; call.B = B; call.C = C; call.M = M; call.N = N; call.K = K;

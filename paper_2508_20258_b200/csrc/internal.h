@@ -33,6 +33,10 @@ inline bool first_use_on_this_device(uint64_t& done_mask) {
   return true;
 }
 
+// The current device, after checking (once per host thread and device) that it exists, is sm_100 and has its primary
+// context bound to this thread.  Returns an sp_status.  Allocates nothing.
+int current_device(int* dev);
+
 // Validates sizes and parameters and fills `out`.  Returns an sp_status.
 int resolve_sched(int64_t M, int64_t N, int32_t tileM, int32_t tileN, int scheme, const sp_params* params, Sched* out);
 
@@ -44,6 +48,10 @@ int validate_gemm_args(const void* A, const void* B, const void* C, int64_t M, i
 // Evaluates the remap on the host (closed forms, curve walks, caller table) and checks
 // that it is a bijection.  Returns SP_OK or SP_ERR_NOT_BIJECTIVE / SP_ERR_INVALID_ARG.
 int build_perm_host(const Sched& sched, const int32_t* custom, std::vector<int32_t>& perm);
+
+// Orders (grid, scheme, parameters) that have passed the bijectivity gate, so that repeated calls do no O(T) host work.
+bool already_validated(const Sched& c);
+void remember_validated(const Sched& c);
 
 // Device evaluation of the same remap into out_dev (T entries).  Not valid for kCustom.
 cudaError_t launch_build_perm(const Sched& sched, int32_t* out_dev, cudaStream_t stream);

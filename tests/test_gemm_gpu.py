@@ -460,3 +460,32 @@ def test_host_entry_point_from_two_threads():
     for (_, _, ref, outs) in jobs:
         for o in outs:
             assert np.array_equal(o.astype(np.float64), ref)
+
+
+def test_table_built_on_one_stream_is_complete_for_the_next_stream():
+    """First use of a table order on stream X, and at once the same order on stream Y: the second call finds the
+    table in the cache and launches without waiting for X, so the table must have been complete before it was
+    published.  Fresh grid shapes (used nowhere else in this suite), so the build really happens here; X is kept busy
+    beforehand so that an unfinished build would still be queued when Y's kernel reads the table."""
+    sx, sy = torch.cuda.Stream(), torch.cuda.Stream()
+    big = torch.empty(1 << 28, dtype=torch.uint8, device="cuda")
+    for (M, N, K, tile, scheme, kw) in [(128 * 19, 128 * 23, 264, (128, 128), sp.HILBERT, {}),
+                                        (256 * 9, 256 * 11, 200, (256, 256), sp.HILBERT_RECT, {}),
+                                        (128 * 21, 256 * 7, 136, (128, 256), sp.DIE_SPLIT, dict(inner_scheme=sp.MORTON))]:
+        A, B = synth.make_inputs(M, N, K, "normal", 1.0, seed=31)
+        dA, dB = dev_bf16(A), dev_bf16(B)
+        want = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        sp.gemm(dA, dB, want, sp.ROW_MAJOR, sp.make_params(tile_m=tile[0], tile_n=tile[1]))
+        cx = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+        cy = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+        torch.cuda.synchronize()
+        p = sp.make_params(tile_m=tile[0], tile_n=tile[1], **kw)
+        with torch.cuda.stream(sx):
+            for _ in range(8):
+                big.fill_(1)                                 # about a millisecond of queued work ahead of the build
+        sp.gemm(dA, dB, cx, scheme, p, sx)
+        sp.gemm(dA, dB, cy, scheme, p, sy)
+        torch.cuda.synchronize()
+        assert sp.get_status() == 0
+        assert torch.equal(cx.view(torch.int16), want.view(torch.int16))
+        assert torch.equal(cy.view(torch.int16), want.view(torch.int16))

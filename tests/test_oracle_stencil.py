@@ -73,3 +73,19 @@ def test_grids_without_interior_are_copied(shape):
     x = np.arange(shape[0] * shape[1], dtype=np.float64).reshape(shape)
     assert np.array_equal(S.stencil2d(x, 9.0, 9.0), x)
     assert np.array_equal(S.stencil2d_points(x, 9.0, 9.0), x)
+
+
+def test_magnitude_hand_case():
+    """The error scale of the GPU tolerance, on a 3 x 3 grid worked by hand: the one interior point gets
+    |c0||x11| + |c1|(|x01| + |x21| + |x10| + |x12|) = 0.5 * 5 + 0.25 * (2 + 8 + 4 + 6) = 7.5 (signs of the inputs
+    and of the weights dropped), the rim its own absolute value."""
+    x = np.array([[1.0, -2.0, 3.0], [-4.0, 5.0, -6.0], [7.0, -8.0, 9.0]])
+    m = S.magnitude(x, -0.5, 0.25)
+    want = np.abs(x)
+    want[1, 1] = 7.5
+    assert np.array_equal(m, want)
+    # the plain stencil of the same grid cancels instead: -0.5 * 5 + 0.25 * (-2 - 8 - 4 - 6) = -7.5
+    assert S.stencil2d(x, -0.5, 0.25)[1, 1] == -7.5
+    # and with weights of one sign on a grid of one sign, magnitude and stencil coincide
+    y = np.abs(x)
+    assert np.array_equal(S.magnitude(y, 0.5, 0.25), S.stencil2d(y, 0.5, 0.25))
