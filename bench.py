@@ -55,6 +55,15 @@ def parse_scheme(spec: str):
         scheme, kw = parse_scheme(spec[:-2])
         kw["flags"] = kw.get("flags", 0) | sp.FLAG_CLC
         return scheme, kw
+    for suffix, bit in (("+hc", 128), ("+ha", 256), ("+hb", 512), ("+ka", 1024), ("+kb", 2048)):
+        if spec.endswith(suffix):    # L2 eviction hints: C / A / B evict_first, A / B evict_last
+            scheme, kw = parse_scheme(spec[:-len(suffix)])
+            kw["flags"] = kw.get("flags", 0) | bit
+            return scheme, kw
+    if spec.endswith("+a"):    # any order, every other tile of a unit walks K from the far end
+        scheme, kw = parse_scheme(spec[:-2])
+        kw["flags"] = kw.get("flags", 0) | sp.FLAG_K_ALTERNATE
+        return scheme, kw
     if spec.endswith("+o"):    # any order, launches declared independent of their predecessor (they overlap its tail)
         scheme, kw = parse_scheme(spec[:-2])
         kw["flags"] = kw.get("flags", 0) | sp.FLAG_OVERLAP
@@ -108,11 +117,12 @@ SWEEPS = {
 DEFAULT_SCHEME = {"cfg1": "group_m:2", "cfg2": "group_m:8", "cfg3": "die_split:m:group_m:8:p", "cfg4": "row_major",
                   "cfg5": "die_split:m:group_m:8:p"}
 FALLBACK_SCHEME = {"cfg3": "group_m:8", "cfg5": "group_m:16"}   # if the topology probe finds no two-way L2 structure
+FALLBACK_SCHEME_BY_TILE = {("cfg3", "256x512"): "group_m:16:s+a+hc", ("cfg5", "256x512"): "group_m:16:s+a+hc"}
 # 8192^3 is timed with two 256x256 2-CTA MMA tiles per scheduler tile (they share the A panel: a quarter less operand
 # traffic from L2); the plain 256x256 scheduler tile is timed beside it and reported in the same line.
 DEFAULT_TILE = {"cfg3": "256x512", "cfg2": "256x512",   # 4096^3: A and B fit in L2, the order hardly matters, the wider tile does
                 "cfg5": "256x512"}
-DEFAULT_SCHEME_BY_TILE = {("cfg3", "256x512"): "group_n:8", ("cfg5", "256x512"): "die_split:m:group_m:8:p",
+DEFAULT_SCHEME_BY_TILE = {("cfg3", "256x512"): "die_split:m:group_m:8:p:s+a+hc", ("cfg5", "256x512"): "die_split:m:group_m:8:p:s+a+hc",
                           ("cfg2", "256x512"): "row_major"}
 
 
@@ -203,7 +213,7 @@ def sustained_leg(fn, flops, stream, gpu_index, seconds=4.0):
 
 def workloads_block(sp, names, peaks, stream):
     """The other named workloads, each timed briefly in the same process: the fastest known (tile, order) for it beside
-    row-major on the same tile (alternating blocks, median of three), and the workload's nominal tile when that is another
+    row-major on the same tile (alternating blocks of a quarter of a second, mean of two), and the workload's nominal tile when that is another
     one.  For the launch-bound 512^3 also what a call costs on the host and how long one launch takes from call to
     completion."""
     import torch
@@ -232,7 +242,7 @@ def workloads_block(sp, names, peaks, stream):
                     raise
                 return False
         if not usable(tile, spec):
-            spec = FALLBACK_SCHEME.get(name, "row_major")
+            spec = FALLBACK_SCHEME_BY_TILE.get((name, tile)) or FALLBACK_SCHEME.get(name, "row_major")
         arms = [("best", tile, spec), ("row_major", tile, "row_major")]
         nominal_tile = f"{w.tile_m}x{w.tile_n}"
         if nominal_tile != tile:
@@ -242,14 +252,17 @@ def workloads_block(sp, names, peaks, stream):
             for _ in range(3):
                 sp.gemm(dA, dB, dC, *arm(t_, s_), stream)
         est = time_steps(sp, dA, dB, dC, *arm(tile, spec), 5, stream) / 5
-        n = int(max(10, min(2000, 40.0 / est)))
+        # blocks of about 0.25 s: long enough for the power limiter to act, which is where a tile order's saved DRAM
+        # traffic turns into clock and time (in a burst of a few milliseconds every order runs at the full clock)
+        n = int(max(10, min(20000, 250.0 / est)))
         ms = {k: [] for k, _, _ in arms}
-        for _ in range(3):
+        for _ in range(2):
             for k, t_, s_ in arms:
                 ms[k].append(time_steps(sp, dA, dB, dC, *arm(t_, s_), n, stream) / n)
-        med = {k: sorted(v)[1] for k, v in ms.items()}
+        med = {k: sum(v) / len(v) for k, v in ms.items()}
         rec = {"shape": [w.M, w.N, w.K], "out": w.out_dtype, "tile": tile, "scheme": spec, "launches_per_block": n,
-               "ms": med["best"], "tflops": flops / med["best"] / 1e9, "frac_of_burst_peak": flops / med["best"] / 1e9 / peaks["bf16_tflops"],
+               "ms": med["best"], "tflops": flops / med["best"] / 1e9,
+               "frac_of_sustained_peak": flops / med["best"] / 1e9 / peaks["bf16_tflops_sustained"],
                "row_major_tflops": flops / med["row_major"] / 1e9, "speedup_over_row_major": med["row_major"] / med["best"]}
         if "nominal_tile" in med:
             rec["nominal_tile"] = {"tile": nominal_tile, "scheme": arms[2][2], "tflops": flops / med["nominal_tile"] / 1e9}
@@ -370,7 +383,7 @@ def run_ours(args) -> int:
     except sp.SpError as err:
         if args.scheme or err.status != sp.ERR_UNSUPPORTED or args.workload not in FALLBACK_SCHEME:
             raise
-        spec = FALLBACK_SCHEME[args.workload]
+        spec = FALLBACK_SCHEME_BY_TILE.get((args.workload, f"{tile_m}x{tile_n}")) or FALLBACK_SCHEME[args.workload]
         scheme, p = params_for(spec)
     tile_s = f"{tile_m}x{tile_n}"
     traffic = None
@@ -380,6 +393,7 @@ def run_ours(args) -> int:
             raise SystemExit(f"no profiler capture of DRAM traffic for ({w.name}, {tile_s}, {spec}): capture it (ncu over "
                              f"`bench.py --profile-sweep`, then `python -m paper_2508_20258_b200.ncuparse --sweep ... --traffic`) "
                              f"or pass --no-traffic to report roofline.traffic as null")
+    sampler = None if args.kernel_only else benchutil.ClockSampler(local_rank, period_s=0.002).start()   # before the warm-up: no idle gap later
     for _ in range(max(args.warmup, 3)):
         sp.gemm(dA, dB, dC, scheme, p, stream)
     torch.cuda.synchronize()
@@ -390,7 +404,6 @@ def run_ours(args) -> int:
                           "ms_per_step": ms / args.steps, "tflops": flops * args.steps / ms / 1e9}), flush=True)
         return 0
 
-    sampler = benchutil.ClockSampler(local_rank, period_s=0.002).start()
     barrier()
     t_host0 = time.perf_counter()
     ms_total = time_steps(sp, dA, dB, dC, scheme, p, args.steps, stream)

@@ -113,6 +113,29 @@ typedef enum {
                                  SP_FLAG_STREAM_K or tracing (SP_ERR_INVALID_ARG).  It still completes after its predecessor, so the
                                  stream order seen by everything else (copies, events, other kernels) is unchanged. */
 
+#define SP_FLAG_K_ALTERNATE 64u /* sp_gemm* only.  Every other tile a persistent unit works on walks the K dimension from the
+                                 far end (k-blocks in descending order).  The tiles of one round advance through K in step, so
+                                 what L2 holds when a round ends is the end of the K range of that round's operand panels; a
+                                 round that shares panels with it and starts there finds them still cached, where a round
+                                 that starts over at k = 0 finds them evicted: fewer DRAM reads (a fifth fewer at 8192^3 under
+                                 bands of eight) and, at the power limit, less time.  The paper has no counterpart: its remap
+                                 chooses which tile a block computes, never the order inside a tile.  C = A.B as before, but
+                                 the fp32 sum of a tile is taken in the order its k-blocks arrive, so the rounding of C
+                                 depends on which round a tile ran in, hence on the order and the unit count (like
+                                 SP_FLAG_STREAM_K, and within the same tolerance); with exactly representable partial sums
+                                 (small integers) C has the same bits either way.  Combines with every scheme and flag. */
+
+/* sp_gemm* only.  L2 eviction priorities for the lines a GEMM's bulk copies bring in or write (the
+ * paper has no counterpart: its lever is which block runs where, not what the cache keeps).  evict_first marks lines as
+ * the first to go when room is needed (an operand that is streamed once per band, C tiles that are written and never
+ * read), evict_last as lines to keep (the operand panels a band of tiles shares from round to round).  Results are
+ * unchanged; only the cache's replacement choices are.  A and B may each be given at most one of the two. */
+#define SP_FLAG_HINT_C_EVICT_FIRST 128u
+#define SP_FLAG_HINT_A_EVICT_FIRST 256u
+#define SP_FLAG_HINT_B_EVICT_FIRST 512u
+#define SP_FLAG_HINT_A_EVICT_LAST 1024u
+#define SP_FLAG_HINT_B_EVICT_LAST 2048u
+
 typedef struct {
   uint32_t struct_size;       /* must be sizeof(sp_params)                                                  */
   int32_t group;              /* G >= 1 for SP_GROUP_M / SP_GROUP_N                                         */
@@ -129,7 +152,7 @@ typedef struct {
                               /*   the A panel); 0,0 = 256x256.  Ignored by sp_tile_map*.                    */
   int32_t out_dtype;          /* sp_gemm*: 0 = C is bf16 (round to nearest even), 1 = C is fp32             */
   int32_t b_layout;           /* sp_gemm*: 0 = B is K x N row-major, 1 = B is N x K row-major               */
-  uint32_t flags;             /* 0, or any of SP_FLAG_DIE_PINNED, _SERPENTINE, _STREAM_K, _OVERLAP, _CLC      */
+  uint32_t flags;             /* 0, or any of SP_FLAG_DIE_PINNED, _SERPENTINE, _STREAM_K, _OVERLAP, _CLC, _K_ALTERNATE, _HINT_* */
 } sp_params;
 
 /* One record per tile, written by sp_gemm_trace. */
@@ -213,7 +236,7 @@ int sp_gemm_host(const void* A_host, const void* B_host, void* C_host, int64_t M
  * library image, so this call performs no cudaMalloc, cudaFree or other allocating call.
  *
  *   A, B, C, M, N, K, scheme, params, stream : as sp_gemm (DEVICE buffers owned by the caller), except that of the
- *                 flags only SP_FLAG_SERPENTINE is accepted: SP_FLAG_DIE_PINNED and SP_FLAG_STREAM_K need memory that
+ *                 flags only SP_FLAG_SERPENTINE, SP_FLAG_K_ALTERNATE and SP_FLAG_HINT_* are accepted: SP_FLAG_DIE_PINNED and SP_FLAG_STREAM_K need memory that
  *                 sp_gemm allocates, SP_FLAG_OVERLAP and SP_FLAG_CLC launches could run beside their predecessor and
  *                 find the shared array rewritten under them (each returns SP_ERR_INVALID_ARG here).
  *   status_host : HOST, may be NULL.  NULL: the call is asynchronous and an expired device-side wait goes

@@ -328,6 +328,24 @@ int validate_gemm_args(const void* A, const void* B, const void* C, int64_t M, i
   return SP_OK;
 }
 
+// The flags that change only how memory is walked or cached (no scratch memory, no scheduling state): K direction per
+// round and L2 eviction priorities.  Shared by every GEMM entry point.
+int apply_memory_flags(const sp_params* params, GemmCall* call) {
+  call->k_alternate = 0; call->hint_a = call->hint_b = call->hint_c = 0;
+  if (!params) return SP_OK;
+  const uint32_t f = params->flags;
+  if (((f & SP_FLAG_HINT_A_EVICT_FIRST) && (f & SP_FLAG_HINT_A_EVICT_LAST)) ||
+      ((f & SP_FLAG_HINT_B_EVICT_FIRST) && (f & SP_FLAG_HINT_B_EVICT_LAST))) {
+    set_error("an operand cannot be both evict_first and evict_last");
+    return SP_ERR_INVALID_ARG;
+  }
+  call->k_alternate = (f & SP_FLAG_K_ALTERNATE) ? 1 : 0;
+  call->hint_a = (f & SP_FLAG_HINT_A_EVICT_FIRST) ? 1 : (f & SP_FLAG_HINT_A_EVICT_LAST) ? 2 : 0;
+  call->hint_b = (f & SP_FLAG_HINT_B_EVICT_FIRST) ? 1 : (f & SP_FLAG_HINT_B_EVICT_LAST) ? 2 : 0;
+  call->hint_c = (f & SP_FLAG_HINT_C_EVICT_FIRST) ? 1 : 0;
+  return SP_OK;
+}
+
 static int gemm_common(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t K, int scheme,
                        const sp_params* params, void* stream, sp_trace_rec* trace, bool want_trace) {
   if (want_trace && !trace) { set_error("trace buffer must not be NULL"); return SP_ERR_INVALID_ARG; }
@@ -365,6 +383,8 @@ static int gemm_common(const void* A, const void* B, void* C, int64_t M, int64_t
     rc = get_table(ds, call.sched, host_perm, scheme == kCustom, call.stream, &call.perm_dev);
     if (rc != SP_OK) return rc;
   }
+  rc = apply_memory_flags(params, &call);
+  if (rc != SP_OK) return rc;
   if (params && (params->flags & SP_FLAG_OVERLAP)) {
     if (want_trace || (params->flags & (SP_FLAG_DIE_PINNED | SP_FLAG_STREAM_K))) {
       set_error("SP_FLAG_OVERLAP cannot be combined with tracing, SP_FLAG_DIE_PINNED or SP_FLAG_STREAM_K");

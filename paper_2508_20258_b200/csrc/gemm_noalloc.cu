@@ -77,7 +77,7 @@ extern "C" int sp_gemm_noalloc(const void* A, const void* B, void* C, int64_t M,
   if (params && (params->flags & (SP_FLAG_STREAM_K | SP_FLAG_CLC | SP_FLAG_OVERLAP | SP_FLAG_DIE_PINNED))) {
     // STREAM_K needs a workspace and DIE_PINNED its counters (both allocated by sp_gemm); OVERLAP and CLC launches may
     // run beside the call before them, which would rewrite the shared array under a running kernel
-    set_error("sp_gemm_noalloc accepts no flag other than SP_FLAG_SERPENTINE (got 0x%x)", params->flags);
+    set_error("sp_gemm_noalloc accepts SP_FLAG_SERPENTINE, SP_FLAG_K_ALTERNATE and SP_FLAG_HINT_* only (got 0x%x)", params->flags);
     return SP_ERR_INVALID_ARG;
   }
   GemmCall call;
@@ -141,6 +141,8 @@ extern "C" int sp_gemm_noalloc(const void* A, const void* B, void* C, int64_t M,
   call.tile_m = tile_m; call.tile_n = tile_n; call.out_f32 = out_f32; call.b_nk = b_nk;
   call.status_dev = status_dev;
   call.trace_dev = nullptr;
+  rc = apply_memory_flags(params, &call);
+  if (rc != SP_OK) return rc;
   call.stream = st;
   rc = launch_gemm(call);
   if (rc != SP_OK) return rc;

@@ -79,6 +79,8 @@ struct GemmArgs {
   int32_t* sk_flags;               // one word per (unit, cta, lane quarter): set to sk_epoch once that partial is complete
   int32_t sk_epoch;                // differs from launch to launch on one workspace, so the flags need no clearing
   int overlap;                     // 1: never waits for its predecessor before working (only before exiting)
+  int hint_a, hint_b, hint_c;      // L2 eviction priority of A loads, B loads, C stores: 0 none, 1 evict_first, 2 evict_last
+  int k_alternate;                 // 1: every other piece of work of a unit walks its k-blocks from the far end (SP_FLAG_K_ALTERNATE)
   int clc;                         // 1: one cluster per tile is launched; running clusters take over the slots of clusters
                                    //    not yet started (cluster launch control) instead of striding through the slots
   Sched sched;
@@ -230,6 +232,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
+      const bool hinted = (args.hint_a | args.hint_b) != 0;
+      const uint64_t pol_a = l2_policy(args.hint_a), pol_b = l2_policy(args.hint_b);
+      auto load_a = [&](uint32_t dst, int x, int y, uint32_t bar) {
+        if (hinted) tma_load_2d_hint<CG>(dst, &tmA, x, y, bar, pol_a); else tma_load_2d<CG>(dst, &tmA, x, y, bar);
+      };
+      auto load_b = [&](uint32_t dst, int x, int y, uint32_t bar) {
+        if (hinted) tma_load_2d_hint<CG>(dst, &tmB, x, y, bar, pol_b); else tma_load_2d<CG>(dst, &tmB, x, y, bar);
+      };
       for (int item = 0; ok; ++item) {
         const Work wk = work_at(item, (kRoleProducer << 8) | 4);
         if (wk.slot < 0) break;
@@ -255,6 +265,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const int col0 = tn * BN + (int)rank * C::kMmaCols;        // + c * kMmaN for the c-th MMA tile
         const bool tracing = args.trace != nullptr && rank == 0 && wk.kind != kWorkContrib;   // a split tile is traced by the piece that stores it
         uint32_t waited = 0;
+        // SP_FLAG_K_ALTERNATE: odd items of a unit load their k-blocks in descending order.  The tiles of one round run in
+        // step, so the round that follows starts on the k-range its predecessor touched last, which is what L2 still holds.
+        const bool k_desc = args.k_alternate && (item & 1);
         if (tracing && lane == 0) {
           sp_trace_rec* rec = args.trace + s;
           uint32_t smid;
@@ -269,18 +282,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           const uint32_t full_leader = CG == 1 ? full_local : mapa(full_local, 0);
           const uint32_t sa = smem_base + stage * C::kStageBytes;
           const uint32_t sb = sa + C::kABytes;
+          const int k_elem = (k_desc ? wk.k0 + wk.k1 - 1 - kb : kb) * kBK;
           if (elect_one()) {
             if (rank == 0) mbar_arrive_expect_tx(full_local, CG * C::kStageBytes);
-            tma_load_2d<CG>(sa, &tmA, kb * kBK, row0, full_leader);
+            load_a(sa, k_elem, row0, full_leader);
             if constexpr (B_NK) {
 #pragma unroll
               for (int c = 0; c < C::kNT; ++c)
-                tma_load_2d<CG>(sb + c * (C::kMmaCols * kBK * 2), &tmB, kb * kBK, col0 + c * C::kMmaN, full_leader);
+                load_b(sb + c * (C::kMmaCols * kBK * 2), k_elem, col0 + c * C::kMmaN, full_leader);
             } else {
 #pragma unroll
               for (int j = 0; j < C::kBCols / 64; ++j) {   // boxes of 64 columns, MMA tile by MMA tile
                 constexpr int per = C::kMmaCols / 64;
-                tma_load_2d<CG>(sb + j * (64 * kBK * 2), &tmB, col0 + (j / per) * C::kMmaN + (j % per) * 64, kb * kBK, full_leader);
+                load_b(sb + j * (64 * kBK * 2), col0 + (j / per) * C::kMmaN + (j % per) * 64, k_elem, full_leader);
               }
             }
           }
@@ -420,6 +434,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   } else {
     // ---------------------------------------------------------------- epilogue
     const int quarter = warp & 3;  // TMEM lanes [32*quarter, 32*quarter + 32) are this warp's
+    auto store_c = [&](uint32_t src, int x, int y) {   // issued by one lane
+      if (args.hint_c) tma_store_2d_hint(&tmC, src, x, y, l2_policy(args.hint_c)); else tma_store_2d(&tmC, src, x, y);
+    };
     if constexpr (C::kNT == 2) {
       // Two MMA tiles per scheduler tile: no second accumulator buffer hides this epilogue.  Four warps serve each
       // accumulator part.  A warp empties its 32 lanes x 256 columns into registers (packed bf16), hands the part back
@@ -470,7 +487,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             __syncwarp();
             if (lane == 0) {
               const int col = col_base + q * 64;
-              if (row0 < args.M && col < args.N) tma_store_2d(&tmC, slice, col, row0);
+              if (row0 < args.M && col < args.N) store_c(slice, col, row0);
               bulk_commit();
             }
           }
@@ -490,7 +507,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             __syncwarp();
             if (lane == 0) {
               const int col = col_base + q * 32;
-              if (row0 < args.M && col < args.N) tma_store_2d(&tmC, slice, col, row0);
+              if (row0 < args.M && col < args.N) store_c(slice, col, row0);
               bulk_commit();
             }
           }
@@ -631,7 +648,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           __syncwarp();
           if (lane == 0) {
             const int col = col_base + q * kChunkCols;
-            if (row0 < args.M && col < args.N) tma_store_2d(&tmC, slice, col, row0);
+            if (row0 < args.M && col < args.N) store_c(slice, col, row0);
             bulk_commit();                                            // also when nothing was stored: keeps the group count in step
           }
         }
@@ -916,6 +933,8 @@ int launch_gemm(const GemmCall& call) {
   args.sk_ws = nullptr; args.sk_flags = nullptr; args.sk_epoch = 0;
   args.overlap = call.overlap;
   args.clc = call.clc;
+  args.k_alternate = call.k_alternate;
+  args.hint_a = call.hint_a; args.hint_b = call.hint_b; args.hint_c = call.hint_c;
   if (call.stream_k) {
     // units are not capped by the tile count here: a problem smaller than a wave is spread over all of them
     const int all_units = gemm_units(call.tile_m, call.tile_n, kMaxTiles);
@@ -938,10 +957,10 @@ int launch_gemm(const GemmCall& call) {
     const int stages = cg == 1 ? (call.tile_n == 128 ? Cfg<1, 128>::kStages : Cfg<1, 256>::kStages)
                                : (call.tile_n == 128 ? Cfg<2, 128>::kStages : call.tile_n == 256 ? Cfg<2, 256>::kStages : Cfg<2, 512>::kStages);
     fprintf(stderr, "[swizzleperf] gemm %dx%dx%d tile %dx%d (%d CTA%s per tile) scheme %d T=%d units=%d grid=%d stages=%d kblocks=%d "
-                    "b=%s out=%s table=%d pinned=%d split_tail=%d/%d clc=%d overlap=%d\n",
+                    "b=%s out=%s table=%d pinned=%d split_tail=%d/%d clc=%d overlap=%d k_alternate=%d\n",
             args.M, args.N, args.K, call.tile_m, call.tile_n, cg, cg > 1 ? "s" : "", call.sched.scheme, call.sched.T, args.units,
             (args.clc ? call.sched.T : args.units) * cg, stages, args.kblocks, call.b_nk ? "NxK" : "KxN", call.out_f32 ? "fp32" : "bf16",
-            call.sched.use_table, args.pinned, args.sk.tiles, args.sk.units, args.clc, args.overlap);
+            call.sched.use_table, args.pinned, args.sk.tiles, args.sk.units, args.clc, args.overlap, args.k_alternate);
   }
   if (cg == 1) return call.tile_n == 128 ? launch_shape<1, 128>(call, tmA, tmB, tmC, args) : launch_shape<1, 256>(call, tmA, tmB, tmC, args);
   if (call.tile_n == 512) return launch_shape<2, 512>(call, tmA, tmB, tmC, args);

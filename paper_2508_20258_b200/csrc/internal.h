@@ -75,12 +75,17 @@ struct GemmCall {
   sp_trace_rec* trace_dev;  // nullptr unless tracing
   int stream_k;             // SP_FLAG_STREAM_K: split the tail wave along k
   int clc;                  // SP_FLAG_CLC: one cluster per tile, tiles of unstarted clusters taken over by running ones
+  int hint_a, hint_b, hint_c;   // SP_FLAG_HINT_*: L2 eviction priority of A loads, B loads, C stores (0 none, 1 first, 2 last)
+  int k_alternate;          // SP_FLAG_K_ALTERNATE: odd pieces of work of a unit walk k downwards
   int overlap;              // SP_FLAG_OVERLAP: launch with programmatic stream serialisation, never wait for the predecessor
   int32_t* sk_flags_dev;    // kSkFlagBytes of flags, zero when allocated
   int32_t sk_epoch;         // value the flags take in this launch: 1, 2, ... per workspace
   float* sk_ws_dev;         // kSkWorkspaceBytes of partial tiles
   cudaStream_t stream;
 };
+
+// Fills the fields of `call` that SP_FLAG_K_ALTERNATE and SP_FLAG_HINT_* set.  Returns an sp_status.
+int apply_memory_flags(const sp_params* params, GemmCall* call);
 
 // Number of persistent units (CTAs or CTA pairs) for this tile shape on the current device.
 int gemm_units(int tile_m, int tile_n, int64_t T);

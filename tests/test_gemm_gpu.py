@@ -489,3 +489,37 @@ def test_table_built_on_one_stream_is_complete_for_the_next_stream():
         assert sp.get_status() == 0
         assert torch.equal(cx.view(torch.int16), want.view(torch.int16))
         assert torch.equal(cy.view(torch.int16), want.view(torch.int16))
+
+
+@pytest.mark.parametrize("tile", [(128, 128), (128, 256), (256, 256), (256, 512)])
+def test_k_alternate_walks_every_k_block_once(tile):
+    """SP_FLAG_K_ALTERNATE: odd rounds of a unit take their k-blocks in descending order.  Small integers make every
+    partial sum exact, so C must equal the oracle bit for bit whatever the order of the k-blocks -- a k-block loaded
+    twice, skipped, or taken from the wrong end of a ragged K shows up as a wrong integer.  Grids with several rounds
+    per unit (more tiles than SMs), ragged M, N and K."""
+    M, N, K = tile[0] * 13 + 40, tile[1] * 15 + 72, 64 * 9 + 24
+    A, B = synth.make_int_inputs(M, N, K, seed=41)
+    ref, _ = G.gemm_full(A, B)
+    for scheme, kw in [(sp.GROUP_N, dict(group=8)), (sp.HILBERT, {}), (sp.ROW_MAJOR, {})]:
+        got, _ = run_gemm(A, B, scheme, tile, out="fp32", flags=sp.FLAG_K_ALTERNATE, **kw)
+        assert np.array_equal(got, ref), (scheme, tile)
+    got, _ = run_gemm(A, B, sp.GROUP_M, tile, out="fp32", b_is_nk=True, group=4, flags=sp.FLAG_K_ALTERNATE)
+    assert np.array_equal(got, ref)
+
+
+def test_k_alternate_within_tolerance_and_with_the_other_schedulers():
+    M, N, K = 256 * 11, 512 * 9 + 128, 1096
+    A, B = synth.make_inputs(M, N, K, "normal", 1.0, seed=42)
+    ref, S = G.gemm_full(A, B)
+    cases = [((256, 512), sp.GROUP_N, dict(group=8, flags=sp.FLAG_K_ALTERNATE)),
+             ((256, 256), sp.GROUP_M, dict(group=8, flags=sp.FLAG_K_ALTERNATE | sp.FLAG_STREAM_K)),
+             ((256, 256), sp.ROW_MAJOR, dict(flags=sp.FLAG_K_ALTERNATE | sp.FLAG_CLC)),
+             ((256, 512), sp.DIE_SPLIT, dict(inner_scheme=sp.GROUP_M, inner_group=4, flags=sp.FLAG_K_ALTERNATE | sp.FLAG_DIE_PINNED))]
+    for tile, scheme, kw in cases:
+        try:
+            got, _ = run_gemm(A, B, scheme, tile, **kw)
+        except sp.SpError as err:                     # die-pinned orders need the two-way L2 structure and enough tiles
+            assert err.status == sp.ERR_UNSUPPORTED and (kw["flags"] & sp.FLAG_DIE_PINNED)
+            continue
+        r = G.compare(got, ref, S)
+        assert r["max_err"] <= TOL, (tile, scheme, r)
