@@ -93,7 +93,8 @@ def parse_scheme(spec: str):
         inter = int("i" in rest)
         g = [int(v) for v in rest if v.isdigit()]
         kw = dict(split_axis=int(a[1] == "n"), inner_scheme=inner, inner_group=g[0] if g else 1, interleave=inter)
-        flags = (2 if "p" in rest else 0) | (4 if "s" in rest else 0)   # p: units pinned to their L2 half; s: serpentine
+        # p: units pinned to their L2 half; s: serpentine; t: per-half ticket queues with stealing (with p)
+        flags = (2 if "p" in rest else 0) | (4 if "s" in rest else 0) | (4096 if "t" in rest else 0)
         if flags:
             kw["flags"] = flags
         return sp.DIE_SPLIT, kw

@@ -113,6 +113,14 @@ typedef enum {
                                  SP_FLAG_STREAM_K or tracing (SP_ERR_INVALID_ARG).  It still completes after its predecessor, so the
                                  stream order seen by everything else (copies, events, other kernels) is unchanged. */
 
+#define SP_FLAG_STEAL 4096u   /* sp_gemm / sp_gemm_trace / sp_gemm_host, together with SP_FLAG_DIE_PINNED.  The slots of each half
+                                 of the tile space are handed out by ticket (one atomic per tile) to the units of that L2
+                                 half, in slot order; a unit that finds its own half's queue empty takes tickets of the other
+                                 half, so no unit idles while a tile is still waiting.  Without the flag each unit owns a
+                                 fixed stride of its half and a half that finishes early waits for the other.  Matters when
+                                 the halves hold unequal work (an odd number of tile rows, a ragged edge) or the GPU is
+                                 shared.  C has the same bits either way (every tile is computed whole, by one unit).  No
+                                 counterpart in the paper, whose blocks cannot trade work once launched. */
 #define SP_FLAG_K_ALTERNATE 64u /* sp_gemm* only.  Every other tile a persistent unit works on walks the K dimension from the
                                  far end (k-blocks in descending order).  The tiles of one round advance through K in step, so
                                  what L2 holds when a round ends is the end of the K range of that round's operand panels; a
@@ -152,7 +160,7 @@ typedef struct {
                               /*   the A panel); 0,0 = 256x256.  Ignored by sp_tile_map*.                    */
   int32_t out_dtype;          /* sp_gemm*: 0 = C is bf16 (round to nearest even), 1 = C is fp32             */
   int32_t b_layout;           /* sp_gemm*: 0 = B is K x N row-major, 1 = B is N x K row-major               */
-  uint32_t flags;             /* 0, or any of SP_FLAG_DIE_PINNED, _SERPENTINE, _STREAM_K, _OVERLAP, _CLC, _K_ALTERNATE, _HINT_* */
+  uint32_t flags;             /* 0, or any of SP_FLAG_DIE_PINNED, _SERPENTINE, _STREAM_K, _OVERLAP, _CLC, _K_ALTERNATE, _STEAL, _HINT_* */
 } sp_params;
 
 /* One record per tile, written by sp_gemm_trace. */
@@ -217,10 +225,11 @@ int sp_gemm_trace(const void* A, const void* B, void* C, int64_t M, int64_t N, i
 /* sp_gemm for callers whose matrices live in HOST memory (pinned or pageable), same layouts and dtypes:
  * copies A and B to a device staging area owned by the library (grown on demand, kept until sp_shutdown),
  * runs sp_gemm, copies C back, and synchronises `stream`; C_host is valid on return.  With 4096 rows or more (and
- * neither a caller table nor SP_FLAG_DIE_PINNED) M is split into row blocks (2048 rows or more, the last one cut
- * further into halves down to 256 rows so that little work is left once the last byte of A has arrived), each computed
+ * no caller table) M is split into row blocks (512 rows, more when M exceeds 16384: C trails A by one block, so
+ * small blocks leave little to do once the last byte of A has arrived), each computed
  * by its own sp_gemm under the same scheme applied to the block's tile grid, so that copies in both directions overlap
- * the compute; the result is the same.  The staging area is shared: calls from several host threads are served one after
+ * the compute; the result is the same (a die-pinned order is applied unpinned to a row block with fewer tiles than
+ * the device has persistent units).  The staging area is shared: calls from several host threads are served one after
  * the other (the function holds a lock for its whole duration).  Adds SP_ERR_TIMEOUT
  * to sp_gemm's errors. */
 int sp_gemm_host(const void* A_host, const void* B_host, void* C_host, int64_t M, int64_t N, int64_t K, int scheme,

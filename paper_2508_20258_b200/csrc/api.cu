@@ -147,7 +147,7 @@ struct TableEntry {
   uint64_t stamp;
 };
 
-constexpr int kHostChunks = 16;  // sp_gemm_host splits M into at most this many row blocks
+constexpr int kHostChunks = 32;  // sp_gemm_host splits M into at most this many row blocks
 
 struct DeviceState {
   int device = -1;
@@ -174,6 +174,7 @@ constexpr size_t kMaxTables = 64;
 
 constexpr size_t kMaxSkStreams = 8;
 constexpr int kDiePairs = 64;   // die-pinned launches that may be in flight at once on one device (different streams)
+constexpr int kDieWords = 5;    // counters per die-pinned launch: arrivals per half (2), units finished, queue heads (2)
 static std::mutex g_valid_mu;
 static std::vector<Sched> g_validated;
 
@@ -241,10 +242,11 @@ int current_device(int* dev) {
 
 static int get_status_word(DeviceState* ds) {
   if (!ds->status) {
-    // status word, then kDiePairs counter sets (arrivals on half 0, arrivals on half 1, units finished) handed to
-    // die-pinned launches in rotation; the last unit of a launch to finish puts its set back to zero
-    SP_CUDA(cudaMalloc(&ds->status, (2 + 3 * kDiePairs) * sizeof(int32_t)));
-    SP_CUDA(cudaMemset(ds->status, 0, (2 + 3 * kDiePairs) * sizeof(int32_t)));
+    // status word, then kDiePairs counter sets (arrivals on half 0, arrivals on half 1, units finished, next ticket of
+    // half 0, of half 1) handed to die-pinned launches in rotation; the last unit of a launch to finish puts its set
+    // back to zero
+    SP_CUDA(cudaMalloc(&ds->status, (2 + kDieWords * kDiePairs) * sizeof(int32_t)));
+    SP_CUDA(cudaMemset(ds->status, 0, (2 + kDieWords * kDiePairs) * sizeof(int32_t)));
   }
   return SP_OK;
 }
@@ -392,6 +394,10 @@ static int gemm_common(const void* A, const void* B, void* C, int64_t M, int64_t
     }
     call.overlap = 1;
   }
+  if (params && (params->flags & SP_FLAG_STEAL) && !(params->flags & SP_FLAG_DIE_PINNED)) {
+    set_error("SP_FLAG_STEAL is a mode of SP_FLAG_DIE_PINNED (per-half queues)");
+    return SP_ERR_INVALID_ARG;
+  }
   if (params && (params->flags & SP_FLAG_DIE_PINNED)) {
     if (scheme != kDieSplit || call.sched.interleave) {
       set_error("SP_FLAG_DIE_PINNED needs SP_DIE_SPLIT with interleave = 0");
@@ -400,7 +406,8 @@ static int gemm_common(const void* A, const void* B, void* C, int64_t M, int64_t
     rc = get_die_map(ds);
     if (rc != SP_OK) return rc;
     call.pinned = 1;
-    call.die_count_dev = ds->status + 2 + 3 * (int)(ds->die_pair_next++ % kDiePairs);
+    call.die_count_dev = ds->status + 2 + kDieWords * (int)(ds->die_pair_next++ % kDiePairs);
+    call.steal = (params->flags & SP_FLAG_STEAL) ? 1 : 0;
     call.half0 = die_split_half0(call.sched);
     call.sms_on_die[0] = ds->sms_on_die[0]; call.sms_on_die[1] = ds->sms_on_die[1];
     for (int i = 0; i < 8; ++i) call.die_mask[i] = ds->die_mask[i];
@@ -558,29 +565,29 @@ int sp_gemm_host(const void* A_host, const void* B_host, void* C_host, int64_t M
     dA = (char*)ds->staging; dB = dA + pad(a_bytes); dC = dB + pad(b_bytes);
   }
   cudaStream_t st = (cudaStream_t)stream;
-  // Row blocks of C are independent: with at least two of them the copy of the next block of A and the copy-out of the
-  // previous block of C overlap the compute of the current one (both PCIe directions busy at once).  The copies in
-  // are the long pole (A and B together are twice the bytes of C), so what counts is how soon after the last byte of A
-  // has landed the last byte of C leaves: the last block is cut into ever smaller ones (halves, down to 256 rows), so
-  // that only a sliver of compute and of copy-out is left behind the end of the copies in.  Caller tables and
-  // die-pinned orders describe the whole grid, so they take the unsplit path.
-  int64_t blk = 2048;
-  while ((M + blk - 1) / blk > kHostChunks - 3) blk *= 2;
+  // Row blocks of C are independent: the copy of the next block of A and the copy-out of the previous block of C
+  // overlap the compute of the current one (both PCIe directions busy at once).  The copies in are the long pole (A and
+  // B together are twice the bytes of C) and the copy-out of a block can only start once that block of A has landed and
+  // been multiplied, so C trails A by one block all the way: what is left to do after the last byte of A has arrived is
+  // one block's compute and copy-out.  Hence many small blocks (512 rows, more when M is large), not a few large ones.
+  // A caller table describes the whole grid, so it takes the unsplit path.
+  int64_t blk = 512;
+  while ((M + blk - 1) / blk > kHostChunks) blk *= 2;
   int64_t row_start[kHostChunks + 1];
   int n_chunks = 0;
-  {
-    int64_t r = 0;
-    while (M - r > blk) { row_start[n_chunks++] = r; r += blk; }
-    int64_t rem = M - r;                                   // the last block, at most blk rows
-    while (rem > 256 && n_chunks < kHostChunks - 1) {
-      const int64_t h = ((rem + 1) / 2 + 255) / 256 * 256;
-      if (h >= rem) break;
-      row_start[n_chunks++] = r; r += h; rem -= h;
-    }
-    row_start[n_chunks++] = r;
-    row_start[n_chunks] = M;
+  for (int64_t r = 0; r < M; r += blk) row_start[n_chunks++] = r;
+  row_start[n_chunks] = M;
+  const bool split = M >= 4096 && scheme != kCustom;
+  // A die-pinned order needs at least one tile per persistent unit; a row block with fewer runs the same order unpinned.
+  const bool pinned = params && (params->flags & SP_FLAG_DIE_PINNED);
+  sp_params unpinned_params;
+  int pin_units = 0, pin_tm = 256, pin_tn = 256;
+  if (pinned) {
+    unpinned_params = *params;
+    unpinned_params.flags &= ~SP_FLAG_DIE_PINNED;
+    if (params->tile_m) { pin_tm = params->tile_m; pin_tn = params->tile_n; }
+    pin_units = gemm_units(pin_tm, pin_tn, kMaxTiles);
   }
-  const bool split = M >= 4096 && scheme != kCustom && !(params && (params->flags & SP_FLAG_DIE_PINNED));
   if (!split) {
     SP_CUDA(cudaMemcpyAsync(dA, A_host, a_bytes, cudaMemcpyHostToDevice, st));
     SP_CUDA(cudaMemcpyAsync(dB, B_host, b_bytes, cudaMemcpyHostToDevice, st));
@@ -617,7 +624,9 @@ int sp_gemm_host(const void* A_host, const void* B_host, void* C_host, int64_t M
   for (int i = 0; i < n_chunks; ++i) {
     const int64_t r0 = row_start[i], nr = row_start[i + 1] - r0;
     SP_CUDA(cudaStreamWaitEvent(st, ev[i], 0));
-    rc = gemm_common(dA + (size_t)r0 * K * 2, dB, dC + (size_t)r0 * N * out_elt, nr, N, K, scheme, params, stream, nullptr, false);
+    const sp_params* pb = params;
+    if (pinned && (pin_units <= 0 || sp_tile_count(nr, N, pin_tm, pin_tn) < pin_units)) pb = &unpinned_params;
+    rc = gemm_common(dA + (size_t)r0 * K * 2, dB, dC + (size_t)r0 * N * out_elt, nr, N, K, scheme, pb, stream, nullptr, false);
     if (rc != SP_OK) break;
     SP_CUDA(cudaEventRecord(ev[kHostChunks + i], st));
     SP_CUDA(cudaStreamWaitEvent(cout, ev[kHostChunks + i], 0));
@@ -833,7 +842,7 @@ int sp_get_status(void* stream, int32_t* detail) {
   if (ds->status) {
     SP_CUDA(cudaMemcpy(&word, ds->status, sizeof word, cudaMemcpyDeviceToHost));
     // after an expired wait a die-pinned launch may have left its counters behind: everything back to zero
-    if (word != 0) SP_CUDA(cudaMemset(ds->status, 0, (2 + 3 * kDiePairs) * sizeof(int32_t)));
+    if (word != 0) SP_CUDA(cudaMemset(ds->status, 0, (2 + kDieWords * kDiePairs) * sizeof(int32_t)));
   }
   if (detail) *detail = word;
   if (word != 0) { set_error("a device-side wait expired (status word 0x%x)", word); return SP_ERR_TIMEOUT; }

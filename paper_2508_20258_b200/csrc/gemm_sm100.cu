@@ -71,7 +71,10 @@ struct GemmArgs {
   int pinned;                      // 0: slot s runs on unit s % units
   int half0;                       // number of slots in half 0 (queue boundary)
   int units_on_die[2];             // persistent units per die (all SMs host one CTA each)
-  int32_t* die_count;              // three device counters, zero at launch: arrivals on half 0, on half 1, units finished
+  int32_t* die_count;              // five device counters, zero at launch: arrivals on half 0, on half 1, units finished,
+                                   // and (SP_FLAG_STEAL) the next ticket of the queue of half 0 and of half 1
+  int steal;                       // 1: the slots of each half are handed out by ticket, a unit whose own half is exhausted
+                                   //    takes tickets of the other half (pinned must be 1)
   uint32_t die_mask[8];            // bit smid = die of that SM (from the topology probe)
   // Stream-K tail (SP_FLAG_STREAM_K): the last sk.tiles slots are split along k over sk.units units.
   SkPlan sk;
@@ -121,7 +124,10 @@ __device__ __forceinline__ uint32_t pack_bf16(uint32_t lo_bits, uint32_t hi_bits
 }
 
 // ------------------------------------------------------------------ the kernel
-template <int CG, int BN, bool B_NK, bool OUT_F32>
+// DYN selects the build that also contains the two dynamic hand-outs of slots (cluster launch control, per-half ticket
+// queues with stealing); the static schedules (fixed stride, die-pinned ranks, k-split tail) run the build without
+// them, which keeps their code and register pressure out of the default path.
+template <int CG, int BN, bool B_NK, bool OUT_F32, bool DYN>
 __global__ void __launch_bounds__((Cfg<CG, BN>::kThreads), 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const __grid_constant__ CUtensorMap tmC, const GemmArgs args) {
@@ -164,7 +170,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     tmem_relinquish<CG>();
   }
   const uint32_t sched_slot = tmem_slot + 8;       // 2 words: die, rank on that die
-  if (args.pinned && threadIdx.x == 32 * 2 && rank == 0) {
+  if (args.pinned && !args.steal && threadIdx.x == 32 * 2 && rank == 0) {
     // the leader learns which L2 half its SM belongs to and takes the next rank there;
     // both CTAs of the unit read the pair of words after the start-up barrier
     uint32_t smid;
@@ -193,7 +199,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
   // whole tiles of this unit: slots s_first, s_first + s_step, ... below s_end; then its segments of the stream-K tail
   int s_first = unit, s_step = args.units, s_end = args.sk.first_slot;
-  if (args.pinned) {
+  if (args.pinned && !args.steal) {
     const uint32_t die = tmem_slot_ptr[2], r = tmem_slot_ptr[3];
     s_step = args.units_on_die[die];
     s_first = (die ? args.half0 : 0) + (int)r;
@@ -207,7 +213,20 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   // of the unit by the hardware; a reader hands the entry back on the leader's barrier).
   auto work_at = [&](int i, int wait_code) -> Work {
     Work w; w.k0 = 0; w.k1 = KB; w.kind = kWorkFull; w.slot = -1;
-    if (args.clc) {
+    if (DYN && args.steal) {
+      // every item comes from the ring: the leader's producer warp took a ticket for it and wrote the slot (or -1)
+      // into the entry of every CTA of the unit
+      const int e = i % kClcDepth;
+      bool oks = mbar_wait_cluster_acquire(clc_full + 8 * e, (uint32_t)(i / kClcDepth) & 1u, args.status, wait_code);
+      oks = __all_sync(0xffffffffu, oks);
+      int got = -1;
+      if (oks) got = *reinterpret_cast<volatile int32_t*>(smem_raw + (clc_resp + 16 * e - smem_u32(smem_raw)));
+      __syncwarp();
+      if (oks && elect_one()) mbar_arrive_cluster(CG == 1 ? clc_empty + 8 * e : mapa(clc_empty + 8 * e, 0));
+      w.slot = got;
+      return w;
+    }
+    if (DYN && args.clc) {
       if (i == 0) { w.slot = unit; return w; }
       const int e = (i - 1) % kClcDepth;
       bool okc = mbar_wait(clc_full + 8 * e, (uint32_t)((i - 1) / kClcDepth) & 1u, args.status, wait_code);
@@ -240,11 +259,45 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       auto load_b = [&](uint32_t dst, int x, int y, uint32_t bar) {
         if (hinted) tma_load_2d_hint<CG>(dst, &tmB, x, y, bar, pol_b); else tma_load_2d<CG>(dst, &tmB, x, y, bar);
       };
+      int my_die = 0;
+      if (DYN && args.steal) {
+        uint32_t smid;
+        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+        my_die = (int)((args.die_mask[(smid >> 5) & 7] >> (smid & 31)) & 1u);
+      }
       for (int item = 0; ok; ++item) {
+        if (DYN && args.steal && rank == 0) {
+          // Take the next ticket of this unit's own half, or, once that queue is empty, of the other half; publish the
+          // slot to every CTA of the unit.  Taken only now, when the loads of the previous tile have all been issued,
+          // so a unit never holds a tile it is not about to start.
+          const int e = item % kClcDepth;
+          if (item >= kClcDepth) {
+            ok = mbar_wait(clc_empty + 8 * e, (uint32_t)(item / kClcDepth - 1) & 1u, args.status, (kRoleProducer << 8) | 5);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+          }
+          if (elect_one()) {
+            const int size0 = args.half0, size1 = T - args.half0;
+            int slot = -1;
+            int t = atomicAdd(args.die_count + 3 + my_die, 1);
+            if (t < (my_die ? size1 : size0)) slot = (my_die ? size0 : 0) + t;
+            else {
+              t = atomicAdd(args.die_count + 3 + (my_die ^ 1), 1);
+              if (t < (my_die ? size0 : size1)) slot = (my_die ? 0 : size0) + t;
+            }
+#pragma unroll
+            for (uint32_t c = 0; c < (uint32_t)CG; ++c) {
+              const uint32_t dst = CG == 1 ? clc_resp + 16 * e : mapa(clc_resp + 16 * e, c);
+              asm volatile("st.shared::cluster.s32 [%0], %1;" ::"r"(dst), "r"(slot) : "memory");
+              mbar_arrive_cluster(CG == 1 ? clc_full + 8 * e : mapa(clc_full + 8 * e, c));
+            }
+          }
+          __syncwarp();
+        }
         const Work wk = work_at(item, (kRoleProducer << 8) | 4);
         if (wk.slot < 0) break;
         const int s = wk.slot;
-        if (args.clc) {
+        if (DYN && args.clc) {
           // ask for the tile after this one: every CTA arms its own barrier for the 16 bytes the hardware will write
           // to it; the leader first makes sure every reader has handed the entry back, then issues the request
           const int e = item % kClcDepth;
@@ -679,7 +732,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     // launch that is given this set needs no clearing in between (and keeps its place right behind this kernel)
     __threadfence();
     if (atomicAdd(args.die_count + 2, 1) == args.units - 1) {
-      args.die_count[0] = 0; args.die_count[1] = 0; args.die_count[2] = 0;
+      args.die_count[0] = 0; args.die_count[1] = 0; args.die_count[2] = 0; args.die_count[3] = 0; args.die_count[4] = 0;
       __threadfence();
     }
   }
@@ -778,7 +831,7 @@ template <int CG, int BN>
 static int max_units() {
   static int cached[64] = {};      // per device
   using C = Cfg<CG, BN>;
-  auto kern = gemm_kernel<CG, BN, false, false>;
+  auto kern = gemm_kernel<CG, BN, false, false, false>;
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return -1;
   if (cached[dev & 63] > 0) return cached[dev & 63];
@@ -810,11 +863,11 @@ int gemm_units(int tile_m, int tile_n, int64_t T) {
   return (int)units;
 }
 
-template <int CG, int BN, bool B_NK, bool OUT_F32>
+template <int CG, int BN, bool B_NK, bool OUT_F32, bool DYN>
 static int launch_variant(const GemmCall& call, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC,
                           const GemmArgs& args) {
   using C = Cfg<CG, BN>;
-  auto kern = gemm_kernel<CG, BN, B_NK, OUT_F32>;
+  auto kern = gemm_kernel<CG, BN, B_NK, OUT_F32, DYN>;
   static uint64_t configured = 0;  // per instantiation, one bit per device
   cudaError_t e = cudaSuccess;
   if (first_use_on_this_device(configured)) {
@@ -840,15 +893,22 @@ static int launch_variant(const GemmCall& call, const CUtensorMap& tmA, const CU
   return SP_OK;
 }
 
+template <int CG, int BN, bool DYN>
+static int launch_layout(const GemmCall& call, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC,
+                         const GemmArgs& args) {
+  if (call.b_nk) {
+    return call.out_f32 ? launch_variant<CG, BN, true, true, DYN>(call, tmA, tmB, tmC, args)
+                        : launch_variant<CG, BN, true, false, DYN>(call, tmA, tmB, tmC, args);
+  }
+  return call.out_f32 ? launch_variant<CG, BN, false, true, DYN>(call, tmA, tmB, tmC, args)
+                      : launch_variant<CG, BN, false, false, DYN>(call, tmA, tmB, tmC, args);
+}
+
 template <int CG, int BN>
 static int launch_shape(const GemmCall& call, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC,
                         const GemmArgs& args) {
-  if (call.b_nk) {
-    return call.out_f32 ? launch_variant<CG, BN, true, true>(call, tmA, tmB, tmC, args)
-                        : launch_variant<CG, BN, true, false>(call, tmA, tmB, tmC, args);
-  }
-  return call.out_f32 ? launch_variant<CG, BN, false, true>(call, tmA, tmB, tmC, args)
-                      : launch_variant<CG, BN, false, false>(call, tmA, tmB, tmC, args);
+  return (args.clc || args.steal) ? launch_layout<CG, BN, true>(call, tmA, tmB, tmC, args)
+                                  : launch_layout<CG, BN, false>(call, tmA, tmB, tmC, args);
 }
 
 // Tensor maps of recent calls, per host thread: a map is a pure function of (address, extents, box, element type), so a
@@ -907,11 +967,13 @@ int launch_gemm(const GemmCall& call) {
     // (stride offset); the next 64 n live in the next box, 8192 bytes on (leading offset)
     args.b_lbo = 64 * kBK * 2; args.b_sbo = 1024; args.b_kstep = kUmmaK * 128;
   }
+  args.steal = 0;
   args.pinned = 0; args.half0 = 0; args.units_on_die[0] = args.units_on_die[1] = 0; args.die_count = nullptr;
   for (int i = 0; i < 8; ++i) args.die_mask[i] = 0;
   if (call.pinned) {
     const int cg_ = call.tile_m / 128;
     args.pinned = 1;
+    args.steal = call.steal;
     args.half0 = call.half0;
     args.units_on_die[0] = call.sms_on_die[0] / cg_;
     args.units_on_die[1] = call.sms_on_die[1] / cg_;
@@ -957,10 +1019,10 @@ int launch_gemm(const GemmCall& call) {
     const int stages = cg == 1 ? (call.tile_n == 128 ? Cfg<1, 128>::kStages : Cfg<1, 256>::kStages)
                                : (call.tile_n == 128 ? Cfg<2, 128>::kStages : call.tile_n == 256 ? Cfg<2, 256>::kStages : Cfg<2, 512>::kStages);
     fprintf(stderr, "[swizzleperf] gemm %dx%dx%d tile %dx%d (%d CTA%s per tile) scheme %d T=%d units=%d grid=%d stages=%d kblocks=%d "
-                    "b=%s out=%s table=%d pinned=%d split_tail=%d/%d clc=%d overlap=%d k_alternate=%d\n",
+                    "b=%s out=%s table=%d pinned=%d split_tail=%d/%d clc=%d overlap=%d k_alternate=%d steal=%d\n",
             args.M, args.N, args.K, call.tile_m, call.tile_n, cg, cg > 1 ? "s" : "", call.sched.scheme, call.sched.T, args.units,
             (args.clc ? call.sched.T : args.units) * cg, stages, args.kblocks, call.b_nk ? "NxK" : "KxN", call.out_f32 ? "fp32" : "bf16",
-            call.sched.use_table, args.pinned, args.sk.tiles, args.sk.units, args.clc, args.overlap, args.k_alternate);
+            call.sched.use_table, args.pinned, args.sk.tiles, args.sk.units, args.clc, args.overlap, args.k_alternate, args.steal);
   }
   if (cg == 1) return call.tile_n == 128 ? launch_shape<1, 128>(call, tmA, tmB, tmC, args) : launch_shape<1, 256>(call, tmA, tmB, tmC, args);
   if (call.tile_n == 512) return launch_shape<2, 512>(call, tmA, tmB, tmC, args);

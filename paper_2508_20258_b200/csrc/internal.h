@@ -67,8 +67,9 @@ struct GemmCall {
   Sched sched;
   const int32_t* perm_dev;  // table for non-arithmetic schemes, else nullptr
   int32_t* status_dev;      // device status word
-  int32_t* die_count_dev;   // die-pinned launches: a set of three device counters nobody else uses while this launch runs
+  int32_t* die_count_dev;   // die-pinned launches: a set of five device counters nobody else uses while this launch runs
   int pinned;               // die-pinned scheduling (SP_DIE_SPLIT + SP_FLAG_DIE_PINNED)
+  int steal;                // SP_FLAG_STEAL: per-half ticket queues, an idle half takes the other's tickets (with pinned)
   int half0;                // slots in half 0
   int sms_on_die[2];
   uint32_t die_mask[8];

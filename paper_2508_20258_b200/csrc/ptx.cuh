@@ -100,6 +100,31 @@ static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity
   }
 }
 
+// Bounded wait whose acquire reaches cluster scope: for a phase completed by a thread of the peer CTA that first wrote
+// plain data into this CTA's shared memory (st.shared::cluster) and then arrived with release at cluster scope.
+static __device__ __noinline__ bool mbar_wait_cluster_acquire(uint32_t bar, uint32_t parity, int32_t* status, int code,
+                                                              unsigned long long timeout_ns = kTimeoutNs) {
+  const unsigned long long t0 = globaltimer();
+  for (uint32_t i = 1;; ++i) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(20000u)
+        : "memory");
+    if (ok) return true;
+    if ((i & 63u) == 0) {
+      if (*(volatile int32_t*)status != 0) return false;
+      if (globaltimer() - t0 > timeout_ns) {
+        atomicCAS(status, 0, code);
+        return false;
+      }
+    }
+  }
+}
+
 __device__ __forceinline__ void st_release_gpu(int32_t* p, int32_t v) {
   asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }

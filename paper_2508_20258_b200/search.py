@@ -1,25 +1,36 @@
 """Enumerative search for the best tile order of one GEMM: the paper's optimisation loop without the LLM.
 
-The paper's loop proposes a remap, validates it (a non-bijective remap is a failure), runs and
-checks the kernel against the ground truth, measures a bottleneck metric, appends the attempt
-to a history buffer and keeps the best validated candidate.  Here the proposals come from a
-fixed list of parameterised orders instead of a language model, validation is the library's own
-bijectivity gate plus bit-identity of C with the row-major run (a swizzle only reorders tiles),
-and the ranking metric is the measured time of back-to-back launches (the L2 hit rate the paper
-ranks by needs a profiler; `profiles/` shows the two agree in ordering).
+The paper's loop proposes a remap, validates it (a non-bijective remap is a failure), runs and checks the kernel
+against a ground truth, measures a bottleneck metric -- the L2 hit rate, which it ranks by because it is a direct,
+low-noise proxy of locality, with run time second -- appends the attempt to a history buffer and keeps the best
+validated candidate.  Here the proposals come from a fixed list of parameterised orders instead of a language model;
+validation is the library's own bijectivity gate; the check is a comparison of sampled rows of C with a ground truth
+the caller supplies (`make_row_checker`: rows of A.B computed independently of this library); and the ranking is
 
-    python -m paper_2508_20258_b200.search --shape 8192x8192x8192
+* ``rank="l2"``: L2 hit rate first, time second, both read from one profiler run over all valid candidates (the
+  profiler wraps `python -m paper_2508_20258_b200.search --launch-once ...`, after that same command has run without
+  it; its CSV is read by `ncuparse`).  Where the profiler may not be used, the loop says so and ranks by time.
+* ``rank="time"``: measured time of back-to-back launches only.
+
+    python -m paper_2508_20258_b200.search --shape 8192x8192x8192 --rank l2
 """
 
 from __future__ import annotations
 
 import argparse
 import json
+import os
+import shutil
+import subprocess
 import sys
+import tempfile
 from dataclasses import asdict, dataclass, field
-from typing import Dict, List, Optional, Sequence, Tuple
+from typing import Callable, Dict, List, Optional, Sequence, Tuple
 
 from . import binding as sp
+from . import ncuparse
+
+NCU_METRICS = "lts__t_sector_hit_rate.pct,dram__bytes_read.sum,dram__bytes_write.sum,gpu__time_duration.sum"
 
 
 @dataclass
@@ -27,10 +38,14 @@ class Attempt:
     name: str
     scheme: int
     params: Dict
-    status: str = "pending"          # "ok" | "broken" (not a bijection) | "unsupported" | "wrong" (C differs)
+    tile: Tuple[int, int] = (256, 256)
+    status: str = "pending"          # "ok" | "broken" (not a bijection) | "unsupported" | "wrong" (C fails the check)
     ms: Optional[float] = None
     tflops: Optional[float] = None
     speedup: Optional[float] = None  # over the first validated attempt (row-major)
+    l2_hit: Optional[float] = None   # lts__t_sector_hit_rate.pct of one profiled launch (rank="l2")
+    dram_mb: Optional[float] = None  # DRAM read + write of that launch
+    ncu_us: Optional[float] = None   # its duration under the profiler
     note: str = ""
 
 
@@ -38,6 +53,8 @@ class Attempt:
 class SearchResult:
     best: Optional[Attempt]
     history: List[Attempt] = field(default_factory=list)
+    rank_used: str = "time"          # "l2" when the profiler's counters decided, else "time"
+    message: str = ""                # why the ranking fell back to time, if it did
 
 
 def default_candidates(units: int) -> List[Tuple[str, int, Dict]]:
@@ -55,26 +72,71 @@ def default_candidates(units: int) -> List[Tuple[str, int, Dict]]:
             c.append((f"die_split:{an}:group_m:{g}:p", sp.DIE_SPLIT,
                       dict(split_axis=axis, inner_scheme=sp.GROUP_M, inner_group=g, flags=2)))
         c.append((f"die_split:{an}:hilbert:p", sp.DIE_SPLIT, dict(split_axis=axis, inner_scheme=sp.HILBERT, flags=2)))
-    # variants of the schedule under one good order: slots handed out by cluster launch control; last wave split along k
-    # (the latter changes the rounding order of the split tiles, so the loop files it under "wrong" unless C is exact)
+    # variants of the schedule under good orders: serpentine bands with K walked in alternating directions (fewer DRAM
+    # reads; the rounding of C then depends on the order, which the row check allows within the GEMM tolerance), and
+    # slots handed out by cluster launch control
+    ka = sp.FLAG_SERPENTINE | sp.FLAG_K_ALTERNATE
+    c.append(("group_m:8:s+a", sp.GROUP_M, dict(group=8, flags=ka)))
+    c.append(("group_m:16:s+a", sp.GROUP_M, dict(group=16, flags=ka)))
+    c.append(("group_n:8:s+a", sp.GROUP_N, dict(group=8, flags=ka)))
+    c.append(("die_split:m:group_m:8:p:s+a", sp.DIE_SPLIT,
+              dict(split_axis=0, inner_scheme=sp.GROUP_M, inner_group=8, flags=ka | sp.FLAG_DIE_PINNED)))
     c.append(("group_m:8+clc", sp.GROUP_M, dict(group=8, flags=sp.FLAG_CLC)))
-    c.append(("group_n:8+clc", sp.GROUP_N, dict(group=8, flags=sp.FLAG_CLC)))
     return c
 
 
+def make_row_checker(rows: Sequence[int], ref_rows, scale_rows, tol: float = 1e-2, floor: float = 2.0 ** -10) -> Callable:
+    """A check for `search`: the given rows of C must match `ref_rows` (float64, len(rows) x N, computed by the caller
+    independently of this library) with |c - ref| <= tol * max(|ref|, floor * scale), `scale_rows` being
+    sum_k |a_ik||b_kj| for the same rows (the GEMM tolerance of this library's tests)."""
+    import numpy as np
+    import torch
+    idx = torch.as_tensor(list(rows), dtype=torch.long)
+    ref = np.asarray(ref_rows, dtype=np.float64)
+    den = np.maximum(np.abs(ref), floor * np.asarray(scale_rows, dtype=np.float64))
+
+    def check(C) -> Tuple[bool, str]:
+        got = C[idx.to(C.device)].to(torch.float64).cpu().numpy()
+        if not np.isfinite(got).all():
+            return False, "non-finite values in C"
+        err = float((np.abs(got - ref) / den).max())
+        return err <= tol, f"max floored relative error {err:.2e} on {len(rows)} rows"
+    return check
+
+
 def search(A, B, C, tile=(256, 256), candidates: Optional[Sequence[Tuple[str, int, Dict]]] = None,
-           launches: int = 50, out_dtype: int = 0, b_layout: int = 0, verbose: bool = False) -> SearchResult:
-    """Tries every candidate order on C = A.B (CUDA tensors) and returns the history and the fastest valid one.
-    `tile` is one (tile_m, tile_n) or a list of them; every candidate is tried under every tile shape."""
+           launches: int = 50, out_dtype: int = 0, b_layout: int = 0, verbose: bool = False,
+           check: Optional[Callable] = None, rank: str = "time", ncu: str = "ncu") -> SearchResult:
+    """Tries every candidate order on C = A.B (CUDA tensors); returns the history and the best valid one.
+    `tile` is one (tile_m, tile_n) or a list of them; every candidate is tried under every tile shape.
+    `check(C) -> (ok, note)` decides whether a run's C is right (see `make_row_checker`); without one only the
+    bijectivity gate and the device status validate a candidate."""
+    if rank not in ("time", "l2"):
+        raise ValueError("rank must be 'time' or 'l2'")
     tiles = [tuple(tile)] if isinstance(tile[0], int) else [tuple(t) for t in tile]
     res = SearchResult(best=None)
-    state = {"truth": None, "base_ms": None}
+    state = {"base_ms": None}
     for t in tiles:
-        _search_tile(A, B, C, t, candidates, launches, out_dtype, b_layout, verbose, res, state, len(tiles) > 1)
+        _search_tile(A, B, C, t, candidates, launches, out_dtype, b_layout, verbose, res, state, len(tiles) > 1, check)
+    ok = [h for h in res.history if h.status == "ok"]
+    res.best = min(ok, key=lambda h: h.ms) if ok else None
+    if rank == "l2" and ok:
+        try:
+            _profile(A, B, ok, out_dtype, b_layout, ncu)
+            ranked = [r["attempt"] for r in ncuparse.rank_by_l2(
+                [{"l2_hit_pct": h.l2_hit, "time_us": h.ms * 1e3, "attempt": h} for h in ok])]
+            if not ranked:
+                raise ncuparse.NcuUnavailable("the profiler returned no L2 counters")
+            res.best, res.rank_used = ranked[0], "l2"
+        except (ncuparse.NcuUnavailable, OSError, subprocess.SubprocessError, ValueError) as e:
+            res.rank_used = "time"
+            res.message = f"L2 counters unavailable ({e}); ranked by time instead"
+            if verbose:
+                print(res.message, file=sys.stderr, flush=True)
     return res
 
 
-def _search_tile(A, B, C, tile, candidates, launches, out_dtype, b_layout, verbose, res, state, tag_tile) -> None:
+def _search_tile(A, B, C, tile, candidates, launches, out_dtype, b_layout, verbose, res, state, tag_tile, check) -> None:
     import torch
 
     M, K = A.shape
@@ -83,27 +145,25 @@ def _search_tile(A, B, C, tile, candidates, launches, out_dtype, b_layout, verbo
     units = sp.gemm_units(tile[0], tile[1], T)
     cands = list(candidates) if candidates is not None else default_candidates(units)
     flops = 2.0 * M * N * K
-    truth = state["truth"]
-    base_ms = state["base_ms"]
     for name, scheme, kw in cands:
-        att = Attempt(name=(f"{tile[0]}x{tile[1]}/" if tag_tile else "") + name, scheme=scheme, params=dict(kw))
+        att = Attempt(name=(f"{tile[0]}x{tile[1]}/" if tag_tile else "") + name, scheme=scheme, params=dict(kw), tile=tuple(tile))
         res.history.append(att)
         p = sp.make_params(tile_m=tile[0], tile_n=tile[1], out_dtype=out_dtype, b_layout=b_layout, **kw)
         try:
             sp.tile_map(M, N, tile[0], tile[1], scheme, p)                    # validation: must be a bijection
-            C.zero_()
+            C.fill_(float("nan"))
             sp.gemm(A, B, C, scheme, p)
             sp.get_status()
         except sp.SpError as e:
             att.status = "broken" if e.status == sp.ERR_NOT_BIJECTIVE else "unsupported"
             att.note = str(e)
             continue
-        bits = C.view(torch.int16 if C.element_size() == 2 else torch.int32)
-        if truth is None:
-            truth = bits.clone()                                              # ground truth: the first valid run
-        elif not torch.equal(bits, truth):
-            att.status = "wrong"
-            continue
+        if check is not None:
+            good, note = check(C)
+            att.note = note
+            if not good:
+                att.status = "wrong"
+                continue
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for _ in range(launches):
@@ -112,14 +172,73 @@ def _search_tile(A, B, C, tile, candidates, launches, out_dtype, b_layout, verbo
         e1.synchronize()
         att.ms = e0.elapsed_time(e1) / launches
         att.tflops = flops / att.ms / 1e9
-        base_ms = base_ms or att.ms
-        att.speedup = base_ms / att.ms
+        state["base_ms"] = state["base_ms"] or att.ms
+        att.speedup = state["base_ms"] / att.ms
         att.status = "ok"
-        if res.best is None or att.ms < res.best.ms:
-            res.best = att
         if verbose:
             print(json.dumps(asdict(att)), flush=True)
-    state["truth"], state["base_ms"] = truth, base_ms
+
+
+def _profile(A, B, attempts: List[Attempt], out_dtype: int, b_layout: int, ncu: str) -> None:
+    """One launch of every attempt under the profiler, in a child process on inputs of the same shape; fills l2_hit,
+    dram_mb and ncu_us.  The child command is first run plainly and must exit 0 before the profiler wraps it."""
+    exe = shutil.which(ncu)
+    if exe is None:
+        raise ncuparse.NcuUnavailable(f"{ncu} not found")
+    M, K = A.shape
+    N = B.shape[0] if b_layout else B.shape[1]
+    with tempfile.TemporaryDirectory(prefix="sp_search_") as tmp:
+        spec = os.path.join(tmp, "candidates.json")
+        with open(spec, "w") as fh:
+            json.dump({"shape": [M, N, K], "out_dtype": out_dtype, "b_layout": b_layout,
+                       "candidates": [{"name": h.name, "scheme": h.scheme, "params": _plain(h.params), "tile": list(h.tile)}
+                                      for h in attempts]}, fh)
+        root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+        child = [sys.executable, "-m", "paper_2508_20258_b200.search", "--launch-once", spec]
+        env = dict(os.environ, PYTHONPATH=root + os.pathsep + os.environ.get("PYTHONPATH", ""))
+        plain = subprocess.run(child, capture_output=True, text=True, env=env, cwd=root, timeout=900)
+        if plain.returncode != 0:
+            raise ncuparse.NcuUnavailable(f"the launch command failed without the profiler: {plain.stderr.strip()[-200:]}")
+        log = os.path.join(tmp, "ncu.csv")
+        cmd = [exe, "--metrics", NCU_METRICS, "--clock-control", "none", "-k", "regex:gemm_kernel", "--csv", "--log-file", log] + child
+        prof = subprocess.run(cmd, capture_output=True, text=True, env=env, cwd=root, timeout=1800)
+        if prof.returncode != 0 or not os.path.exists(log):
+            raise ncuparse.NcuUnavailable(f"profiler exit code {prof.returncode}: {(prof.stdout + prof.stderr).strip()[-300:]}")
+        rows = ncuparse.per_launch_table(log, [h.name for h in attempts])
+    for h, r in zip(attempts, rows):
+        h.l2_hit = r["l2_hit_pct"]
+        h.dram_mb = None if r["dram_bytes"] is None else r["dram_bytes"] / 1e6
+        h.ncu_us = r["time_us"]
+
+
+def _plain(kw: Dict) -> Dict:
+    return {k: (list(map(int, v)) if k == "custom_perm" and v is not None else v) for k, v in kw.items()}
+
+
+def _launch_once(spec_path: str) -> int:
+    """The command the profiler wraps: one launch per candidate, in list order, on seeded inputs of the given shape."""
+    import torch
+    with open(spec_path) as fh:
+        spec = json.load(fh)
+    M, N, K = spec["shape"]
+    A, B, C = _inputs(M, N, K, spec["out_dtype"], spec["b_layout"])
+    for c in spec["candidates"]:
+        p = sp.make_params(tile_m=c["tile"][0], tile_n=c["tile"][1], out_dtype=spec["out_dtype"], b_layout=spec["b_layout"], **c["params"])
+        sp.gemm(A, B, C, c["scheme"], p)
+    torch.cuda.synchronize()
+    if sp.get_status() != 0:
+        return 1
+    print(json.dumps({"launch_order": [c["name"] for c in spec["candidates"]]}), flush=True)
+    return 0
+
+
+def _inputs(M, N, K, out_dtype=0, b_layout=0):
+    import torch
+    g = torch.Generator(device="cuda").manual_seed(0)
+    A = torch.randn((M, K), device="cuda", generator=g).bfloat16()
+    B = torch.randn((N, K) if b_layout else (K, N), device="cuda", generator=g).bfloat16()
+    C = torch.empty((M, N), device="cuda", dtype=torch.float32 if out_dtype else torch.bfloat16)
+    return A, B, C
 
 
 def main(argv=None) -> int:
@@ -128,16 +247,23 @@ def main(argv=None) -> int:
     ap.add_argument("--shape", default="8192x8192x8192")
     ap.add_argument("--tile", default="256x256,256x512", help="one or more MxN scheduler tiles, comma separated")
     ap.add_argument("--launches", type=int, default=100)
+    ap.add_argument("--rank", default="time", choices=["time", "l2"], help="l2: L2 hit rate first (profiler), time second")
+    ap.add_argument("--launch-once", metavar="SPEC.json", help=argparse.SUPPRESS)
     a = ap.parse_args(argv)
+    if a.launch_once:
+        return _launch_once(a.launch_once)
     M, N, K = (int(v) for v in a.shape.split("x"))
     tile = [tuple(int(v) for v in t.split("x")) for t in a.tile.split(",")]
-    g = torch.Generator(device="cuda").manual_seed(0)
-    A = torch.randn((M, K), device="cuda", generator=g).bfloat16()
-    B = torch.randn((K, N), device="cuda", generator=g).bfloat16()
-    C = torch.empty((M, N), device="cuda", dtype=torch.bfloat16)
-    r = search(A, B, C, tile, launches=a.launches, verbose=True)
-    print(json.dumps({"best": asdict(r.best) if r.best else None,
-                      "tried": len(r.history), "broken": [h.name for h in r.history if h.status == "broken"]}))
+    A, B, C = _inputs(M, N, K)
+    # ground truth for the check: sampled rows of A.B from the fp64 matrix product of the tensor library
+    rows = sorted({0, M - 1} | {int(v) for v in torch.randint(0, M, (30,), generator=torch.Generator().manual_seed(1))})
+    Ad, Bd = A[rows].double(), B.double()
+    ref, scale = (Ad @ Bd).cpu().numpy(), (Ad.abs() @ Bd.abs()).cpu().numpy()
+    del Ad, Bd
+    r = search(A, B, C, tile, launches=a.launches, verbose=True, check=make_row_checker(rows, ref, scale), rank=a.rank)
+    print(json.dumps({"best": asdict(r.best) if r.best else None, "rank_used": r.rank_used, "message": r.message,
+                      "tried": len(r.history), "broken": [h.name for h in r.history if h.status == "broken"],
+                      "wrong": [h.name for h in r.history if h.status == "wrong"]}))
     return 0
 
 

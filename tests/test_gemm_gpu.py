@@ -523,3 +523,49 @@ def test_k_alternate_within_tolerance_and_with_the_other_schedulers():
             continue
         r = G.compare(got, ref, S)
         assert r["max_err"] <= TOL, (tile, scheme, r)
+
+
+def test_stealing_between_the_die_queues():
+    """SP_FLAG_STEAL: each half's slots are handed out by ticket to the units of its L2 half; a unit whose own queue
+    is empty takes tickets of the other half.  Every tile must still run exactly once, under the same map, with the
+    same bits; on a lopsided grid (half 0 holds two tile rows, half 1 one) units of half 1's die must end up running
+    slots of half 0, which the fixed die-pinned assignment never lets them do; and on an even grid nothing needs to
+    be stolen in bulk."""
+    die, conf, _ = sp.probe_topology()
+    if conf < 0.8 or (die < 0).any():
+        pytest.skip("no two-way L2 structure measured on this device")
+    K = 512
+    kw = dict(split_axis=0, inner_scheme=sp.GROUP_N, inner_group=8)
+    for (M, N, tile, lopsided) in [(3 * 256, 60 * 256, (256, 256), True), (8 * 256, 40 * 256, (256, 256), False),
+                                   (2 * 128 + 40, 80 * 256 + 8, (128, 256), True), (6 * 256, 20 * 512, (256, 512), False)]:
+        A, B = synth.make_int_inputs(M, N, K, seed=M + N)
+        dA, dB = dev_bf16(A), dev_bf16(B)
+        ref = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        sp.gemm(dA, dB, ref, sp.ROW_MAJOR, sp.make_params(tile_m=tile[0], tile_n=tile[1]))
+        want = R.tile_map(M, N, tile[0], tile[1], sp.DIE_SPLIT, R.Params(**kw))
+        Tm, Tn = -(-M // tile[0]), -(-N // tile[1])
+        h0 = len(R.die_split_halves(Tm, Tn, 0, sp.GROUP_N, 8)[0])
+        crossed = {}
+        for flags in (sp.FLAG_DIE_PINNED, sp.FLAG_DIE_PINNED | sp.FLAG_STEAL):
+            p = sp.make_params(tile_m=tile[0], tile_n=tile[1], flags=flags, **kw)
+            dC = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+            tr = sp.gemm_trace(dA, dB, dC, sp.DIE_SPLIT, p)
+            assert sp.get_status() == 0
+            assert torch.equal(dC.view(torch.int16), ref.view(torch.int16))
+            assert tr["slot"].tolist() == list(range(Tm * Tn)) and tr["tile"].tolist() == want   # every slot once, same map
+            on_die = die[tr["smid"]]
+            d0 = int(np.bincount(on_die[:h0], minlength=2).argmax())          # the die that serves half 0
+            crossed[flags] = int((on_die[:h0] != d0).sum()) + int((on_die[h0:] == d0).sum())
+            # plain launches (not traced) of the same mode, twice: the ticket counters must come back to zero
+            for _ in range(2):
+                dC.fill_(float("nan"))
+                sp.gemm(dA, dB, dC, sp.DIE_SPLIT, p)
+                assert sp.get_status() == 0
+                assert torch.equal(dC.view(torch.int16), ref.view(torch.int16))
+        if lopsided:
+            # half 0 has twice the tiles: with tickets the other die's units come over for a good share of them
+            assert crossed[sp.FLAG_DIE_PINNED | sp.FLAG_STEAL] >= h0 // 8, crossed
+            assert crossed[sp.FLAG_DIE_PINNED | sp.FLAG_STEAL] > crossed[sp.FLAG_DIE_PINNED]
+    with pytest.raises(sp.SpError) as e:                                      # a mode of the pinned split only
+        sp.gemm(dA, dB, ref, sp.GROUP_M, sp.make_params(tile_m=256, tile_n=256, group=4, flags=sp.FLAG_STEAL))
+    assert e.value.status == sp.ERR_INVALID_ARG

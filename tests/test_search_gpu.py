@@ -1,62 +1,82 @@
-"""The enumerative search loop: broken remaps are recorded as failures, valid ones are checked
-against the ground truth and ranked, the best is a validated candidate."""
+"""The enumerative search loop: broken remaps are recorded as failures, valid ones are checked against rows of the
+CPU oracle and ranked (by L2 hit rate first when the profiler may be used, else by time), the best is a validated
+candidate."""
 
+import numpy as np
 import pytest
 
 import paper_2508_20258_b200 as sp
-from paper_2508_20258_b200 import search
+from oracle import gemm as G
+from paper_2508_20258_b200 import search, synth
 
 pytestmark = pytest.mark.gpu
 torch = pytest.importorskip("torch")
 
 
-def test_search_loop_validates_ranks_and_keeps_history():
+def _problem(M, N, K, seed):
+    A, B = synth.make_inputs(M, N, K, "normal", 1.0, seed=seed)
+    dA = torch.from_numpy(A.view(np.int16)).cuda().view(torch.bfloat16)
+    dB = torch.from_numpy(B.view(np.int16)).cuda().view(torch.bfloat16)
+    dC = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    rows = [0, 1, 255, 256, 1000, M // 2 - 1, M // 2, M - 129, M - 1]
+    ref, S = G.gemm_rows(A, B, rows)                       # the ground truth of the loop: rows of the fp64 CPU oracle
+    return dA, dB, dC, search.make_row_checker(rows, ref, S)
+
+
+def test_search_loop_validates_checks_against_the_oracle_and_keeps_history():
     M, N, K = 4096, 5120, 512                     # 16 x 20 tiles of 256 x 256
-    g = torch.Generator(device="cuda").manual_seed(1)
-    A = torch.randn((M, K), device="cuda", generator=g).bfloat16()
-    B = torch.randn((K, N), device="cuda", generator=g).bfloat16()
-    C = torch.empty((M, N), device="cuda", dtype=torch.bfloat16)
+    dA, dB, dC, check = _problem(M, N, K, 1)
     cands = [("row_major", sp.ROW_MAJOR, {}), ("group_m:4", sp.GROUP_M, dict(group=4)), ("hilbert", sp.HILBERT, {}),
              ("xcd:4:74:literal", sp.XCD, dict(num_xcds=4, wave=74, xcd_balanced=0)),       # 74 = 19+19+18+18: reaches 74
              ("xcd:2:74", sp.XCD, dict(num_xcds=2, wave=74, xcd_balanced=1)),
+             ("group_m:4:s+a", sp.GROUP_M, dict(group=4, flags=sp.FLAG_SERPENTINE | sp.FLAG_K_ALTERNATE)),
              ("custom:dup", sp.CUSTOM, dict(custom_perm=[0] * 320))]
-    r = search.search(A, B, C, (256, 256), cands, launches=5)
+    r = search.search(dA, dB, dC, (256, 256), cands, launches=5, check=check)
     by = {h.name: h for h in r.history}
     assert [h.name for h in r.history] == [c[0] for c in cands]
     assert by["xcd:4:74:literal"].status == "broken" and by["custom:dup"].status == "broken"
     ok = [h for h in r.history if h.status == "ok"]
-    assert {h.name for h in ok} == {"row_major", "group_m:4", "hilbert", "xcd:2:74"}
-    assert all(h.ms > 0 and h.tflops > 0 for h in ok) and by["row_major"].speedup == 1.0
-    assert r.best is not None and r.best.status == "ok" and r.best.ms == min(h.ms for h in ok)
+    assert {h.name for h in ok} == {"row_major", "group_m:4", "hilbert", "xcd:2:74", "group_m:4:s+a"}
+    assert all(h.ms > 0 and h.tflops > 0 and "relative error" in h.note for h in ok) and by["row_major"].speedup == 1.0
+    assert r.rank_used == "time" and r.best is not None and r.best.status == "ok" and r.best.ms == min(h.ms for h in ok)
     assert len(search.default_candidates(74)) > 20
+    # a check that cannot be met files every runnable candidate under "wrong" and leaves no best
+    bad = search.search(dA, dB, dC, (256, 256), cands[:2], launches=2, check=lambda C: (False, "refused"))
+    assert [h.status for h in bad.history] == ["wrong", "wrong"] and bad.best is None
 
 
-def test_recommended_configuration_runs_and_beats_the_smallest_tile():
-    import numpy as np
-    from oracle import gemm as G
-    from paper_2508_20258_b200 import synth
+def test_search_loop_ranks_by_l2_hit_rate_when_the_profiler_may_be_used():
+    """8192 x 8192 x 2048 (A and B 32 MiB each, C 128 MiB: larger than L2 together): one profiler run over the valid
+    candidates fills the L2 hit rate of each; the best is the one the paper's ranking picks (hit rate first, time
+    second).  Where the profiler is closed the loop must say so and fall back to time."""
+    M, N, K = 8192, 8192, 2048
+    dA, dB, dC, check = _problem(M, N, K, 2)
+    cands = [("row_major", sp.ROW_MAJOR, {}), ("group_m:8", sp.GROUP_M, dict(group=8)), ("group_n:2", sp.GROUP_N, dict(group=2)),
+             ("xcd:4:74:literal", sp.XCD, dict(num_xcds=4, wave=74, xcd_balanced=0)),
+             ("group_m:8:s+a", sp.GROUP_M, dict(group=8, flags=sp.FLAG_SERPENTINE | sp.FLAG_K_ALTERNATE))]
+    r = search.search(dA, dB, dC, (256, 256), cands, launches=5, check=check, rank="l2")
+    ok = [h for h in r.history if h.status == "ok"]
+    assert {h.name for h in ok} == {"row_major", "group_m:8", "group_n:2", "group_m:8:s+a"}
+    if r.rank_used == "time":
+        assert "unavailable" in r.message and r.best.ms == min(h.ms for h in ok)
+        pytest.skip(r.message)
+    assert all(h.l2_hit is not None and 0 < h.l2_hit <= 100 and h.dram_mb > 0 and h.ncu_us > 0 for h in ok)
+    top = max(round(h.l2_hit, 1) for h in ok)
+    assert round(r.best.l2_hit, 1) == top and r.best.ms == min(h.ms for h in ok if round(h.l2_hit, 1) == top)
+    assert all(h.l2_hit is None for h in r.history if h.status != "ok")
+
+
+def test_recommended_configuration_runs_and_matches_the_oracle():
     M, N, K = 4096, 6144, 2048
     A, B = synth.make_int_inputs(M, N, K, seed=4)
     dA = torch.from_numpy(A.view(np.int16)).cuda().view(torch.bfloat16)
     dB = torch.from_numpy(B.view(np.int16)).cuda().view(torch.bfloat16)
     dC = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
     scheme, p = sp.recommend(M, N, K)
+    assert (p.tile_m, p.tile_n) in [(256, 512), (256, 256)]       # a large tile for a large problem
     sp.gemm(dA, dB, dC, scheme, p)
     assert sp.get_status() == 0
     rows = [0, 255, 256, 2047, M - 1]
     ref, _ = G.gemm_rows(A, B, rows)
     want = G.bf16_bits_to_f64(synth.f32_to_bf16_bits(ref.astype(np.float32)))
     assert np.array_equal(G.bf16_bits_to_f64(dC[rows].view(torch.int16).cpu().numpy().view(np.uint16)), want)
-
-    def timed(s_, p_):
-        for _ in range(5):
-            sp.gemm(dA, dB, dC, s_, p_)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(50):
-            sp.gemm(dA, dB, dC, s_, p_)
-        e1.record()
-        e1.synchronize()
-        return e0.elapsed_time(e1)
-    small = timed(sp.ROW_MAJOR, sp.make_params(tile_m=128, tile_n=128))
-    assert timed(scheme, p) < small / 1.2
