@@ -225,7 +225,7 @@ int sp_gemm_trace(const void* A, const void* B, void* C, int64_t M, int64_t N, i
 /* sp_gemm for callers whose matrices live in HOST memory (pinned or pageable), same layouts and dtypes:
  * copies A and B to a device staging area owned by the library (grown on demand, kept until sp_shutdown),
  * runs sp_gemm, copies C back, and synchronises `stream`; C_host is valid on return.  With 4096 rows or more (and
- * no caller table) M is split into row blocks (512 rows, more when M exceeds 16384: C trails A by one block, so
+ * no caller table) M is split into row blocks (256 rows, more when M exceeds 8192: C trails A by one block, so
  * small blocks leave little to do once the last byte of A has arrived), each computed
  * by its own sp_gemm under the same scheme applied to the block's tile grid, so that copies in both directions overlap
  * the compute; the result is the same (a die-pinned order is applied unpinned to a row block with fewer tiles than
