@@ -915,6 +915,71 @@ def run_stencil(args) -> int:
     return 0
 
 
+SOFTMAX_SWEEP = ["single:row_major", "single:group_m:8", "two:row_major", "two:col_major", "two:group_m:8", "two:hilbert",
+                 "rev:row_major", "rev:col_major", "rev:group_m:8", "rev:group_n:4", "rev:hilbert", "rev:hilbert_rect"]
+
+
+def run_softmax(args) -> int:
+    """Fourth workload (the paper's softmax case study): row softmax of an fp32 matrix, single pass and in the two-phase
+    tiled form under each tile order, the second phase in the same or in reverse slot order.  HBM bound: algorithmic
+    bytes = 2 * M * N * 4 (every element read once, written once).  Specs are `mode:order` with mode single / two / rev."""
+    import torch
+    import paper_2508_20258_b200 as sp
+    M, N = (int(v) for v in args.softmax.split("x"))
+    torch.cuda.set_device(0)
+    g = torch.Generator(device="cuda").manual_seed(13)
+    x = torch.randn((M, N), device="cuda", generator=g, dtype=torch.float32) * 3.0
+    out = torch.empty_like(x)
+    stream = torch.cuda.current_stream()
+    peaks = benchutil.measured_peaks(ROOT)
+    nbytes = 2.0 * M * N * 4
+    specs = args.scheme.split(",") if args.scheme else SOFTMAX_SWEEP
+    modes = {"single": sp.SOFTMAX_SINGLE_PASS, "two": sp.SOFTMAX_TWO_PHASE, "rev": sp.SOFTMAX_TWO_PHASE_REVERSED}
+
+    def timed(spec, n):
+        mode, order = spec.split(":", 1)
+        scheme, kw = parse_scheme(order)
+        p = sp.make_params(**kw)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(n):
+            sp.softmax(x, out, modes[mode], scheme, p, stream)
+        e1.record(stream)
+        e1.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    if args.profile_sweep:
+        for spec in specs:
+            timed(spec, 1)
+        assert sp.get_status() == 0
+        print(json.dumps({"profile_sweep": "softmax", "shape": [M, N], "launch_order": specs}), flush=True)
+        return 0
+    for spec in specs:
+        timed(spec, 3)
+        one = timed(spec, 5)
+        n = int(max(10, min(1000, 200.0 / one)))
+        ms = min(timed(spec, n) for _ in range(2))
+        gbs = nbytes / ms / 1e6
+        print(json.dumps({"softmax": [M, N], "scheme": spec, "ms": ms, "GB/s": gbs,
+                          "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                       "frac": gbs / peaks["hbm_gbs"], "peak_kind": f"copy bandwidth, {peaks['source']}"}}),
+              flush=True)
+    assert sp.get_status() == 0
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for name, fn in (("torch.softmax (context only)", lambda: torch.softmax(x, dim=1, out=out)),
+                     ("torch copy_ of the matrix (context only)", lambda: out.copy_(x))):
+        for _ in range(3):
+            fn()
+        e0.record(stream)
+        for _ in range(20):
+            fn()
+        e1.record(stream)
+        e1.synchronize()
+        ms = e0.elapsed_time(e1) / 20
+        print(json.dumps({"softmax": [M, N], "scheme": name, "ms": ms, "GB/s": nbytes / ms / 1e6}), flush=True)
+    return 0
+
+
 def main() -> int:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -943,12 +1008,15 @@ def main() -> int:
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--transpose", default=None, metavar="MxN", help="time sp_transpose on an M x N 16-bit matrix instead")
     ap.add_argument("--stencil", default=None, metavar="MxN", help="time sp_stencil2d on an M x N fp32 grid instead")
+    ap.add_argument("--softmax", default=None, metavar="MxN", help="time sp_softmax on an M x N fp32 matrix instead")
     args = ap.parse_args()
     args.resume_key = f"{args.workload}|{args.shape}|{args.tile}|{args.b_layout}"
     if args.transpose:
         return run_transpose(args)
     if args.stencil:
         return run_stencil(args)
+    if args.softmax:
+        return run_softmax(args)
     if args.impl == "reference":
         return run_reference(args)
     return run_ours(args)

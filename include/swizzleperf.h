@@ -297,6 +297,37 @@ int sp_transpose(const void* in, void* out, int64_t M, int64_t N, int scheme, co
 int sp_stencil2d(const void* in, void* out, int64_t M, int64_t N, float c_center, float c_neighbor, int scheme,
                  const sp_params* params, void* stream);
 
+/* Row softmax of an fp32 matrix, out[i][j] = exp(in[i][j] - max_j in[i][:]) / sum_j exp(in[i][j] - max_j in[i][:]), in
+ * the two forms the paper's softmax case study contrasts (there the rows are reduced in two phases, the maximum first, then
+ * the exponentials and their sum, with the chunks of a row spread over blocks; the remap the paper finds keeps a row's
+ * chunks in one chiplet's L2 between the phases):
+ *   mode SP_SOFTMAX_SINGLE_PASS        : blocks of whole rows pass through shared memory once; every byte crosses HBM
+ *                                        once per direction.  N <= 16384 (a row must fit a 64 KiB buffer), else
+ *                                        SP_ERR_UNSUPPORTED.  `scheme` / `params` order the row blocks, as for
+ *                                        sp_tile_map(M, N, rows, N, ...) with rows = min(32, 16384 / N) for N <= 2048
+ *                                        (a warp per row) and min(8, 16384 / N) above (all warps on every row).
+ *   mode SP_SOFTMAX_TWO_PHASE          : the matrix is cut into SP_SOFTMAX_TILE_M x SP_SOFTMAX_TILE_N tiles, ordered exactly as
+ *                                        for sp_tile_map(M, N, 32, 512, ...).  A first launch leaves per tile and row
+ *                                        the partial maximum and partial sum; a second one combines them per row, reads
+ *                                        the tiles again (from L2 where they still are) and writes the result.
+ *   mode SP_SOFTMAX_TWO_PHASE_REVERSED : the same, the second launch walking the slots backwards, so that it starts with
+ *                                        the tiles the first one touched last.
+ * Arithmetic in fp32; exp through the hardware's 2^x of (difference x log2 e); sums by lanes, then by shuffles.
+ *   in  : DEVICE, M x N row-major fp32, finite values, read-only.
+ *   out : DEVICE, M x N row-major fp32, fully overwritten; must not overlap `in`.
+ * The two-phase modes keep their partials (8 bytes per row and column chunk) in device memory owned by the library,
+ * grown on demand and shared by all calls on the device: two-phase calls that overlap on the GPU (different streams)
+ * race on it; serialise them.
+ * Errors: SP_ERR_INVALID_ARG (NULL, sizes, in == out, mode), SP_ERR_ALIGNMENT (pointers not 16-byte aligned, N not a
+ * multiple of 4), SP_ERR_NOT_BIJECTIVE, SP_ERR_UNSUPPORTED, SP_ERR_DEVICE, SP_ERR_CUDA.  Asynchronous on `stream`. */
+#define SP_SOFTMAX_TILE_M 32
+#define SP_SOFTMAX_TILE_N 512
+#define SP_SOFTMAX_SINGLE_PASS 0
+#define SP_SOFTMAX_TWO_PHASE 1
+#define SP_SOFTMAX_TWO_PHASE_REVERSED 2
+int sp_softmax(const void* in, void* out, int64_t M, int64_t N, int32_t mode, int scheme, const sp_params* params,
+               void* stream);
+
 /* A starting configuration for sp_gemm on this hardware: tile shape, order and its parameters for a given problem.
  * The paper arrives at a remap by searching with measurements in the loop; this is the short table that this
  * library's own sweeps on B200 distil to (no counterpart in the paper, and no substitute for measuring: the search

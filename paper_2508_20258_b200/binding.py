@@ -57,7 +57,7 @@ TRACE_DTYPE = np.dtype([("slot", "<i4"), ("tile", "<i4"), ("smid", "<i4"), ("uni
                         ("mma_wait_acc", "<u4"), ("load_wait_stage", "<u4"), ("epi_wait_acc", "<u4")])
 
 EXPORTS = ["sp_tile_count", "sp_tile_map", "sp_tile_map_device", "sp_gemm", "sp_gemm_trace", "sp_gemm_host",
-           "sp_gemm_noalloc", "sp_transpose", "sp_stencil2d", "sp_gemm_units", "sp_streamk_plan", "sp_recommend",
+           "sp_gemm_noalloc", "sp_transpose", "sp_stencil2d", "sp_softmax", "sp_gemm_units", "sp_streamk_plan", "sp_recommend",
            "sp_probe_dispatch", "sp_probe_topology", "sp_probe_l2_capacity", "sp_selftest_timeout", "sp_selftest_pinned_tickets", "sp_get_status", "sp_last_error", "sp_shutdown"]
 
 
@@ -97,6 +97,8 @@ def lib() -> ctypes.CDLL:
         L.sp_transpose.argtypes = [vp, vp, i64, i64, ctypes.c_int, pp, vp]
         L.sp_stencil2d.restype = ctypes.c_int
         L.sp_stencil2d.argtypes = [vp, vp, i64, i64, ctypes.c_float, ctypes.c_float, ctypes.c_int, pp, vp]
+        L.sp_softmax.restype = ctypes.c_int
+        L.sp_softmax.argtypes = [vp, vp, i64, i64, i32, ctypes.c_int, pp, vp]
         L.sp_gemm_units.restype = ctypes.c_int
         L.sp_gemm_units.argtypes = [i32, i32, i64]
         L.sp_recommend.restype = ctypes.c_int
@@ -284,6 +286,24 @@ def stencil2d(x, out, c_center: float, c_neighbor: float, scheme: int = ROW_MAJO
             raise ValueError("x and out must be contiguous CUDA tensors")
     _check(lib().sp_stencil2d(x.data_ptr(), out.data_ptr(), M, N, c_center, c_neighbor, scheme, _pp(params),
                               _stream_handle(stream)))
+
+
+SOFTMAX_TILE = (32, 512)
+SOFTMAX_SINGLE_PASS, SOFTMAX_TWO_PHASE, SOFTMAX_TWO_PHASE_REVERSED = 0, 1, 2
+
+
+def softmax(x, out, mode: int = SOFTMAX_SINGLE_PASS, scheme: int = ROW_MAJOR, params: Optional[SpParams] = None,
+            stream=None) -> None:
+    """out = row softmax of x (fp32 [M, N]); single pass through shared memory, or the two-phase tiled form whose tiles
+    are visited in the given order (asynchronous)."""
+    import torch
+    M, N = x.shape
+    if tuple(out.shape) != (M, N) or x.dtype != torch.float32 or out.dtype != torch.float32:
+        raise ValueError("need fp32 input and output of the same [M, N] shape")
+    for t in (x, out):
+        if not t.is_cuda or not t.is_contiguous():
+            raise ValueError("x and out must be contiguous CUDA tensors")
+    _check(lib().sp_softmax(x.data_ptr(), out.data_ptr(), M, N, mode, scheme, _pp(params), _stream_handle(stream)))
 
 
 def gemm_units(tile_m: int, tile_n: int, T: int) -> int:

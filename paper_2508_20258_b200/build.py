@@ -9,7 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libswizzleperf.so")
-SOURCES = ["api.cu", "remap_device.cu", "gemm_sm100.cu", "gemm_noalloc.cu", "probes.cu", "transpose_sm100.cu", "stencil_sm100.cu"]
+SOURCES = ["api.cu", "remap_device.cu", "gemm_sm100.cu", "gemm_noalloc.cu", "probes.cu", "transpose_sm100.cu", "stencil_sm100.cu", "softmax_sm100.cu"]
 
 
 def _nvcc() -> str:

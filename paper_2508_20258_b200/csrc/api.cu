@@ -157,6 +157,8 @@ struct DeviceState {
   int die_known = 0;            // 0: not probed, 1: usable map, -1: probe found no two-way structure
   int sms_on_die[2] = {0, 0};
   uint32_t die_mask[8] = {};
+  void* softmax_ws = nullptr;   // partial maxima and sums of the two-phase softmax (grow-only)
+  size_t softmax_ws_bytes = 0;
   void* staging = nullptr;      // device copies of A, B, C for sp_gemm_host (grow-only)
   size_t staging_bytes = 0;
   cudaStream_t copy_in = nullptr, copy_out = nullptr;   // sp_gemm_host: copies overlap the chunked compute
@@ -721,6 +723,60 @@ static int units_or_nominal(int tile_m, int tile_n) {
   return 148 / (tile_m / 128);
 }
 
+int sp_softmax(const void* in, void* out, int64_t M, int64_t N, int32_t mode, int scheme, const sp_params* params,
+               void* stream) {
+  if (!in || !out) { set_error("in and out must not be NULL"); return SP_ERR_INVALID_ARG; }
+  if (M <= 0 || N <= 0) { set_error("M and N must be positive"); return SP_ERR_INVALID_ARG; }
+  if (M >= (1ll << 31) - 256 || N >= (1ll << 31) - 1024) { set_error("dimension too large"); return SP_ERR_UNSUPPORTED; }
+  if (mode != SP_SOFTMAX_SINGLE_PASS && mode != SP_SOFTMAX_TWO_PHASE && mode != SP_SOFTMAX_TWO_PHASE_REVERSED) {
+    set_error("unknown softmax mode %d", mode);
+    return SP_ERR_INVALID_ARG;
+  }
+  if (((uintptr_t)in | (uintptr_t)out) & 15u) { set_error("in and out must be 16-byte aligned"); return SP_ERR_ALIGNMENT; }
+  if ((N % 4) != 0) { set_error("N must be a multiple of 4 (16-byte row pitch)"); return SP_ERR_ALIGNMENT; }
+  if (in == out) { set_error("out must not overlap in"); return SP_ERR_INVALID_ARG; }
+  int tile_m = SP_SOFTMAX_TILE_M;
+  int64_t tile_n = SP_SOFTMAX_TILE_N;
+  if (mode == SP_SOFTMAX_SINGLE_PASS) {
+    tile_m = softmax_rows_per_block(N);
+    tile_n = N;
+    if (tile_m < 1) { set_error("single-pass softmax needs a row to fit a 64 KiB buffer (N <= 16384); use a two-phase mode"); return SP_ERR_UNSUPPORTED; }
+  }
+  Sched sched;
+  int rc = resolve_sched(M, N, tile_m, (int32_t)tile_n, scheme, params, &sched);
+  if (rc != SP_OK) return rc;
+  std::vector<int32_t> host_perm;
+  if (scheme == kCustom || !already_validated(sched)) {
+    rc = build_perm_host(sched, params ? params->custom_perm : nullptr, host_perm);
+    if (rc != SP_OK) return rc;
+    if (scheme != kCustom) remember_validated(sched);
+  }
+  int dev = 0;
+  rc = current_device(&dev);
+  if (rc != SP_OK) return rc;
+  std::lock_guard<std::mutex> lock(g_mu);
+  DeviceState* ds = device_state(dev);
+  rc = get_status_word(ds);
+  if (rc != SP_OK) return rc;
+  const int32_t* perm_dev = nullptr;
+  if (sched.use_table) {
+    rc = get_table(ds, sched, host_perm, scheme == kCustom, (cudaStream_t)stream, &perm_dev);
+    if (rc != SP_OK) return rc;
+  }
+  float* partial = nullptr;
+  if (mode != SP_SOFTMAX_SINGLE_PASS) {
+    const size_t need = (size_t)M * (size_t)sched.Tn * 2 * sizeof(float);
+    if (ds->softmax_ws_bytes < need) {
+      if (ds->softmax_ws) cudaFree(ds->softmax_ws);   // synchronises: no kernel can still be using it
+      ds->softmax_ws = nullptr; ds->softmax_ws_bytes = 0;
+      SP_CUDA(cudaMalloc(&ds->softmax_ws, need));
+      ds->softmax_ws_bytes = need;
+    }
+    partial = static_cast<float*>(ds->softmax_ws);
+  }
+  return launch_softmax(in, out, M, N, mode, sched, perm_dev, partial, ds->status, (cudaStream_t)stream);
+}
+
 int sp_recommend(int64_t M, int64_t N, int64_t K, int32_t out_dtype, int32_t b_layout, sp_params* params, int* scheme) {
   if (!params || !scheme) { set_error("params and scheme must not be NULL"); return SP_ERR_INVALID_ARG; }
   if (M <= 0 || N <= 0 || K <= 0) { set_error("M, N, K must be positive"); return SP_ERR_INVALID_ARG; }
@@ -865,6 +921,8 @@ void sp_shutdown(void) {
     d.status = nullptr;
     if (d.staging) cudaFree(d.staging);
     d.staging = nullptr; d.staging_bytes = 0;
+    if (d.softmax_ws) cudaFree(d.softmax_ws);
+    d.softmax_ws = nullptr; d.softmax_ws_bytes = 0;
     for (auto& sk : d.sk_spaces) cudaFree(sk.mem);
     d.sk_spaces.clear();
     if (d.copy_in) {

@@ -101,6 +101,9 @@ int launch_stencil(const void* in, void* out, int64_t M, int64_t N, float c_cent
                    const int32_t* perm_dev, int32_t* status_dev, cudaStream_t stream);
 int launch_transpose(const void* in, void* out, int64_t M, int64_t N, const Sched& sched, const int32_t* perm_dev,
                      int32_t* status_dev, cudaStream_t stream);
+int softmax_rows_per_block(int64_t N);   // single pass: rows of one block, 0 when a row does not fit a buffer
+int launch_softmax(const void* in, void* out, int64_t M, int64_t N, int mode, const Sched& sched, const int32_t* perm_dev,
+                   float* partial_dev, int32_t* status_dev, cudaStream_t stream);
 int selftest_timeout(int32_t* status_dev, int timeout_us, int32_t* code_host, int64_t* waited_us_host);
 int probe_dispatch(int n_blocks, int cluster, int32_t* smid_host, uint64_t* start_host);
 int probe_topology(int32_t* sm_to_die_host, int32_t* n_sm, float* confidence, uint32_t* lat_host);
