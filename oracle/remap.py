@@ -162,46 +162,51 @@ def morton(Tm: int, Tn: int) -> List[int]:
 # the paper's formula (appendix listing for GEMM): chiplet-aware transposition
 # ----------------------------------------------------------------------------------
 def hilbert_rect_cells(width: int, height: int) -> List[Tuple[int, int]]:
-    """Generalised Hilbert curve over a width x height rectangle, by the published recursive construction (not in the
-    paper): a rectangle spanned by a major vector a and a minor vector b is walked directly when one cell thick, cut in
-    two along a when 2|a| > 3|b|, else cut into three parts walked along b, along a, and back.  Returns the cells
-    (x, y) in visiting order."""
+    """Generalised Hilbert curve over a width x height rectangle: the cells (x, y) in visiting order.
+
+    Not in the paper.  The construction is the "generalized Hilbert curve" for rectangles of arbitrary size that Jakub
+    Cerveny published (2018, with a reference implementation under the BSD 2-clause licence); it is restated here from
+    its rules, as a work list of oriented rectangles.  An oriented rectangle has a corner, a unit direction `along` with
+    a length (the side the curve runs along, entering at the corner and leaving at the far end of that side) and a unit
+    direction `across` with a length:
+
+      * one cell thick (either way): walk it;
+      * more than 1.5 times as long as thick: cut it in two along its length;
+      * else three parts: a first strip of the thickness, walked across-wise; the rest, walked along; and the first
+        strip's other half, walked back across-wise towards the exit corner.
+
+    Halves are floor(length / 2) when the direction points the positive way and ceil(length / 2) when it points the
+    negative way (the rule is "floor of the signed half"); a cut that would leave an odd first piece of a side longer
+    than 2 is moved by one, so that pieces meet at even offsets and steps stay unit steps where parity allows."""
+    def half(length: int, direction: Tuple[int, int]) -> int:
+        positive = direction[0] + direction[1] > 0
+        return length // 2 if positive else (length + 1) // 2
+
+    def evened(piece: int, whole: int) -> int:
+        return piece + 1 if (piece % 2 == 1 and whole > 2) else piece
+
     out: List[Tuple[int, int]] = []
-
-    def sgn(v: int) -> int:
-        return (v > 0) - (v < 0)
-
-    def gen(x: int, y: int, ax: int, ay: int, bx: int, by: int) -> None:
-        w, h = abs(ax + ay), abs(bx + by)
-        dax, day, dbx, dby = sgn(ax), sgn(ay), sgn(bx), sgn(by)
-        if h == 1:
-            for _ in range(w):
-                out.append((x, y))
-                x, y = x + dax, y + day
-            return
-        if w == 1:
-            for _ in range(h):
-                out.append((x, y))
-                x, y = x + dbx, y + dby
-            return
-        ax2, ay2, bx2, by2 = ax // 2, ay // 2, bx // 2, by // 2     # floor division, also for negative vectors
-        w2, h2 = abs(ax2 + ay2), abs(bx2 + by2)
-        if 2 * w > 3 * h:
-            if w2 % 2 and w > 2:
-                ax2, ay2 = ax2 + dax, ay2 + day                     # prefer even steps
-            gen(x, y, ax2, ay2, bx, by)
-            gen(x + ax2, y + ay2, ax - ax2, ay - ay2, bx, by)
-        else:
-            if h2 % 2 and h > 2:
-                bx2, by2 = bx2 + dbx, by2 + dby
-            gen(x, y, bx2, by2, ax2, ay2)
-            gen(x + bx2, y + by2, ax, ay, bx - bx2, by - by2)
-            gen(x + (ax - dax) + (bx2 - dbx), y + (ay - day) + (by2 - dby), -bx2, -by2, -(ax - ax2), -(ay - ay2))
-
-    if width >= height:
-        gen(0, 0, width, 0, 0, height)
-    else:
-        gen(0, 0, 0, height, width, 0)
+    x_dir, y_dir = (1, 0), (0, 1)
+    first = ((0, 0), x_dir, width, y_dir, height) if width >= height else ((0, 0), y_dir, height, x_dir, width)
+    todo = [first]                                   # last in, first out: parts are pushed in reverse visiting order
+    while todo:
+        (cx, cy), along, la, across, lc = todo.pop()
+        if lc == 1 or la == 1:
+            step, n = (along, la) if lc == 1 else (across, lc)
+            out.extend((cx + i * step[0], cy + i * step[1]) for i in range(n))
+            continue
+        back = (-along[0], -along[1])
+        if 2 * la > 3 * lc:
+            cut = evened(half(la, along), la)
+            todo.append(((cx + cut * along[0], cy + cut * along[1]), along, la - cut, across, lc))
+            todo.append(((cx, cy), along, cut, across, lc))
+            continue
+        strip = evened(half(lc, across), lc)         # thickness of the first and third part
+        near = half(la, along)                       # how far the first part reaches along the length
+        far_corner = (cx + (la - 1) * along[0] + (strip - 1) * across[0], cy + (la - 1) * along[1] + (strip - 1) * across[1])
+        todo.append((far_corner, (-across[0], -across[1]), strip, back, la - near))
+        todo.append(((cx + strip * across[0], cy + strip * across[1]), along, la, across, lc - strip))
+        todo.append(((cx, cy), across, strip, along, near))
     return out
 
 

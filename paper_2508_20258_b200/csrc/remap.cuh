@@ -56,10 +56,11 @@ SP_HD int isgn(int v) { return (v > 0) - (v < 0); }
 SP_HD int iabs(int v) { return v < 0 ? -v : v; }
 SP_HD int floor_half(int v) { return v >= 0 ? v / 2 : -((-v + 1) / 2); }
 
-// Cell number d of the generalised Hilbert curve over a rectangle of `width` x `height` cells (the published recursive
-// construction for arbitrary rectangles: a rectangle spanned by a major vector a and a minor vector b is cut in two
-// along a when it is long, else into three parts walked b-wise, a-wise and back).  Instead of generating the whole
-// curve, this descends into the part that holds index d: O(log) steps, no table.  The curve starts at (0, 0) and
+// Cell number d of the generalised Hilbert curve over a rectangle of `width` x `height` cells.  The curve is the
+// "generalized Hilbert curve" for rectangles of arbitrary size published by Jakub Cerveny (2018; reference implementation
+// under the BSD 2-clause licence): a rectangle spanned by a major vector a and a minor vector b is cut in two along a when
+// it is long, else into three parts walked b-wise, a-wise and back.  This is not that implementation: instead of
+// generating the whole curve it descends into the part that holds index d: O(log) steps, no table.  The curve starts at (0, 0) and
 // moves one cell at a time (one diagonal step can occur when the sides' parities force it).
 SP_HD void hilbert_rect_cell(int width, int height, int d, int& cx, int& cy) {
   int x = 0, y = 0, ax, ay, bx, by;
