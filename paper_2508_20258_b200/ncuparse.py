@@ -13,7 +13,7 @@ Three uses, all from one parser:
 Command line:
 
     python -m paper_2508_20258_b200.ncuparse --launch-list launches.csv
-    python -m paper_2508_20258_b200.ncuparse --sweep l2sweep.csv --order plain.log [--markdown]
+    python -m paper_2508_20258_b200.ncuparse --sweep l2sweep.csv --order plain.log [--markdown [--sustained sweep.jsonl]]
     python -m paper_2508_20258_b200.ncuparse --sweep l2sweep.csv --order plain.log --traffic \
         --workload cfg3 --tile 256x512 --date 2026-11-25 --command "ncu ... python bench.py --profile-sweep ..."
 
@@ -145,10 +145,23 @@ def rank_by_l2(rows: Sequence[Dict]) -> List[Dict]:
     return sorted(usable, key=lambda r: (-round(r["l2_hit_pct"], 1), r.get("time_us") or float("inf")))
 
 
-def markdown(rows: Sequence[Dict]) -> str:
+def read_sustained(path: str) -> Dict[str, Dict]:
+    """The JSON lines of `bench.py --sweep-sustained`: scheme -> {"tflops", "speedup_vs_first"}."""
+    out: Dict[str, Dict] = {}
+    with open(path) as fh:
+        for line in fh:
+            line = line.strip()
+            if line.startswith("{") and "sweep_sustained" in line:
+                j = json.loads(line)
+                out[j["scheme"]] = {"tflops": j["tflops"], "speedup_vs_first": j["speedup_vs_first"]}
+    return out
+
+
+def markdown(rows: Sequence[Dict], sustained: Optional[Dict[str, Dict]] = None) -> str:
     base = next((r for r in rows if r["scheme"] == "row_major"), rows[0] if rows else None)
-    out = ["| scheme | L2 hit % | dL2 vs first/row-major | read hit % | DRAM rd MB | DRAM wr MB | ncu us | SM GHz | tensor % |",
-           "|---|---|---|---|---|---|---|---|---|"]
+    out = ["| scheme | L2 hit % | dL2 vs first/row-major | read hit % | DRAM rd MB | DRAM wr MB | ncu us | SM GHz | tensor % |"
+           + (" sustained TF | x first |" if sustained else ""),
+           "|---|---|---|---|---|---|---|---|---|" + ("---|---|" if sustained else "")]
 
     def f(v, spec="{:.1f}"):
         return "-" if v is None else spec.format(v)
@@ -159,7 +172,9 @@ def markdown(rows: Sequence[Dict]) -> str:
         out.append(f"| {r['scheme']} | {f(r['l2_hit_pct'])} | {d or '-'} | {f(r['l2_read_hit_pct'])} | "
                    f"{f(r['dram_read_bytes'] and r['dram_read_bytes'] / 1e6, '{:.0f}')} | "
                    f"{f(r['dram_write_bytes'] and r['dram_write_bytes'] / 1e6, '{:.0f}')} | {f(r['time_us'], '{:.0f}')} | "
-                   f"{f(r['sm_ghz'], '{:.2f}')} | {f(r['tensor_active_pct'])} |")
+                   f"{f(r['sm_ghz'], '{:.2f}')} | {f(r['tensor_active_pct'])} |"
+                   + ((f" {f(sustained.get(r['scheme'], {}).get('tflops'), '{:.0f}')} |"
+                       f" {f(sustained.get(r['scheme'], {}).get('speedup_vs_first'), '{:.3f}')} |") if sustained else ""))
     return "\n".join(out)
 
 
@@ -195,6 +210,7 @@ def main(argv: Optional[Sequence[str]] = None) -> int:
     ap.add_argument("--launch-list", metavar="CSV")
     ap.add_argument("--sweep", metavar="CSV")
     ap.add_argument("--order", metavar="LOG", help="output of the same command run without the profiler (holds the launch order)")
+    ap.add_argument("--sustained", metavar="JSONL", help="output of bench.py --sweep-sustained: adds its columns to the table")
     ap.add_argument("--kernel", default="gemm_kernel")
     ap.add_argument("--markdown", action="store_true")
     ap.add_argument("--traffic", action="store_true", help="store DRAM bytes per (workload, tile, order) in ncu_traffic.json")
@@ -220,7 +236,7 @@ def main(argv: Optional[Sequence[str]] = None) -> int:
             n = update_traffic(rows, a.workload or o["profile_sweep"], a.tile or o["tile"], a.date, a.command)
             print(f"{n} entries written to {TRAFFIC_PATH}")
         if a.markdown or not a.traffic:
-            print(markdown(rows) if a.markdown else json.dumps(rows, indent=1))
+            print(markdown(rows, read_sustained(a.sustained) if a.sustained else None) if a.markdown else json.dumps(rows, indent=1))
         return 0
     ap.error("nothing to do")
     return 2
