@@ -6,12 +6,13 @@
 // traffic from L2 per flop, at the price of an epilogue that is not hidden behind the next tile's mainloop.
 // Unit u runs slots u, u + units, u + 2*units, ...; slot s computes tile slot_to_tile(s).
 //
-// Warp roles (192 threads; 320 for BN = 512):
+// Warp roles (192 threads; 384 for BN = 512, where warps 2 and 3 idle so that the epilogue warps start on a warp-group
+// boundary and the register file can be re-divided: 72 registers for the issuing group, 216 for the epilogue groups):
 //   warp 0         : TMA producer   -- A and B k-blocks into a ring of 128B-swizzled smem stages (whole warp in the
 //                                      loop, one elected lane issues)
 //   warp 1         : MMA issuer     -- tcgen05.mma, fp32 accumulators in TMEM (two buffers, or two parts of one tile
 //                                      for BN = 512); elected lane issues; the warp also owns TMEM alloc / dealloc
-//   warps 2..5     : epilogue       -- (2..9 for BN = 512, four per accumulator part) tcgen05.ld, convert, stage 32 rows x 128 bytes per warp in swizzled smem,
+//   warps 2..5     : epilogue       -- (4..11 for BN = 512, four per accumulator part) tcgen05.ld, convert, stage 32 rows x 128 bytes per warp in swizzled smem,
 //                                      TMA store (full 128-byte rows; ragged edges clipped by the tensor map)
 //
 // Synchronisation: mbarriers only.  full[s]/empty[s] per smem stage, tmem_full[b]/tmem_empty[b]
@@ -46,7 +47,13 @@ struct Cfg {
   static constexpr int kNT = BN / kMmaN;                        // MMA tiles side by side in one scheduler tile
   static constexpr int kBufs = kNT == 1 ? 2 : 1;                // accumulator buffers of BN columns in the 512 TMEM columns
   static constexpr int kEpiWarps = kNT == 1 ? 4 : 8;            // one per TMEM lane quarter and accumulator part
-  static constexpr int kThreads = 64 + 32 * kEpiWarps;          // producer warp, MMA warp, epilogue warps
+  // Warps: producer, MMA issuer, then the epilogue warps.  With two MMA tiles the epilogue warps start on a warp-group
+  // boundary (warps 2 and 3 idle), so that the register file can be re-divided between the groups (setmaxnreg works
+  // per group of four warps): the two issuing warps need few registers, the epilogue warps many.
+  static constexpr int kEpi0 = kNT == 1 ? 2 : 4;                // first epilogue warp
+  static constexpr int kThreads = 32 * (kEpi0 + kEpiWarps);
+  static constexpr int kGroup = 2;                                  // kNT == 2: k-blocks issued part by part at both ends of a tile
+  static constexpr int kRegsIssue = 72, kRegsEpilogue = 216;    // kNT == 2: 128 x 72 + 256 x 216 = 64512 registers
   static constexpr int kMmaCols = kMmaN / CG;                   // columns of B one CTA supplies to one MMA
   static constexpr int kBCols = BN / CG;                        // columns of B held by one CTA
   static constexpr uint32_t kABytes = 128 * kBK * 2;            // 128 rows of A
@@ -243,6 +250,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     return w;
   };
 
+  if (warp < C::kEpi0) {
+  if constexpr (C::kNT == 2) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsIssue));
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer
     // The whole warp walks the loop (uniform control flow, uniform operands); one elected
@@ -394,23 +403,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         uint32_t wait_acc = 0, wait_data = 0;
         if (tracing && lane == 0) args.trace[s].t_mma_begin = globaltimer();
         if constexpr (C::kNT == 2) {
-          // K-blocks are issued in groups: the first two and the last two k-blocks of a tile as pairs, the rest one by
-          // one.  Inside a group the first MMA tile's MMAs come before the second's.  The first accumulator part is then
-          // complete 1024 cycles of MMAs before the second, and the next tile starts on it equally early: the epilogue
-          // warps of one part drain it while the tensor pipe works on the other.  The body keeps the full look-ahead.
+          // K-blocks are issued in groups: the first kGroup and the last kGroup k-blocks of a tile as a group, the rest one
+          // by one.  Inside a group the first MMA tile's MMAs come before the second's (each k-block as soon as it has
+          // landed).  The first accumulator part is then complete kGroup x 512 cycles of MMAs before the second, and the
+          // next tile starts on it equally early: the epilogue warps of one part drain it (about 1800 cycles) while the
+          // tensor pipe works on the other.  The body keeps the full look-ahead of the ring; a group holds kGroup of its
+          // stages until the second part has used them.  Groups of 3 and 4 were measured: 1 % slower than 2, with the
+          // same tensor-pipe activity (the stages a longer group holds back cost what its longer cover gains).
+          constexpr int G = C::kGroup;
           int kb = 0;
           while (kb < KB && ok) {
-            const bool paired = KB >= 4 && (kb == 0 || kb == KB - 2);
-            const int g = paired ? 2 : 1;
-            uint32_t st0 = 0, st1 = 0;
-            for (int i = 0; i < g && ok; ++i) {                    // operands of the whole group must have landed
-              ok = mbar_wait_timed(bar_full + 8 * stage, phase, args.status, (kRoleMma << 8) | 2, tracing, &wait_data);
-              if (i == 0) st0 = (uint32_t)stage; else st1 = (uint32_t)stage;
-              if (++stage == S) { stage = 0; phase ^= 1u; }
-            }
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tcgen05_fence_after();
+            const bool grouped = KB >= 2 * G && (kb == 0 || kb == KB - G);
+            const int g = grouped ? G : 1;
+            uint32_t st[G];
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
               if (kb == 0) {                                        // the part must have been drained by the previous tile's epilogue
@@ -419,9 +424,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 if (!ok) break;
                 tcgen05_fence_after();
               }
-              if (elect_one()) {
-                for (int i = 0; i < g; ++i) {
-                  const uint32_t sa = smem_base + (i == 0 ? st0 : st1) * C::kStageBytes;
+#pragma unroll
+              for (int i = 0; i < G; ++i) {
+                if (i >= g) break;
+                if (c == 0) {                                       // the first part takes each k-block as soon as it has landed
+                  ok = mbar_wait_timed(bar_full + 8 * stage, phase, args.status, (kRoleMma << 8) | 2, tracing, &wait_data);
+                  ok = __all_sync(0xffffffffu, ok);
+                  if (!ok) break;
+                  tcgen05_fence_after();
+                  st[i] = (uint32_t)stage;
+                  if (++stage == S) { stage = 0; phase ^= 1u; }
+                }
+                if (elect_one()) {
+                  const uint32_t sa = smem_base + st[i] * C::kStageBytes;
                   const uint32_t sb = sa + C::kABytes + (uint32_t)(c * C::kMmaCols * kBK * 2);
 #pragma unroll
                   for (int k = 0; k < kBK / kUmmaK; ++k) {
@@ -429,17 +444,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     const uint64_t db = desc_at(db0, (sb >> 4) + k * b_kstep16);
                     umma_bf16<CG>(tmem_base + (uint32_t)(c * C::kMmaN), da, db, idesc, (uint32_t)(((kb + i) | k) != 0));
                   }
+                  if (c == 1) umma_commit<CG>(bar_empty + 8 * st[i]);          // both parts have used the stage
+                  if (kb + i + 1 == KB) umma_commit<CG>(bar_tfull + 8 * c);     // this part is complete
                 }
-                if (kb + g == KB) umma_commit<CG>(bar_tfull + 8 * c);     // this part is complete
+                __syncwarp();
               }
-              __syncwarp();
+              if (!ok) break;
             }
             if (!ok) break;
-            if (elect_one()) {
-              umma_commit<CG>(bar_empty + 8 * st0);
-              if (g == 2) umma_commit<CG>(bar_empty + 8 * st1);
-            }
-            __syncwarp();
             kb += g;
           }
         } else {
@@ -484,8 +496,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       }
     }
     __syncwarp();
+  }
   } else {
     // ---------------------------------------------------------------- epilogue
+    if constexpr (C::kNT == 2) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(C::kRegsEpilogue));
     const int quarter = warp & 3;  // TMEM lanes [32*quarter, 32*quarter + 32) are this warp's
     auto store_c = [&](uint32_t src, int x, int y) {   // issued by one lane
       if (args.hint_c) tma_store_2d_hint(&tmC, src, x, y, l2_policy(args.hint_c)); else tma_store_2d(&tmC, src, x, y);
@@ -495,8 +509,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       // accumulator part.  A warp empties its 32 lanes x 256 columns into registers (packed bf16), hands the part back
       // to the MMA issuer at once, and only then stages and stores (one 4 KiB slice per warp), which overlaps the
       // mainloop that has already resumed; the other part's warps are never held up by these stores.
-      const int c = (warp - 2) >> 2;                               // the part this warp serves
-      const uint32_t slice = epi_base + (uint32_t)((warp - 2) * 4096);
+      const int c = (warp - C::kEpi0) >> 2;                        // the part this warp serves
+      const uint32_t slice = epi_base + (uint32_t)((warp - C::kEpi0) * 4096);
       const uint32_t rowaddr = slice + (uint32_t)lane * 128u;
       const uint32_t sw = (uint32_t)lane & 7u;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c * C::kMmaN);
@@ -518,12 +532,16 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         if constexpr (!OUT_F32) {
           uint32_t pk[C::kMmaN / 2];
 #pragma unroll
-          for (int q = 0; q < C::kMmaN / 32; ++q) {
-            uint32_t v[32];
-            tmem_ld_32x32b_x32(taddr + (uint32_t)(q * 32), v);
+          for (int q = 0; q < C::kMmaN / 64; ++q) {                  // two read-outs of 32 columns in flight per round trip
+            uint32_t v[32], w[32];
+            tmem_ld_32x32b_x32(taddr + (uint32_t)(q * 64), v);
+            tmem_ld_32x32b_x32(taddr + (uint32_t)(q * 64 + 32), w);
             tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 16; ++j) pk[q * 16 + j] = pack_bf16(v[2 * j], v[2 * j + 1]);
+            for (int j = 0; j < 16; ++j) {
+              pk[q * 32 + j] = pack_bf16(v[2 * j], v[2 * j + 1]);
+              pk[q * 32 + 16 + j] = pack_bf16(w[2 * j], w[2 * j + 1]);
+            }
           }
           tcgen05_fence_before();
           __syncwarp();
@@ -568,7 +586,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           __syncwarp();
           if (lane == 0) mbar_arrive_cluster(mapa(bar_tempty + 8 * c, 0));
         }
-        if (lane == 0 && args.trace && rank == 0 && warp == 6) {   // the second part finishes last
+        if (lane == 0 && args.trace && rank == 0 && warp == C::kEpi0 + 4) {   // the second part finishes last
           args.trace[s].t_end = globaltimer();
           args.trace[s].epi_wait_acc = wait_epi;
         }
@@ -681,7 +699,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             if (lane == 0) bulk_wait_read_1();
             __syncwarp();
           }
-          const uint32_t slice = epi_base + (uint32_t)((warp - 2) * 8192 + (chunk & 1) * 4096);
+          const uint32_t slice = epi_base + (uint32_t)((warp - C::kEpi0) * 8192 + (chunk & 1) * 4096);
           const uint32_t rowaddr = slice + (uint32_t)lane * 128u;
           const uint32_t sw = (uint32_t)lane & 7u;                     // 128-byte swizzle: 16-byte unit j of row r sits at j ^ (r % 8)
           if constexpr (OUT_F32) {
@@ -713,7 +731,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
         }
       }
-      if (ok && lane == 0 && args.trace && rank == 0 && warp == 2) {
+      if (ok && lane == 0 && args.trace && rank == 0 && warp == C::kEpi0) {
         args.trace[s].t_end = globaltimer();
         args.trace[s].epi_wait_acc = wait_epi;
       }

@@ -84,8 +84,10 @@ __device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity
   return ok != 0;
 }
 
-// Bounded wait.  Returns false after kTimeoutNs or once the status word is set by anyone.
-static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, int32_t* status, int code,
+// Bounded wait.  Returns false after kTimeoutNs or once the status word is set by anyone.  (Inlined, like the other
+// bounded waits below: a kernel that re-divides its registers between warp groups cannot make calls from the re-divided
+// regions.)
+static __device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, int32_t* status, int code,
                                             unsigned long long timeout_ns = kTimeoutNs) {
   const unsigned long long t0 = globaltimer();
   for (uint32_t i = 1;; ++i) {
@@ -102,7 +104,7 @@ static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity
 
 // Bounded wait whose acquire reaches cluster scope: for a phase completed by a thread of the peer CTA that first wrote
 // plain data into this CTA's shared memory (st.shared::cluster) and then arrived with release at cluster scope.
-static __device__ __noinline__ bool mbar_wait_cluster_acquire(uint32_t bar, uint32_t parity, int32_t* status, int code,
+static __device__ __forceinline__ bool mbar_wait_cluster_acquire(uint32_t bar, uint32_t parity, int32_t* status, int code,
                                                               unsigned long long timeout_ns = kTimeoutNs) {
   const unsigned long long t0 = globaltimer();
   for (uint32_t i = 1;; ++i) {
@@ -170,7 +172,7 @@ __device__ __forceinline__ void clc_decode(uint32_t resp, uint32_t& valid, uint3
 }
 
 // Bounded wait for a word in global memory to take the value `want` (written by another CTA with st_release_gpu).
-static __device__ __noinline__ bool flag_wait(const int32_t* flag, int32_t want, int32_t* status, int code,
+static __device__ __forceinline__ bool flag_wait(const int32_t* flag, int32_t want, int32_t* status, int code,
                                               unsigned long long timeout_ns = kTimeoutNs) {
   if (ld_acquire_gpu(flag) == want) return true;
   const unsigned long long t0 = globaltimer();
