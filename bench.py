@@ -119,9 +119,9 @@ SWEEPS = {
              "die_split:n:group_m:16:p", "die_split:m:group_n:16:p", "group_m:16:s+a", "group_m:16:s+a+hc", "group_n:8:s+a+hc",
              "die_split:m:group_m:8:p:s+a+hc", "die_split:m:group_m:16:p:s+a+hc"],
 }
-DEFAULT_SCHEME = {"cfg1": "group_m:2", "cfg2": "group_m:8", "cfg3": "die_split:m:group_m:8:p", "cfg4": "row_major",
-                  "cfg5": "die_split:m:group_m:8:p"}
-FALLBACK_SCHEME = {"cfg3": "group_m:8", "cfg5": "group_m:16"}   # if the topology probe finds no two-way L2 structure
+DEFAULT_SCHEME = {"cfg1": "group_m:2", "cfg2": "group_m:8", "cfg3": "die_split:m:group_m:8:p:s+a+hc", "cfg4": "row_major",
+                  "cfg5": "die_split:m:group_m:16:p:s+a+hc"}
+FALLBACK_SCHEME = {"cfg3": "group_m:8:s+a+hc", "cfg5": "group_m:16:s+a+hc"}   # if the topology probe finds no two-way L2 structure
 FALLBACK_SCHEME_BY_TILE = {("cfg3", "256x512"): "group_m:16:s+a+hc", ("cfg5", "256x512"): "group_m:16:s+a+hc"}
 # 8192^3 is timed with two 256x256 2-CTA MMA tiles per scheduler tile (they share the A panel: a quarter less operand
 # traffic from L2); the plain 256x256 scheduler tile is timed beside it and reported in the same line.
@@ -330,8 +330,10 @@ def run_ours(args) -> int:
         if not (args.tile or args.scheme or args.sweep or args.sweep_sustained or args.profile_sweep or args.alternate):
             rs, rp = sp.recommend(Ms, Ns, Ks, 0, b_nk)      # nothing asked for: the library's own suggestion for the shape
             args.tile = f"{rp.tile_m}x{rp.tile_n}"
-            args.scheme = {sp.ROW_MAJOR: "row_major", sp.COL_MAJOR: "col_major", sp.GROUP_M: f"group_m:{rp.group}",
-                           sp.GROUP_N: f"group_n:{rp.group}"}[rs] + ("+k" if rp.flags & sp.FLAG_STREAM_K else "")
+            args.scheme = ({sp.ROW_MAJOR: "row_major", sp.COL_MAJOR: "col_major", sp.GROUP_M: f"group_m:{rp.group}",
+                            sp.GROUP_N: f"group_n:{rp.group}"}[rs] + (":s" if rp.flags & sp.FLAG_SERPENTINE else "")
+                           + ("+a" if rp.flags & sp.FLAG_K_ALTERNATE else "") + ("+hc" if rp.flags & sp.FLAG_HINT_C_EVICT_FIRST else "")
+                           + ("+k" if rp.flags & sp.FLAG_STREAM_K else ""))
     else:
         w = synth.WORKLOADS[args.workload]
         _, A, B = synth.make_workload(args.workload, b_is_nk=bool(b_nk))

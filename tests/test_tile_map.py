@@ -224,7 +224,10 @@ def test_recommendation_is_valid_and_matches_what_the_sweeps_found():
         assert (p.tile_m, p.tile_n) == tile and s == scheme and p.group == group, (M, N, K)
     s, p = sp.recommend(1024, 1024, 8192)                 # few tiles, long k: the k-split is suggested
     assert p.flags == sp.FLAG_STREAM_K and p.tile_n <= 256
-    assert sp.recommend(8192, 8192, 8192)[1].flags == 0 and sp.recommend(512, 512, 512)[1].flags == 0
+    # band orders come with serpentine bands, alternating K and evict_first C stores; orders that need no bands with no flag
+    bands = sp.FLAG_SERPENTINE | sp.FLAG_K_ALTERNATE | sp.FLAG_HINT_C_EVICT_FIRST
+    assert sp.recommend(8192, 8192, 8192)[1].flags == bands and sp.recommend(16384, 16384, 4096)[1].flags == bands
+    assert sp.recommend(512, 512, 512)[1].flags == 0 and sp.recommend(4096, 4096, 4096)[1].flags == 0
     rng = np.random.default_rng(0)
     for _ in range(200):                                  # always a supported tile and a bijective order
         M, N, K = (int(rng.integers(1, 40000)), int(rng.integers(1, 5000)) * 8, int(rng.integers(1, 3000)) * 8)
