@@ -312,6 +312,7 @@ def gemm_units(tile_m: int, tile_n: int, T: int) -> int:
 
 FLAG_DIE_PINNED, FLAG_SERPENTINE, FLAG_STREAM_K, FLAG_OVERLAP, FLAG_CLC, FLAG_K_ALTERNATE = 2, 4, 8, 16, 32, 64
 FLAG_STEAL = 4096
+FLAG_TRACE = 1      # reserved (tracing is its own entry point)
 FLAG_HINT_C_EVICT_FIRST, FLAG_HINT_A_EVICT_FIRST, FLAG_HINT_B_EVICT_FIRST, FLAG_HINT_A_EVICT_LAST, FLAG_HINT_B_EVICT_LAST = 128, 256, 512, 1024, 2048
 STREAMK_MAX_SEGMENTS = 8
 WORK_FULL, WORK_CONTRIB, WORK_OWNER = 0, 1, 2

@@ -70,3 +70,31 @@ def test_stencil_and_transpose_reject_bad_arguments_before_touching_a_device():
     assert L.sp_transpose(a, a, 64, 64, sp.ROW_MAJOR, None, None) == sp.ERR_INVALID_ARG
     first = ctypes.c_int32(0)
     assert L.sp_streamk_plan(16, 4, 8, ctypes.byref(first), None) == sp.ERR_INVALID_ARG
+
+
+def test_flag_and_mode_constants_match_the_header():
+    text = open(os.path.join(ROOT, "include", "swizzleperf.h")).read()
+    defs = {m.group(1): int(m.group(2)) for m in re.finditer(r"#define\s+(SP_[A-Z_0-9]+)\s+(\d+)u?\b", text)}
+    flags = {k[len("SP_FLAG_"):]: v for k, v in defs.items() if k.startswith("SP_FLAG_")}
+    assert len(flags) >= 12 and len(set(flags.values())) == len(flags)            # one bit each, no bit twice
+    assert all(v & (v - 1) == 0 for v in flags.values())
+    for name, value in flags.items():
+        assert getattr(binding, "FLAG_" + name) == value, name
+    assert (defs["SP_SOFTMAX_SINGLE_PASS"], defs["SP_SOFTMAX_TWO_PHASE"], defs["SP_SOFTMAX_TWO_PHASE_REVERSED"]) == \
+        (binding.SOFTMAX_SINGLE_PASS, binding.SOFTMAX_TWO_PHASE, binding.SOFTMAX_TWO_PHASE_REVERSED)
+    assert (defs["SP_SOFTMAX_TILE_M"], defs["SP_SOFTMAX_TILE_N"]) == binding.SOFTMAX_TILE
+    assert (defs["SP_STENCIL_TILE_M"], defs["SP_STENCIL_TILE_N"]) == binding.STENCIL_TILE
+    assert defs["SP_TRANSPOSE_TILE"] == binding.TRANSPOSE_TILE
+
+
+def test_softmax_rejects_bad_arguments_before_touching_a_device():
+    L = sp.lib()
+    a, b = 0x1000, 0x200000
+    assert L.sp_softmax(a, b, 64, 126, 0, sp.ROW_MAJOR, None, None) == sp.ERR_ALIGNMENT
+    assert L.sp_softmax(a + 4, b, 64, 128, 0, sp.ROW_MAJOR, None, None) == sp.ERR_ALIGNMENT
+    assert L.sp_softmax(a, a, 64, 128, 1, sp.ROW_MAJOR, None, None) == sp.ERR_INVALID_ARG
+    assert L.sp_softmax(a, b, 64, 128, 7, sp.ROW_MAJOR, None, None) == sp.ERR_INVALID_ARG
+    assert L.sp_softmax(a, b, 0, 128, 0, sp.ROW_MAJOR, None, None) == sp.ERR_INVALID_ARG
+    assert L.sp_softmax(a, b, 64, 16388, 0, sp.ROW_MAJOR, None, None) == sp.ERR_UNSUPPORTED     # a row must fit a buffer
+    bad = sp.make_params(num_xcds=4, xcd_balanced=0)      # 5 x 2 tiles of 32 x 512: the printed formula leaves [0, 10)
+    assert L.sp_softmax(a, b, 160, 1024, 1, sp.XCD, ctypes.byref(bad), None) == sp.ERR_NOT_BIJECTIVE

@@ -569,3 +569,54 @@ def test_stealing_between_the_die_queues():
     with pytest.raises(sp.SpError) as e:                                      # a mode of the pinned split only
         sp.gemm(dA, dB, ref, sp.GROUP_M, sp.make_params(tile_m=256, tile_n=256, group=4, flags=sp.FLAG_STEAL))
     assert e.value.status == sp.ERR_INVALID_ARG
+
+
+def test_flag_combinations_refused_and_accepted():
+    """Every clash between flags is refused before anything is launched (C keeps its contents); the combinations that are
+    allowed give the oracle's result, exactly (small integers)."""
+    M, N, K = 2048, 2560, 192
+    A, B = synth.make_int_inputs(M, N, K, seed=77)
+    ref, _ = G.gemm_full(A, B)
+    dA, dB = dev_bf16(A), dev_bf16(B)
+    dC = torch.full((M, N), 7.0, dtype=torch.float32, device="cuda")
+    split = dict(inner_scheme=sp.GROUP_M, inner_group=4)
+
+    def call(scheme, tile=(256, 256), **kw):
+        sp.gemm(dA, dB, dC, scheme, sp.make_params(tile_m=tile[0], tile_n=tile[1], out_dtype=1, **kw))
+
+    refused = [(sp.GROUP_M, dict(group=4, flags=sp.FLAG_STEAL)),                                   # a mode of the pinned split
+               (sp.GROUP_M, dict(group=4, flags=sp.FLAG_DIE_PINNED)),                              # pinning needs the split order
+               (sp.DIE_SPLIT, dict(interleave=1, flags=sp.FLAG_DIE_PINNED, **split)),
+               (sp.ROW_MAJOR, dict(flags=sp.FLAG_HINT_A_EVICT_FIRST | sp.FLAG_HINT_A_EVICT_LAST)),
+               (sp.ROW_MAJOR, dict(flags=sp.FLAG_HINT_B_EVICT_FIRST | sp.FLAG_HINT_B_EVICT_LAST)),
+               (sp.DIE_SPLIT, dict(flags=sp.FLAG_DIE_PINNED | sp.FLAG_CLC, **split)),
+               (sp.DIE_SPLIT, dict(flags=sp.FLAG_DIE_PINNED | sp.FLAG_STREAM_K, **split)),
+               (sp.DIE_SPLIT, dict(flags=sp.FLAG_DIE_PINNED | sp.FLAG_OVERLAP, **split)),
+               (sp.ROW_MAJOR, dict(flags=sp.FLAG_CLC | sp.FLAG_STREAM_K)),
+               (sp.ROW_MAJOR, dict(flags=sp.FLAG_OVERLAP | sp.FLAG_STREAM_K))]
+    for scheme, kw in refused:
+        with pytest.raises(sp.SpError) as e:
+            call(scheme, **kw)
+        assert e.value.status == sp.ERR_INVALID_ARG, (scheme, kw)
+    with pytest.raises(sp.SpError) as e:
+        call(sp.ROW_MAJOR, tile=(256, 512), flags=sp.FLAG_STREAM_K)
+    assert e.value.status == sp.ERR_UNSUPPORTED
+    torch.cuda.synchronize()
+    assert bool((dC == 7.0).all())                                                                  # nothing ran
+
+    mem = sp.FLAG_K_ALTERNATE | sp.FLAG_HINT_C_EVICT_FIRST | sp.FLAG_HINT_A_EVICT_LAST | sp.FLAG_HINT_B_EVICT_FIRST
+    accepted = [(sp.GROUP_N, (256, 512), dict(group=2, flags=mem | sp.FLAG_SERPENTINE)),
+                (sp.GROUP_M, (256, 256), dict(group=2, flags=mem | sp.FLAG_STREAM_K)),
+                (sp.HILBERT, (128, 256), dict(flags=mem | sp.FLAG_CLC)),
+                (sp.ROW_MAJOR, (128, 128), dict(flags=mem | sp.FLAG_OVERLAP)),
+                (sp.DIE_SPLIT, (128, 256), dict(flags=mem | sp.FLAG_SERPENTINE | sp.FLAG_DIE_PINNED | sp.FLAG_STEAL, **split)),
+                (sp.DIE_SPLIT, (256, 128), dict(flags=mem | sp.FLAG_DIE_PINNED, **split))]
+    for scheme, tile, kw in accepted:
+        dC.fill_(float("nan"))
+        try:
+            call(scheme, tile=tile, **kw)
+        except sp.SpError as err:                      # die-pinned modes need the two-way L2 structure
+            assert err.status == sp.ERR_UNSUPPORTED and (kw["flags"] & sp.FLAG_DIE_PINNED)
+            continue
+        assert sp.get_status() == 0
+        assert np.array_equal(dC.cpu().numpy().astype(np.float64), ref), (scheme, tile, kw)
