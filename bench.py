@@ -112,14 +112,14 @@ SWEEPS = {
              "group_m:8:s", "group_m:8+a", "group_m:8:s+a", "group_n:8:s+a", "group_m:16:s+a", "group_m:8:s+a+hc",
              "die_split:m:group_m:8:p:s+a", "die_split:m:group_m:8:p:s+a+hc", "die_split:n:group_n:4:p:s+a+hc",
              "die_split:m:group_m:8:p:t:s+a+hc"],
-    "cfg4": [f"group_m:{g}" for g in (1, 2, 4, 8, 16, 32, 64)] + [f"group_n:{g}" for g in (1, 2, 4, 8)],
+    "cfg4": [f"group_m:{g}" for g in (1, 2, 4, 8, 16, 32, 64)] + [f"group_n:{g}" for g in (1, 2, 4, 8)] + ["row_major+a+hc"],
     "cfg5": [f"group_m:{g}" for g in (1, 2, 4, 8, 16, 32)] + [f"group_n:{g}" for g in (2, 4, 8, 16, 32)] +
             ["hilbert", "die_split:m:group_m:8", "die_split:m:hilbert", "die_split:m:group_m:8:i",
              "die_split:m:group_m:8:p", "die_split:m:group_m:16:p", "die_split:n:group_n:16:p", "die_split:m:hilbert:p",
              "die_split:n:group_m:16:p", "die_split:m:group_n:16:p", "group_m:16:s+a", "group_m:16:s+a+hc", "group_n:8:s+a+hc",
              "die_split:m:group_m:8:p:s+a+hc", "die_split:m:group_m:16:p:s+a+hc"],
 }
-DEFAULT_SCHEME = {"cfg1": "group_m:2", "cfg2": "group_m:8", "cfg3": "die_split:m:group_m:8:p:s+a+hc", "cfg4": "row_major",
+DEFAULT_SCHEME = {"cfg1": "group_m:2", "cfg2": "group_m:8", "cfg3": "die_split:m:group_m:8:p:s+a+hc", "cfg4": "row_major+a+hc",
                   "cfg5": "die_split:m:group_m:16:p:s+a+hc"}
 FALLBACK_SCHEME = {"cfg3": "group_m:8:s+a+hc", "cfg5": "group_m:16:s+a+hc"}   # if the topology probe finds no two-way L2 structure
 FALLBACK_SCHEME_BY_TILE = {("cfg3", "256x512"): "group_m:16:s+a+hc", ("cfg5", "256x512"): "group_m:16:s+a+hc"}

@@ -198,12 +198,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   unit_sync<CG>();
   tcgen05_fence_after();
   const uint32_t tmem_base = *tmem_slot_ptr;
-  // Every launch is made with programmatic stream serialisation: the set-up above may run while the kernel before
-  // this one on the stream is still finishing (its CTAs leaving free the SMs ours start on).  From here on global
-  // memory is touched, so an ordinary launch now waits until that kernel has completed and its writes are visible;
-  // a launch declared independent of it (SP_FLAG_OVERLAP) goes straight on and waits only before it exits.
-  if (!args.overlap) asm volatile("griddepcontrol.wait;" ::: "memory");
-
   // whole tiles of this unit: slots s_first, s_first + s_step, ... below s_end; then its segments of the stream-K tail
   int s_first = unit, s_step = args.units, s_end = args.sk.first_slot;
   if (args.pinned && !args.steal) {
@@ -213,6 +207,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     s_end = die ? T : args.half0;
   }
   const int n_whole = s_first < s_end ? (s_end - s_first + s_step - 1) / s_step : 0;
+  // The first tile of a fixed schedule does not depend on the kernel before this one: the producer warp decodes it now
+  // (arithmetic orders; a table lives in global memory), off the path that starts when that kernel has finished.  For a
+  // grid of a few tiles the chain of integer divisions is a few per cent of the launch.
+  int t_first = -1;
+  if (warp == 0 && !args.sched.use_table && n_whole > 0 && !(DYN && (args.steal || args.clc))) t_first = slot_to_tile(args.sched, s_first);
+  // Every launch is made with programmatic stream serialisation: the set-up above may run while the kernel before
+  // this one on the stream is still finishing (its CTAs leaving free the SMs ours start on).  From here on global
+  // memory is touched, so an ordinary launch now waits until that kernel has completed and its writes are visible;
+  // a launch declared independent of it (SP_FLAG_OVERLAP) goes straight on and waits only before it exits.
+  if (!args.overlap) asm volatile("griddepcontrol.wait;" ::: "memory");
+
   const int n_items = n_whole + sk_segments(args.sk, unit, KB);
   // The i-th piece of work of this unit; slot < 0 when there is none.  Called by whole warps, every role with its own
   // counter.  With cluster launch control the first tile is the cluster's own and every further one comes from a
@@ -321,7 +326,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           }
           __syncwarp();
         }
-        const int t = tile_of_slot(args, s);
+        const int t = (item == 0 && t_first >= 0) ? t_first : tile_of_slot(args, s);
         const int tm = t / Tn, tn = t - tm * Tn;
         const int row0 = tm * TILE_M + (int)rank * 128;
         const int col0 = tn * BN + (int)rank * C::kMmaCols;        // + c * kMmaN for the c-th MMA tile

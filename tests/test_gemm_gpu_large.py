@@ -64,7 +64,7 @@ CASES = [
     ("cfg3", None, [(sp.ROW_MAJOR, {}), (sp.GROUP_M, dict(group=8)), (sp.HILBERT, {}),
               (sp.DIE_SPLIT, dict(split_axis=0, inner_scheme=sp.GROUP_M, inner_group=8)),
               (sp.DIE_SPLIT, dict(split_axis=0, inner_scheme=sp.GROUP_M, inner_group=8, flags=2))]),
-    ("cfg4", None, [(sp.ROW_MAJOR, {}), (sp.GROUP_M, dict(group=4)), (sp.GROUP_N, dict(group=2))]),
+    ("cfg4", None, [(sp.ROW_MAJOR, {}), (sp.ROW_MAJOR, dict(flags=BENCH_FLAGS)), (sp.GROUP_M, dict(group=4)), (sp.GROUP_N, dict(group=2))]),
     ("cfg5", None, [(sp.GROUP_M, dict(group=16)), (sp.HILBERT, {}),
               (sp.DIE_SPLIT, dict(split_axis=0, inner_scheme=sp.GROUP_M, inner_group=8, flags=2))]),
 ]
