@@ -109,3 +109,50 @@ def test_two_level_model_lands_near_the_measured_dram_reads():
     for got, measured in ((gn8, 823), (row, 1141), (gm8, 939), (gn8sa, 678)):
         assert abs(got - measured) <= 0.10 * measured, (got, measured)
     assert gn8sa < gn8 < gm8 < row
+
+
+# DRAM MB read per launch at 8192^3 with the 256x512 tile, from the profiler's counters on B200 (one launch each), for
+# orders spelled as (split axis or None, inner order, band width, serpentine, pinned halves, K alternating).
+MEASURED_8192_WIDE_TILE = [
+    ((None, "row", 1, False, False, False), 1097.1), ((None, "col", 1, False, False, False), 1122.5),
+    ((None, "gm", 2, False, False, False), 1123.1), ((None, "gm", 4, False, False, False), 1174.5),
+    ((None, "gm", 8, False, False, False), 911.6), ((None, "gm", 16, False, False, False), 850.6),
+    ((None, "gn", 2, False, False, False), 1174.4), ((None, "gn", 4, False, False, False), 883.4),
+    ((None, "gn", 8, False, False, False), 820.9), ((None, "gn", 16, False, False, False), 1097.1),
+    ((None, "gm", 8, True, False, False), 827.0), ((None, "gm", 8, False, False, True), 816.9),
+    ((None, "gm", 8, True, False, True), 739.7), ((None, "gm", 16, True, False, True), 692.6),
+    ((None, "gn", 8, True, False, True), 674.0),
+    ((0, "gm", 8, False, False, False), 911.5), ((1, "gm", 8, False, False, False), 935.4),
+    ((0, "gm", 4, False, True, False), 910.5), ((0, "gm", 8, False, True, False), 847.0),
+    ((0, "gm", 16, False, True, False), 1112.3), ((0, "gn", 8, False, True, False), 848.1),
+    ((1, "gm", 8, False, True, False), 962.5), ((1, "gn", 4, False, True, False), 815.3),
+    ((1, "gn", 8, False, True, False), 1085.4),
+    ((0, "gm", 8, True, True, True), 670.2), ((1, "gn", 4, True, True, True), 638.0), ((0, "gn", 8, True, True, True), 665.5),
+]
+
+
+def test_two_level_model_against_every_captured_order_of_the_headline_shape():
+    """27 orders, banded, split, pinned to the halves or not, K one way or alternating: the model lands within 2 % of the
+    counter where K is walked one way and within 7 % where it alternates (it is optimistic there: real units drift out
+    of step).  Pinned halves: the units of die 0 take the first half of the slots, those of die 1 the second."""
+    Tm, Tn, U = 32, 16, 74
+    kw = dict(Tm=Tm, Tn=Tn, K=8192, tile_m=256, tile_n=512, units=U, capacity_per_half=63 << 20)
+    inner_id = {"row": R.ROW_MAJOR, "col": R.COL_MAJOR, "gm": R.GROUP_M, "gn": R.GROUP_N}
+    worst = {False: 0.0, True: 0.0}
+    for (axis, inner, g, serp, pinned, alt), measured in MEASURED_8192_WIDE_TILE:
+        flags = 4 if serp else 0
+        if axis is None:
+            perm = R.tile_map(Tm * 256, Tn * 512, 256, 512, inner_id[inner], R.Params(group=g, flags=flags))
+        else:
+            perm = R.tile_map(Tm * 256, Tn * 512, 256, 512, R.DIE_SPLIT,
+                              R.Params(split_axis=axis, inner_scheme=inner_id[inner], inner_group=g, flags=flags))
+        extra = {}
+        if pinned:
+            n0, h0 = U // 2, len(perm) // 2
+            extra = dict(die_of_unit=lambda u: 0 if u < n0 else 1,
+                         slots_of_unit=lambda u: range(u, h0, n0) if u < n0 else range(h0 + u - n0, len(perm), U - n0))
+        got = L.simulate_two_level(perm, k_alternate=alt, **kw, **extra)["dram_read_bytes"] / 1e6
+        err = abs(got - measured) / measured
+        assert err <= (0.07 if alt else 0.02), ((axis, inner, g, serp, pinned, alt), got, measured)
+        worst[alt] = max(worst[alt], err)
+    assert worst[False] <= 0.02 and worst[True] <= 0.07
