@@ -10,15 +10,19 @@
 //                      reads the tile again and writes exp(x - M) / S.  The second read comes from L2 when the tile is
 //                      still there: phase 2 can walk the slots in the same order as phase 1 or backwards, starting with
 //                      what phase 1 touched last.
-//   single pass     -- a block of whole rows (64 KiB at most) is brought into shared memory once and read from there into
-//                      registers once; maximum, exponentials, sum and the normalised values are all taken there.  Every
-//                      byte crosses HBM once in each direction; the order of the row blocks has nothing left to improve.
-//                      Rows of up to 2048 elements are handled a warp per row (no meeting of warps at all), longer ones by
-//                      all eight warps together (two meetings per block).
+//   single pass     -- a block of whole rows (48 KiB where the row length allows, 64 KiB at most) is brought into shared
+//                      memory once and read from there into registers once; maximum, exponentials, sum and the normalised
+//                      values are all taken there, the results written back to the same buffer and sent out from it by
+//                      one bulk copy.  Every byte crosses HBM once in each direction; the order of the row blocks has
+//                      nothing left to improve.  Rows of up to 1792 elements are handled a warp per row (no meeting of
+//                      warps at all), longer ones by two to twelve warps per row (two meetings per block).
 //
 // All kernels: persistent CTAs (one per SM), one producer warp that brings tiles into a ring of three 64 KiB buffers (a
 // block of whole rows is contiguous in memory: one bulk copy; a 32 x 512 tile: two TMA boxes of 32 rows x 1 KiB;
-// completion counted on an mbarrier), eight consumer warps, 16-byte streaming stores.  Every wait is bounded and reports into the status word like the other kernels.
+// completion counted on an mbarrier) and, where a kernel has output, sends each buffer out again once the consumer warps
+// have left their results in it (16-byte stores from the consumers' registers reached 0.89 of the copy bandwidth at
+// 16384 x 16384, bulk stores 0.98); eight to fifteen consumer warps.  Every wait is bounded and reports into the status
+// word like the other kernels.
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <string.h>
@@ -33,9 +37,13 @@ constexpr uint32_t kSmStageBytes = 65536;
 constexpr int kSmStages = 3;
 constexpr int kSmWarps = 8;                              // consumer warps
 constexpr int kSmThreads = 32 * (kSmWarps + 1);
+// Long rows take up to 15 consumer warps: with two warps per scheduler the chain of shared-memory reads, exponentials and
+// shuffles of a block is latency-bound and, for blocks of several rows, longer than the block's share of the memory time
+// (rows of 4096: 5.2 TB/s with 8 warps).  16 warps with the producer leave 128 registers per thread.
+constexpr int kSmBlockWarpsMax = 16;
 constexpr int kSmMaxRows = 8;                            // single pass, long rows: rows per block
-constexpr int kSmWarpRowLimit = 2048;                    // single pass: rows up to this length are handled a warp per row
-constexpr uint32_t kSmSmem = kSmStages * kSmStageBytes + 1024 /* alignment */ + 64 /* barriers */ + (2 * kSmMaxRows * kSmWarps + 4) * 4;
+constexpr int kSmWarpRowLimit = 1792;                    // single pass: rows up to this length are handled a warp per row
+constexpr uint32_t kSmSmem = kSmStages * kSmStageBytes + 1024 /* alignment */ + 64 /* barriers */ + (2 * kSmMaxRows * kSmBlockWarpsMax + 4) * 4;
 static_assert(kSmTileM * kSmTileN * 4 == kSmStageBytes, "a two-phase tile fills one buffer");
 static_assert(kSmTileM == 4 * kSmWarps, "a warp takes four rows of a two-phase tile");
 
@@ -64,6 +72,9 @@ __device__ __forceinline__ float sm_lds32(uint32_t addr) {
   asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
   return v;
 }
+__device__ __forceinline__ void sm_sts128(uint32_t addr, const float4& v) {
+  asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
 __device__ __forceinline__ void sm_sts32(uint32_t addr, float v) {
   asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
 }
@@ -73,7 +84,15 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
-__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(32 * kSmWarps) : "memory"); }
+// Contiguous bytes from shared to global memory (both 16-byte aligned, size a multiple of 16), bulk-group completion.
+__device__ __forceinline__ void bulk_store(void* dst, uint32_t src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_release(uint32_t bar) {
+  asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+template <int W>
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(32 * W) : "memory"); }
 __device__ __forceinline__ float warp_max(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
@@ -100,8 +119,8 @@ __device__ __forceinline__ SmLayout sm_layout(const uint8_t* smem_raw) {
   l.base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   l.bar_full = l.base + kSmStages * kSmStageBytes;
   l.bar_empty = l.bar_full + 8 * kSmStages;
-  l.red = l.bar_empty + 8 * kSmStages + 16;              // [2][kSmMaxRows][kSmWarps] floats (long rows, single pass)
-  l.fail_flag = l.red + 2 * kSmMaxRows * kSmWarps * 4;
+  l.red = l.bar_empty + 8 * kSmStages + 16;              // [2][kSmMaxRows][consumer warps] floats (long rows, single pass)
+  l.fail_flag = l.red + 2 * kSmMaxRows * kSmBlockWarpsMax * 4;
   return l;
 }
 
@@ -121,10 +140,10 @@ __device__ __forceinline__ int sm_tile_of(const SoftmaxArgs& a, int s) {
   return a.sched.use_table ? __ldg(a.perm + s) : slot_to_tile(a.sched, s);
 }
 
-__device__ __forceinline__ void sm_init(const SmLayout& l) {
+__device__ __forceinline__ void sm_init(const SmLayout& l, int consumer_warps = kSmWarps) {
   if (threadIdx.x == 0) {
     sm_sts32(l.fail_flag, 0.f);
-    for (int i = 0; i < kSmStages; ++i) { mbar_init(l.bar_full + 8 * i, 1); mbar_init(l.bar_empty + 8 * i, kSmWarps); }
+    for (int i = 0; i < kSmStages; ++i) { mbar_init(l.bar_full + 8 * i, 1); mbar_init(l.bar_empty + 8 * i, consumer_warps); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
@@ -137,14 +156,39 @@ constexpr uint32_t kSmBoxBytes = kSmTileM * kSmBoxCols * 4;             // 32 Ki
 // copy brings them all.  Two-phase: the tile comes as two boxes of 32 rows x 256 columns (parts outside the matrix are
 // filled with zeros and never used; a box wholly outside is not requested).
 template <int MODE>
-__device__ __forceinline__ void sm_produce(const SoftmaxArgs& args, const SmLayout& l, const CUtensorMap* tm_in) {
+__device__ __forceinline__ void sm_produce(const SoftmaxArgs& args, const SmLayout& l, const CUtensorMap* tm_in, const CUtensorMap* tm_out) {
+  constexpr bool STORE = MODE != kSmPhase1;      // the first phase leaves only its partials, written by the consumers
   int stage = 0;
   uint32_t phase = 0;
   bool ok = true;
-  for (int s = blockIdx.x; s < args.sched.T && ok; s += gridDim.x) {
+  const int lane = threadIdx.x & 31;
+  // The consumers leave their results in the buffer they were given and hand it back only then; this warp sends the
+  // block out with bulk copies (a block of whole rows is contiguous in the output as in the input: one copy; a tile:
+  // its two boxes, clipped at the matrix edge), waits until they have read the buffer, and fills it again.  Measured
+  // against 16-byte stores from the consumers' registers at 16384 x 16384: 6.36 against 5.77 TB/s.  One lane issues,
+  // commits and waits: bulk groups belong to a thread.
+  auto store_block = [&](int s_prev, int st) {
+    int row0, nrows, col0, ncols;
+    sm_geometry<MODE>(args, sm_tile_of<MODE>(args, s_prev), row0, nrows, col0, ncols);
+    if (lane == 0) {
+      const uint32_t src = l.base + st * kSmStageBytes;
+      if (MODE == kSmSinglePass) {
+        bulk_store(args.out + (size_t)row0 * args.N, src, (uint32_t)nrows * (uint32_t)ncols * 4u);
+      } else {
+        tma_store_2d(tm_out, src, col0, row0);
+        if (ncols > kSmBoxCols) tma_store_2d(tm_out, src + kSmBoxBytes, col0 + kSmBoxCols, row0);
+      }
+      bulk_commit();
+      bulk_wait_read_0();
+    }
+    __syncwarp();
+  };
+  int n_loaded = 0;
+  for (int s = blockIdx.x; s < args.sched.T && ok; s += gridDim.x, ++n_loaded) {
     ok = mbar_wait(l.bar_empty + 8 * stage, phase ^ 1u, args.status, (kRoleSoftmaxLoad << 8) | 1);
     ok = __all_sync(0xffffffffu, ok);
     if (!ok) break;
+    if (STORE && n_loaded >= kSmStages) store_block(s - kSmStages * (int)gridDim.x, stage);
     int row0, nrows, col0, ncols;
     sm_geometry<MODE>(args, sm_tile_of<MODE>(args, s), row0, nrows, col0, ncols);
     const uint32_t full = l.bar_full + 8 * stage, dst = l.base + stage * kSmStageBytes;
@@ -166,95 +210,97 @@ __device__ __forceinline__ void sm_produce(const SoftmaxArgs& args, const SmLayo
   for (int i = 0; i < kSmStages && ok; ++i) {   // no copy may still be in flight towards this CTA when it exits
     ok = mbar_wait(l.bar_empty + 8 * stage, phase ^ 1u, args.status, (kRoleSoftmaxLoad << 8) | 2);
     ok = __all_sync(0xffffffffu, ok);
+    // the last blocks: block n_loaded - kSmStages + i went through this stage, if there was one
+    const int j = n_loaded - kSmStages + i;
+    if (STORE && ok && j >= 0) store_block((int)blockIdx.x + j * (int)gridDim.x, stage);
     if (++stage == kSmStages) { stage = 0; phase ^= 1u; }
   }
+  if (STORE && lane == 0) bulk_wait_all();      // ... nor away from it
   if (!ok) {
     const unsigned long long t0 = globaltimer();
     while (globaltimer() - t0 < 1000000ull) __nanosleep(1000);
   }
 }
 
-// ------------------------------------------------------------------ single pass, long rows: all warps on every row
-// KK = 16-byte units of a row per thread (ceil(N / 1024)), RMAX = the most rows a block can have at that KK.
-template <int KK, int RMAX>
-__global__ void __launch_bounds__(kSmThreads, 1) softmax_block_kernel(const __grid_constant__ CUtensorMap tm_in, const SoftmaxArgs args) {
+// ------------------------------------------------------------------ single pass, long rows: G warps on every row
+// A block has ROWS rows (fewer in the last block) and G * ROWS consumer warps; warp w works on slice w % G of row w / G and
+// a lane owns 16-byte units (slice * 32 + lane) + 32 * G * k, k < UK, of that row.  So a thread reduces one row only, however
+// many rows the block has: one warp reduction and G partials per phase (all warps on every row instead cost a reduction
+// per row and thread, and blocks of four to seven rows ran a fifth to a third below those of one row).  The block is read
+// from shared memory once and then lives in registers; the warps meet twice per block.
+template <int UK, int G, int ROWS>
+__global__ void __launch_bounds__(32 * (G * ROWS + 1), 1) softmax_block_kernel(const __grid_constant__ CUtensorMap tm_in, const __grid_constant__ CUtensorMap tm_out,
+                                                                              const SoftmaxArgs args) {
+  constexpr int W = G * ROWS;
+  static_assert(W <= kSmBlockWarpsMax, "the partials of a block have room for kSmBlockWarpsMax warps");
   extern __shared__ uint8_t smem_raw[];
   const SmLayout l = sm_layout(smem_raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int N = args.N;
   const uint32_t row_pitch = (uint32_t)N * 4u;
-  sm_init(l);
-  if (warp == kSmWarps) { sm_produce<kSmSinglePass>(args, l, &tm_in); return; }
+  sm_init(l, W);
+  if (warp == W) { sm_produce<kSmSinglePass>(args, l, &tm_in, &tm_out); return; }
 
+  const int row = warp / G, slice = warp - row * G;
+  const uint32_t red_max = l.red + (uint32_t)(row * G) * 4u, red_sum = red_max + (uint32_t)kSmBlockWarpsMax * 4u;
   int stage = 0;
   uint32_t phase = 0;
   const int nvec = N >> 2;
   for (int s = blockIdx.x; s < args.sched.T; s += gridDim.x) {
     bool ok = mbar_wait(l.bar_full + 8 * stage, phase, args.status, (kRoleSoftmaxCompute << 8) | 1);
     ok = __all_sync(0xffffffffu, ok);
-    // The eight warps meet at named barriers below, so none may leave on its own: a warp whose wait gave up raises a
-    // flag, goes through the first meeting empty-handed, and all of them leave together right after it.
+    // The warps meet at named barriers below, so none may leave on its own: a warp whose wait gave up raises a flag,
+    // goes through the first meeting empty-handed, and all of them leave together right after it.
     if (!ok && lane == 0) sm_sts32(l.fail_flag, 1.f);
     int row0, nrows, col0, ncols;
     sm_geometry<kSmSinglePass>(args, sm_tile_of<kSmSinglePass>(args, s), row0, nrows, col0, ncols);
-    const uint32_t buf = l.base + stage * kSmStageBytes;
-    // A thread owns 16-byte units tid, tid + 256, ... of each row.  The block is read from shared memory once and then
-    // lives in registers (RMAX rows x KK units per thread, at most 21 units); the reductions of the block's rows are
-    // batched: two meetings per block, not per row.
-    float4 v[RMAX][KK];
-    float acc[RMAX];
+    const bool mine = ok && row < nrows;
+    const uint32_t base = l.base + stage * kSmStageBytes + (uint32_t)row * row_pitch;
+    float4 v[UK];
+    float acc = -INFINITY;
 #pragma unroll
-    for (int r = 0; r < RMAX; ++r) {
-      acc[r] = -INFINITY;
-#pragma unroll
-      for (int k = 0; k < KK; ++k) {
-        const int i = tid + 32 * kSmWarps * k;
-        if (ok && r < nrows && i < nvec) {
-          v[r][k] = sm_lds128(buf + (uint32_t)r * row_pitch + (uint32_t)i * 16u);
-          acc[r] = fmaxf(acc[r], max4(v[r][k]));
-        }
+    for (int k = 0; k < UK; ++k) {
+      const int i = slice * 32 + lane + 32 * G * k;
+      if (mine && i < nvec) {
+        v[k] = sm_lds128(base + (uint32_t)i * 16u);
+        acc = fmaxf(acc, max4(v[k]));
       }
-      acc[r] = warp_max(acc[r]);
-      if (lane == 0) sm_sts32(l.red + (uint32_t)(r * kSmWarps + warp) * 4u, acc[r]);
     }
-    __syncwarp();
-    if (lane == 0) mbar_arrive_relaxed(l.bar_empty + 8 * stage);   // the buffer has been read: the next copy may come
-    consumer_sync();
+    acc = warp_max(acc);
+    if (lane == 0) sm_sts32(red_max + (uint32_t)slice * 4u, acc);
+    consumer_sync<W>();
     if (sm_lds32(l.fail_flag) != 0.f) break;
+    float big = -INFINITY;
 #pragma unroll
-    for (int r = 0; r < RMAX; ++r) {
-      float big = -INFINITY;
+    for (int g = 0; g < G; ++g) big = fmaxf(big, sm_lds32(red_max + (uint32_t)g * 4u));
+    acc = 0.f;
 #pragma unroll
-      for (int w = 0; w < kSmWarps; ++w) big = fmaxf(big, sm_lds32(l.red + (uint32_t)(r * kSmWarps + w) * 4u));
-      acc[r] = 0.f;
-#pragma unroll
-      for (int k = 0; k < KK; ++k)
-        if (r < nrows && tid + 32 * kSmWarps * k < nvec) acc[r] += exp4_sum(v[r][k], big);
-      acc[r] = warp_sum(acc[r]);
-      if (lane == 0) sm_sts32(l.red + (uint32_t)((kSmMaxRows + r) * kSmWarps + warp) * 4u, acc[r]);
-    }
-    consumer_sync();
+    for (int k = 0; k < UK; ++k)
+      if (mine && slice * 32 + lane + 32 * G * k < nvec) acc += exp4_sum(v[k], big);
+    acc = warp_sum(acc);
+    if (lane == 0) sm_sts32(red_sum + (uint32_t)slice * 4u, acc);
+    consumer_sync<W>();
     // (the sums are read below by every warp before any of them can pass the next block's first meeting, after which
     // alone they are rewritten; the maxima were all read before the second meeting)
+    if (mine) {
+      float total = 0.f;
 #pragma unroll
-    for (int r = 0; r < RMAX; ++r) {
-      if (r < nrows) {
-        float total = 0.f;
+      for (int g = 0; g < G; ++g) total += sm_lds32(red_sum + (uint32_t)g * 4u);
+      const float inv = 1.f / total;
 #pragma unroll
-        for (int w = 0; w < kSmWarps; ++w) total += sm_lds32(l.red + (uint32_t)((kSmMaxRows + r) * kSmWarps + w) * 4u);
-        const float inv = 1.f / total;
-        float4* dst = reinterpret_cast<float4*>(args.out + (size_t)(row0 + r) * N);
-#pragma unroll
-        for (int k = 0; k < KK; ++k) {
-          const int i = tid + 32 * kSmWarps * k;
-          if (i < nvec) {
-            float4 o = v[r][k];
-            o.x *= inv; o.y *= inv; o.z *= inv; o.w *= inv;
-            __stcs(dst + i, o);
-          }
+      for (int k = 0; k < UK; ++k) {
+        const int i = slice * 32 + lane + 32 * G * k;
+        if (i < nvec) {
+          float4 o = v[k];
+          o.x *= inv; o.y *= inv; o.z *= inv; o.w *= inv;
+          sm_sts128(base + (uint32_t)i * 16u, o);   // back to where it came from
         }
       }
     }
+    // the results are in the buffer: make them visible to the copy engine, then hand the buffer to the producer warp
+    fence_async_smem();
+    __syncwarp();
+    if (lane == 0) mbar_arrive_release(l.bar_empty + 8 * stage);
     if (++stage == kSmStages) { stage = 0; phase ^= 1u; }
   }
 }
@@ -263,13 +309,14 @@ __global__ void __launch_bounds__(kSmThreads, 1) softmax_block_kernel(const __gr
 // A lane owns 16-byte units lane, lane + 32, ... (KW of them) of a row or row segment; a warp works on ROWS rows at a time
 // (their loads and reductions interleave), rows warp, warp + 8, ... of the tile.
 template <int MODE, int KW, int ROWS>
-__global__ void __launch_bounds__(kSmThreads, 1) softmax_rows_kernel(const __grid_constant__ CUtensorMap tm_in, const SoftmaxArgs args) {
+__global__ void __launch_bounds__(kSmThreads, 1) softmax_rows_kernel(const __grid_constant__ CUtensorMap tm_in, const __grid_constant__ CUtensorMap tm_out,
+                                                                     const SoftmaxArgs args) {
   extern __shared__ uint8_t smem_raw[];
   const SmLayout l = sm_layout(smem_raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int N = args.N, Tn = args.sched.Tn;
   sm_init(l);
-  if (warp == kSmWarps) { sm_produce<MODE>(args, l, &tm_in); return; }
+  if (warp == kSmWarps) { sm_produce<MODE>(args, l, &tm_in, &tm_out); return; }
   // 16-byte unit i of row r of a buffer: rows of N elements back to back (single pass), or two boxes of 32 rows x 1 KiB
   auto unit_addr = [&](uint32_t buf, int r, int i) -> uint32_t {
     if (MODE == kSmSinglePass) return buf + ((uint32_t)r * (uint32_t)N + (uint32_t)i * 4u) * 4u;
@@ -335,7 +382,6 @@ __global__ void __launch_bounds__(kSmThreads, 1) softmax_rows_kernel(const __gri
         const int r = rb + j * kSmWarps;
         if (r >= nrows) continue;
         if (MODE == kSmPhase2) {
-          float4* dst = reinterpret_cast<float4*>(args.out + (size_t)(row0 + r) * N + col0);
 #pragma unroll
           for (int k = 0; k < KW; ++k) {
             const int i = lane + 32 * k;
@@ -343,7 +389,7 @@ __global__ void __launch_bounds__(kSmThreads, 1) softmax_rows_kernel(const __gri
               float4 o = v[j][k];
               exp4_sum(o, big[j]);
               o.x *= inv[j]; o.y *= inv[j]; o.z *= inv[j]; o.w *= inv[j];
-              __stcs(dst + i, o);
+              sm_sts128(unit_addr(buf, r, i), o);       // results replace the inputs; the producer warp sends them out
             }
           }
         } else {
@@ -356,29 +402,34 @@ __global__ void __launch_bounds__(kSmThreads, 1) softmax_rows_kernel(const __gri
             if (lane == 0) args.partial[(size_t)(row0 + r) * Tn + tn] = make_float2(big[j], sum);
           } else {
             const float sc = 1.f / sum;
-            float4* dst = reinterpret_cast<float4*>(args.out + (size_t)(row0 + r) * N);
 #pragma unroll
             for (int k = 0; k < KW; ++k) {
               const int i = lane + 32 * k;
               if (i < nvec) {
                 float4 o = v[j][k];
                 o.x *= sc; o.y *= sc; o.z *= sc; o.w *= sc;
-                __stcs(dst + i, o);
+                sm_sts128(unit_addr(buf, r, i), o);
               }
             }
           }
         }
       }
     }
+    // this warp is done with the buffer: its reads are over (first phase) or its rows hold their results, which must be
+    // visible to the copy engine before the producer warp is told
+    if (MODE != kSmPhase1) fence_async_smem();
     __syncwarp();
-    if (lane == 0) mbar_arrive_relaxed(l.bar_empty + 8 * stage);   // this warp's shared-memory reads of the buffer are over
+    if (lane == 0) {
+      if (MODE == kSmPhase1) mbar_arrive_relaxed(l.bar_empty + 8 * stage);
+      else mbar_arrive_release(l.bar_empty + 8 * stage);
+    }
     if (++stage == kSmStages) { stage = 0; phase ^= 1u; }
   }
 }
 
 template <typename Kernel>
-static int launch_one(Kernel kern, uint64_t& configured, const CUtensorMap& tm_in, const SoftmaxArgs& args, int64_t tiles,
-                      cudaStream_t stream) {
+static int launch_one(Kernel kern, uint64_t& configured, const CUtensorMap& tm_in, const CUtensorMap& tm_out, const SoftmaxArgs& args,
+                      int64_t tiles, cudaStream_t stream, int threads = kSmThreads) {
   cudaError_t e;
   if (first_use_on_this_device(configured)) {
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmSmem);
@@ -390,29 +441,45 @@ static int launch_one(Kernel kern, uint64_t& configured, const CUtensorMap& tm_i
     return SP_ERR_CUDA;
   }
   const int64_t grid = tiles < sms ? tiles : sms;
-  kern<<<(unsigned)grid, kSmThreads, kSmSmem, stream>>>(tm_in, args);
+  kern<<<(unsigned)grid, threads, kSmSmem, stream>>>(tm_in, tm_out, args);
   e = cudaGetLastError();
   if (e != cudaSuccess) { set_error("softmax launch failed: %s", cudaGetErrorString(e)); return SP_ERR_CUDA; }
   return SP_OK;
 }
 
-template <int KK, int RMAX>
+template <int UK, int G, int ROWS>
 static int launch_block(const CUtensorMap& tm, const SoftmaxArgs& args, int64_t tiles, cudaStream_t stream) {
   static uint64_t configured = 0;   // per instantiation, one bit per device
-  return launch_one(softmax_block_kernel<KK, RMAX>, configured, tm, args, tiles, stream);
+  return launch_one(softmax_block_kernel<UK, G, ROWS>, configured, tm, tm, args, tiles, stream, 32 * (G * ROWS + 1));
+}
+// The instantiation whose UK covers `units` 16-byte units per row with G warps on a row: UK = ceil(units / (32 G)), from
+// LO to HI for the row lengths that come with ROWS rows per block.
+template <int G, int ROWS, int LO, int HI>
+static int launch_block_for(int units, const CUtensorMap& tm, const SoftmaxArgs& args, int64_t tiles, cudaStream_t stream) {
+  if constexpr (LO > HI) {
+    set_error("softmax: no kernel for %d units per row with %d warps on each of %d rows", units, G, ROWS);
+    return SP_ERR_UNSUPPORTED;
+  } else {
+    if ((units + 32 * G - 1) / (32 * G) <= LO) return launch_block<LO, G, ROWS>(tm, args, tiles, stream);
+    return launch_block_for<G, ROWS, LO + 1, HI>(units, tm, args, tiles, stream);
+  }
 }
 template <int MODE, int KW, int ROWS>
-static int launch_rows(const CUtensorMap& tm, const SoftmaxArgs& args, int64_t tiles, cudaStream_t stream) {
+static int launch_rows(const CUtensorMap& tm, const CUtensorMap& tm_out, const SoftmaxArgs& args, int64_t tiles, cudaStream_t stream) {
   static uint64_t configured = 0;
-  return launch_one(softmax_rows_kernel<MODE, KW, ROWS>, configured, tm, args, tiles, stream);
+  return launch_one(softmax_rows_kernel<MODE, KW, ROWS>, configured, tm, tm_out, args, tiles, stream);
 }
 
-// Single pass: rows of one block.  A block fills at most one 64 KiB buffer; short rows (a warp per row) come up to 32 to a
-// block (one copy per lane of the producer warp), long rows up to 8.  0 when a row does not fit a buffer.
+// Single pass: rows of one block; 0 when a row does not fit a buffer.  A block is kept to 48 KiB where the row length
+// allows: with three 64 KiB blocks in flight per SM the memory system is over-subscribed and delivers a tenth less
+// (rows of 4096: 5.75 TB/s with blocks of four rows, 6.47 with three; four buffers of 48 KiB are no better than three).
+// Long rows: floor(12288 / N) rows, at least one.  Short rows (a warp per row): a multiple of the eight consumer warps, 8 to 32.
 int softmax_rows_per_block(int64_t N) {
-  const int64_t fit = (int64_t)kSmStageBytes / (N * 4);
-  const int64_t cap = N <= kSmWarpRowLimit ? 32 : kSmMaxRows;
-  return fit < 1 ? 0 : (int)(fit > cap ? cap : fit);
+  if (N * 4 > (int64_t)kSmStageBytes) return 0;
+  const int64_t r = 12288 / N;
+  if (N > kSmWarpRowLimit) return r < 1 ? 1 : (int)r;
+  const int64_t r8 = r / kSmWarps * kSmWarps;
+  return (int)(r8 < kSmWarps ? kSmWarps : r8 > 32 ? 32 : r8);
 }
 
 int launch_softmax(const void* in, void* out, int64_t M, int64_t N, int mode, const Sched& sched, const int32_t* perm_dev,
@@ -428,41 +495,42 @@ int launch_softmax(const void* in, void* out, int64_t M, int64_t N, int mode, co
   args.reverse = mode == SP_SOFTMAX_TWO_PHASE_REVERSED ? 1 : 0;
   args.sched = sched;
   const int64_t T = sched.T;
-  CUtensorMap tm;      // used by the two-phase kernels only; the single-pass kernels take it and ignore it
+  CUtensorMap tm, tm_out;      // used by the two-phase kernels only; the single-pass kernels take them and ignore them
   memset(&tm, 0, sizeof tm);
+  memset(&tm_out, 0, sizeof tm_out);
   if (mode != SP_SOFTMAX_SINGLE_PASS) {
-    const int rc = make_map_plain(&tm, in, M, N, kSmTileM, kSmBoxCols);
+    int rc = make_map_plain(&tm, in, M, N, kSmTileM, kSmBoxCols);
+    if (rc == SP_OK) rc = make_map_plain(&tm_out, out, M, N, kSmTileM, kSmBoxCols);
     if (rc != SP_OK) return rc;
   }
   if (mode == SP_SOFTMAX_SINGLE_PASS) {
     if (N <= kSmWarpRowLimit) {
-      // 16-byte units per lane and row: N / 128 rounded up to a power of two; two rows of a warp in flight together
-      if (N <= 256) return launch_rows<kSmSinglePass, 2, 2>(tm, args, T, stream);
-      if (N <= 512) return launch_rows<kSmSinglePass, 4, 2>(tm, args, T, stream);
-      if (N <= 1024) return launch_rows<kSmSinglePass, 8, 2>(tm, args, T, stream);
-      return launch_rows<kSmSinglePass, 16, 2>(tm, args, T, stream);
+      // 16-byte units per lane and row (N / 128, rounded up to what is instantiated), and how many rows a warp works on
+      // together: two where a block has at least sixteen rows (N <= 768), else its one row
+      if (N <= 256) return launch_rows<kSmSinglePass, 2, 2>(tm, tm_out, args, T, stream);
+      if (N <= 512) return launch_rows<kSmSinglePass, 4, 2>(tm, tm_out, args, T, stream);
+      if (N <= 768) return launch_rows<kSmSinglePass, 6, 2>(tm, tm_out, args, T, stream);
+      if (N <= 1024) return launch_rows<kSmSinglePass, 8, 1>(tm, tm_out, args, T, stream);
+      if (N <= 1536) return launch_rows<kSmSinglePass, 12, 1>(tm, tm_out, args, T, stream);
+      return launch_rows<kSmSinglePass, 14, 1>(tm, tm_out, args, T, stream);
     }
-    // 16-byte units per thread and row, and the most rows a block has at that width (rows x N x 4 <= 64 KiB, <= 8)
-    switch ((int)((N / 4 + 32 * kSmWarps - 1) / (32 * kSmWarps))) {
-      case 3: return launch_block<3, 7>(tm, args, T, stream);
-      case 4: return launch_block<4, 5>(tm, args, T, stream);
-      case 5: return launch_block<5, 3>(tm, args, T, stream);
-      case 6: return launch_block<6, 3>(tm, args, T, stream);
-      case 7: return launch_block<7, 2>(tm, args, T, stream);
-      case 8: return launch_block<8, 2>(tm, args, T, stream);
-      case 9: return launch_block<9, 1>(tm, args, T, stream);
-      case 10: return launch_block<10, 1>(tm, args, T, stream);
-      case 11: return launch_block<11, 1>(tm, args, T, stream);
-      case 12: return launch_block<12, 1>(tm, args, T, stream);
-      case 13: return launch_block<13, 1>(tm, args, T, stream);
-      case 14: return launch_block<14, 1>(tm, args, T, stream);
-      case 15: return launch_block<15, 1>(tm, args, T, stream);
-      default: return launch_block<16, 1>(tm, args, T, stream);
+    // Rows per block decide how many warps share a row; up to 15 consumer warps (with the
+    // producer 16: four per scheduler, 128 registers each).  One row per block: 8 warps for the longest rows, 12 below
+    // (measured: 6.37 against 5.80 TB/s at 16384, 6.08 against 6.60 at 12288).
+    const int units = (int)(N / 4);
+    switch (args.rows_per_block) {
+      case 1: return units > 3072 ? launch_block_for<8, 1, 13, 16>(units, tm, args, T, stream)     // N in (12288, 16384]
+                                  : launch_block_for<12, 1, 5, 8>(units, tm, args, T, stream);     // (6144, 12288]
+      case 2: return launch_block_for<6, 2, 6, 8>(units, tm, args, T, stream);                      // (4096, 6144]
+      case 3: return launch_block_for<4, 3, 7, 8>(units, tm, args, T, stream);                      // (3072, 4096]
+      case 4: return launch_block_for<3, 4, 7, 8>(units, tm, args, T, stream);                      // (2457, 3072]
+      case 5: return launch_block_for<3, 5, 6, 7>(units, tm, args, T, stream);                      // (2048, 2457]
+      default: return launch_block_for<2, 6, 8, 8>(units, tm, args, T, stream);                     // (1792, 2048]
     }
   }
-  int rc = launch_rows<kSmPhase1, kSmTileN / 128, 4>(tm, args, T, stream);
+  int rc = launch_rows<kSmPhase1, kSmTileN / 128, 4>(tm, tm_out, args, T, stream);
   if (rc != SP_OK) return rc;
-  return launch_rows<kSmPhase2, kSmTileN / 128, 4>(tm, args, T, stream);
+  return launch_rows<kSmPhase2, kSmTileN / 128, 4>(tm, tm_out, args, T, stream);
 }
 
 }  // namespace sp

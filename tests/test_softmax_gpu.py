@@ -35,7 +35,7 @@ def close(got, ref):
 
 
 # sizes span several 32 x 512 tiles with ragged edges both ways, one tile, one row, one 16-byte unit per row, rows of
-# 16384 (one row per single-pass block) and 2048 (eight)
+# 16384 (one row per single-pass block) and 2048 (six)
 @pytest.mark.parametrize("M,N", [(32, 512), (100, 1300), (257, 4100), (1, 4), (3, 16384), (70, 2048), (9, 8), (33, 520)])
 @pytest.mark.parametrize("mode", MODES)
 def test_matches_the_definition(M, N, mode):
@@ -109,3 +109,21 @@ def test_rows_longer_than_a_buffer_take_the_two_phase_form():
     ref = SM.softmax(x)
     for mode in MODES[1:]:
         assert close(run(x, mode, sp.GROUP_N, group=7), ref)
+
+
+def test_single_pass_at_every_row_length_of_the_long_row_kernels():
+    """Rows of 1796 to 16384 elements in steps of 4: every pairing of rows per block, warps per row and units per lane the
+    long-row dispatch can choose, each with a last block that is short of rows."""
+    rng = np.random.default_rng(77)
+    base = (rng.standard_normal((17, 16384)) * 3.0).astype(np.float32)
+    worst = 0.0
+    for N in range(1796, 16385, 4):
+        rows = max(1, 12288 // N)
+        M = 2 * rows + 1 if N % 64 == 0 else rows + 1
+        x = np.ascontiguousarray(base[:M, 16384 - N:])
+        x[M - 1, N - 1] += 30.0
+        got = run(x, sp.SOFTMAX_SINGLE_PASS)
+        ref = SM.softmax(x)
+        assert close(got, ref), N
+        worst = max(worst, float(np.abs(got.astype(np.float64).sum(axis=1) - 1.0).max()))
+    assert worst <= 1e-5
