@@ -9,11 +9,11 @@
 //
 // Per tile: one TMA load of the tile plus its halo, 66 rows x 136 columns (the box starts 4 columns, i.e. 16 bytes,
 // left of the tile: a TMA copy must start on a 16-byte boundary; out-of-range parts are filled with zeros and never
-// used, because rim points copy their input), into a ring of four buffers.  Eight consumer warps take eight rows
+// used, because rim points copy their input), into a ring of three buffers.  Eight consumer warps take eight rows
 // each: a lane owns four adjacent columns, keeps a three-row window in registers, gets its west / east neighbours
-// from the adjacent lanes by shuffle (the outermost lanes read the halo columns), and writes 16 bytes per row
-// straight to global memory: a warp instruction stores 512 contiguous bytes.  Memory bound: every input byte is
-// read from HBM once (halos come from L2), every output byte written once.
+// from the adjacent lanes by shuffle (the outermost lanes read the halo columns), and writes 16 bytes per row into a
+// staging slice of its warp (8 rows x 512 bytes, two per warp), which lane 0 then sends out with one TMA store.
+// Memory bound: every input byte is read from HBM once (halos come from L2), every output byte written once.
 #include <cuda.h>
 #include <cuda_runtime.h>
 
@@ -26,12 +26,17 @@ constexpr int kStTileM = SP_STENCIL_TILE_M, kStTileN = SP_STENCIL_TILE_N;
 constexpr int kStBoxRows = kStTileM + 2, kStBoxCols = kStTileN + 8;
 constexpr uint32_t kStBoxBytes = kStBoxRows * kStBoxCols * 4;          // 35904
 constexpr uint32_t kStBuf = (kStBoxBytes + 1023u) & ~1023u;             // buffers stay 1 KiB aligned
-constexpr int kStStages = 4;     // measured: 5 and 6 buffers are no faster; two or three CTAs per SM with fewer buffers
-constexpr int kStCtasPerSm = 1;  //   each are 12-15 % slower (more tiles in flight at once, poorer DRAM page locality)
+constexpr int kStStages = 3;     // measured: four to six buffers are no faster (row-major 6.31 TB/s with four, 6.40 with three);
+constexpr int kStCtasPerSm = 1;  //   two or three CTAs per SM with fewer buffers each are 12-15 % slower (more tiles in flight
+                                 //   at once, poorer DRAM page locality)
 constexpr int kStConsumerWarps = 8;
 constexpr int kStRowsPerWarp = kStTileM / kStConsumerWarps;
 constexpr int kStThreads = 32 * (kStConsumerWarps + 1);
-constexpr uint32_t kStSmem = kStStages * kStBuf + 1024 + 128;
+// Output: every consumer warp owns two staging slices of its 8 rows x 128 columns and sends a finished slice out with one
+// TMA store (16-byte stores from registers reached 0.945 of the copy bandwidth in row-major order, 0.82-0.89 otherwise).
+constexpr uint32_t kStOutSlice = kStRowsPerWarp * kStTileN * 4;                      // 4 KiB
+constexpr uint32_t kStOutBytes = kStConsumerWarps * 2 * kStOutSlice;                 // 64 KiB
+constexpr uint32_t kStSmem = kStStages * kStBuf + kStOutBytes + 1024 + 128;
 static_assert(kStTileN == 128, "a lane owns four of the 128 columns of a tile row");
 
 struct StencilArgs {
@@ -58,10 +63,11 @@ __device__ __forceinline__ float lds32(uint32_t addr) {
 }
 
 __global__ void __launch_bounds__(kStThreads, kStCtasPerSm)
-stencil_kernel(const __grid_constant__ CUtensorMap tmIn, const StencilArgs args) {
+stencil_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ CUtensorMap tmOut, const StencilArgs args) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t bar_full = base + kStStages * kStBuf, bar_empty = bar_full + 8 * kStStages;
+  const uint32_t out_base = base + kStStages * kStBuf;
+  const uint32_t bar_full = out_base + kStOutBytes, bar_empty = bar_full + 8 * kStStages;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int T = args.sched.T, Tn = args.sched.Tn;
   const int step = gridDim.x;
@@ -110,10 +116,15 @@ stencil_kernel(const __grid_constant__ CUtensorMap tmIn, const StencilArgs args)
   int stage = 0;
   uint32_t phase = 0;
   bool ok = true;
+  uint32_t parity = 0;                             // which of this warp's two output slices
   for (int s = blockIdx.x; s < T && ok; s += step) {
     ok = mbar_wait(bar_full + 8 * stage, phase, args.status, (kRoleStencilCompute << 8) | 1);
     ok = __all_sync(0xffffffffu, ok);
     if (!ok) break;
+    // the store issued two tiles ago (lane 0's: bulk groups belong to a thread) has read the slice about to be refilled
+    if (lane == 0) bulk_wait_read_1();
+    __syncwarp();
+    const uint32_t slice = out_base + ((uint32_t)warp * 2u + parity) * kStOutSlice + (uint32_t)lane * 16u;
     const int t = tile_of(s);
     const int tm = t / Tn, tn = t - tm * Tn;
     const int gj = tn * kStTileN + 4 * lane;       // first of this lane's four columns
@@ -137,24 +148,33 @@ stencil_kernel(const __grid_constant__ CUtensorMap tmIn, const StencilArgs args)
       if (gi == 0 || gi == args.M - 1) o = cur;    // the rim keeps its input
       if (gj == 0) o.x = cur.x;
       if (gj + 3 == args.N - 1) o.w = cur.w;
-      if (gi < args.M && gj < args.N)              // N is a multiple of 4: a lane's four columns are in range together
-        __stcs(reinterpret_cast<float4*>(args.out + (size_t)gi * args.N + gj), o);
+      // (points beyond the grid's edge are written too: the store below is clipped there)
+      st_shared_16(slice + (uint32_t)k * (kStTileN * 4u), __float_as_uint(o.x), __float_as_uint(o.y), __float_as_uint(o.z),
+                   __float_as_uint(o.w));
       up = cur;
       cur = down;
     }
+    fence_async_smem();                            // the slice must be visible to the copy engine
     __syncwarp();
-    // relaxed: a releasing arrive would first wait for this warp's global stores to be acknowledged (measured: the
-    // largest stall of the kernel); the buffer only needs the warp's shared-memory reads to be over, and they are,
-    // their values having been used
-    if (lane == 0) mbar_arrive_relaxed(bar_empty + 8 * stage);
+    if (lane == 0) {
+      // relaxed: the input buffer only needs the warp's shared-memory reads to be over, and they are, their values
+      // having been used
+      mbar_arrive_relaxed(bar_empty + 8 * stage);
+      const int gi0 = tm * kStTileM + r0;
+      if (gi0 < args.M) tma_store_2d(&tmOut, slice, tn * kStTileN, gi0);   // lane 0: `slice` is the slice's first byte
+      bulk_commit();
+    }
+    parity ^= 1u;
     if (++stage == kStStages) { stage = 0; phase ^= 1u; }
   }
+  if (lane == 0) bulk_wait_all();
 }
 
 int launch_stencil(const void* in, void* out, int64_t M, int64_t N, float c_center, float c_neighbor, const Sched& sched,
                    const int32_t* perm_dev, int32_t* status_dev, cudaStream_t stream) {
-  CUtensorMap tmIn;
+  CUtensorMap tmIn, tmOut;
   int rc = make_map_plain(&tmIn, in, M, N, kStBoxRows, kStBoxCols);
+  if (rc == SP_OK) rc = make_map_plain(&tmOut, out, M, N, kStRowsPerWarp, kStTileN);
   if (rc != SP_OK) return rc;
   static uint64_t configured = 0;   // one bit per device
   cudaError_t e;
@@ -176,7 +196,7 @@ int launch_stencil(const void* in, void* out, int64_t M, int64_t N, float c_cent
   args.M = (int)M; args.N = (int)N;
   args.c_center = c_center; args.c_neighbor = c_neighbor;
   args.sched = sched;
-  stencil_kernel<<<(unsigned)grid, kStThreads, kStSmem, stream>>>(tmIn, args);
+  stencil_kernel<<<(unsigned)grid, kStThreads, kStSmem, stream>>>(tmIn, tmOut, args);
   e = cudaGetLastError();
   if (e != cudaSuccess) { set_error("stencil launch failed: %s", cudaGetErrorString(e)); return SP_ERR_CUDA; }
   return SP_OK;
