@@ -45,7 +45,8 @@ constexpr int kSmMaxRows = 8;                            // single pass, long ro
 constexpr int kSmWarpRowLimit = 1792;                    // single pass: rows up to this length are handled a warp per row
 constexpr uint32_t kSmSmem = kSmStages * kSmStageBytes + 1024 /* alignment */ + 64 /* barriers */ + (2 * kSmMaxRows * kSmBlockWarpsMax + 4) * 4;
 static_assert(kSmTileM * kSmTileN * 4 == kSmStageBytes, "a two-phase tile fills one buffer");
-static_assert(kSmTileM == 4 * kSmWarps, "a warp takes four rows of a two-phase tile");
+constexpr int kSmPhaseWarps = 16;                       // two-phase kernels: consumer warps
+static_assert(kSmTileM % kSmPhaseWarps == 0, "the rows of a two-phase tile are shared out evenly");
 
 struct SoftmaxArgs {
   const float* in;
@@ -307,16 +308,16 @@ __global__ void __launch_bounds__(32 * (G * ROWS + 1), 1) softmax_block_kernel(c
 
 // ------------------------------------------------------------------ a warp per row: short rows (single pass), and the two phases
 // A lane owns 16-byte units lane, lane + 32, ... (KW of them) of a row or row segment; a warp works on ROWS rows at a time
-// (their loads and reductions interleave), rows warp, warp + 8, ... of the tile.
-template <int MODE, int KW, int ROWS>
-__global__ void __launch_bounds__(kSmThreads, 1) softmax_rows_kernel(const __grid_constant__ CUtensorMap tm_in, const __grid_constant__ CUtensorMap tm_out,
+// (their loads and reductions interleave), rows warp, warp + W, ... of the tile (W consumer warps).
+template <int MODE, int KW, int ROWS, int W>
+__global__ void __launch_bounds__(32 * (W + 1), 1) softmax_rows_kernel(const __grid_constant__ CUtensorMap tm_in, const __grid_constant__ CUtensorMap tm_out,
                                                                      const SoftmaxArgs args) {
   extern __shared__ uint8_t smem_raw[];
   const SmLayout l = sm_layout(smem_raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int N = args.N, Tn = args.sched.Tn;
-  sm_init(l);
-  if (warp == kSmWarps) { sm_produce<MODE>(args, l, &tm_in, &tm_out); return; }
+  sm_init(l, W);
+  if (warp == W) { sm_produce<MODE>(args, l, &tm_in, &tm_out); return; }
   // 16-byte unit i of row r of a buffer: rows of N elements back to back (single pass), or two boxes of 32 rows x 1 KiB
   auto unit_addr = [&](uint32_t buf, int r, int i) -> uint32_t {
     if (MODE == kSmSinglePass) return buf + ((uint32_t)r * (uint32_t)N + (uint32_t)i * 4u) * 4u;
@@ -334,13 +335,13 @@ __global__ void __launch_bounds__(kSmThreads, 1) softmax_rows_kernel(const __gri
     const uint32_t buf = l.base + stage * kSmStageBytes;
     const int nvec = ncols >> 2;
     const int tn = col0 / kSmTileN;
-    for (int rb = warp; rb < nrows; rb += kSmWarps * ROWS) {
+    for (int rb = warp; rb < nrows; rb += W * ROWS) {
       float4 v[ROWS][KW];
       float m[ROWS];
       float2 part[ROWS];                       // phase 2: this lane's share of the row's partials, folded as they come
 #pragma unroll
       for (int j = 0; j < ROWS; ++j) {
-        const int r = rb + j * kSmWarps;
+        const int r = rb + j * W;
         m[j] = -INFINITY;
         part[j] = make_float2(-INFINITY, 0.f);
         if (r < nrows) {
@@ -379,7 +380,7 @@ __global__ void __launch_bounds__(kSmThreads, 1) softmax_rows_kernel(const __gri
       }
 #pragma unroll
       for (int j = 0; j < ROWS; ++j) {
-        const int r = rb + j * kSmWarps;
+        const int r = rb + j * W;
         if (r >= nrows) continue;
         if (MODE == kSmPhase2) {
 #pragma unroll
@@ -464,10 +465,10 @@ static int launch_block_for(int units, const CUtensorMap& tm, const SoftmaxArgs&
     return launch_block_for<G, ROWS, LO + 1, HI>(units, tm, args, tiles, stream);
   }
 }
-template <int MODE, int KW, int ROWS>
+template <int MODE, int KW, int ROWS, int W = kSmWarps>
 static int launch_rows(const CUtensorMap& tm, const CUtensorMap& tm_out, const SoftmaxArgs& args, int64_t tiles, cudaStream_t stream) {
   static uint64_t configured = 0;
-  return launch_one(softmax_rows_kernel<MODE, KW, ROWS>, configured, tm, tm_out, args, tiles, stream);
+  return launch_one(softmax_rows_kernel<MODE, KW, ROWS, W>, configured, tm, tm_out, args, tiles, stream, 32 * (W + 1));
 }
 
 // Single pass: rows of one block; 0 when a row does not fit a buffer.  A block is kept to 48 KiB where the row length
@@ -528,9 +529,10 @@ int launch_softmax(const void* in, void* out, int64_t M, int64_t N, int mode, co
       default: return launch_block_for<2, 6, 8, 8>(units, tm, args, T, stream);                     // (1792, 2048]
     }
   }
-  int rc = launch_rows<kSmPhase1, kSmTileN / 128, 4>(tm, tm_out, args, T, stream);
+  // sixteen consumer warps, two rows of the tile each
+  int rc = launch_rows<kSmPhase1, kSmTileN / 128, kSmTileM / kSmPhaseWarps, kSmPhaseWarps>(tm, tm_out, args, T, stream);
   if (rc != SP_OK) return rc;
-  return launch_rows<kSmPhase2, kSmTileN / 128, 4>(tm, tm_out, args, T, stream);
+  return launch_rows<kSmPhase2, kSmTileN / 128, kSmTileM / kSmPhaseWarps, kSmPhaseWarps>(tm, tm_out, args, T, stream);
 }
 
 }  // namespace sp
