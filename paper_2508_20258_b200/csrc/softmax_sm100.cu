@@ -41,7 +41,7 @@ constexpr int kSmThreads = 32 * (kSmWarps + 1);
 // shuffles of a block is latency-bound and, for blocks of several rows, longer than the block's share of the memory time
 // (rows of 4096: 5.2 TB/s with 8 warps).  16 warps with the producer leave 128 registers per thread.
 constexpr int kSmBlockWarpsMax = 16;
-constexpr int kSmMaxRows = 8;                            // single pass, long rows: rows per block
+constexpr int kSmMaxRows = 8;                            // single pass, long rows: room for the partials of a block (it has at most six rows)
 constexpr int kSmWarpRowLimit = 1792;                    // single pass: rows up to this length are handled a warp per row
 constexpr uint32_t kSmSmem = kSmStages * kSmStageBytes + 1024 /* alignment */ + 64 /* barriers */ + (2 * kSmMaxRows * kSmBlockWarpsMax + 4) * 4;
 static_assert(kSmTileM * kSmTileN * 4 == kSmStageBytes, "a two-phase tile fills one buffer");
