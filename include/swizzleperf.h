@@ -306,7 +306,7 @@ int sp_stencil2d(const void* in, void* out, int64_t M, int64_t N, float c_center
  *                                        SP_ERR_UNSUPPORTED.  `scheme` / `params` order the row blocks, as for
  *                                        sp_tile_map(M, N, rows, N, ...) with, in integer arithmetic, rows =
  *                                        max(1, 12288 / N) for N > 1792 (blocks of at most 48 KiB, several warps on a
- *                                        row) and rows = min(32, max(8, 12288 / N / 8 * 8)) for N <= 1792 (a warp per row).
+ *                                        row) and rows = min(96, max(8, 12288 / N / 8 * 8)) for N <= 1792 (a warp per row).
  *   mode SP_SOFTMAX_TWO_PHASE          : the matrix is cut into SP_SOFTMAX_TILE_M x SP_SOFTMAX_TILE_N tiles, ordered exactly as
  *                                        for sp_tile_map(M, N, 32, 512, ...).  A first launch leaves per tile and row
  *                                        the partial maximum and partial sum; a second one combines them per row, reads

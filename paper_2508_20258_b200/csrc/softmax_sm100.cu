@@ -55,7 +55,7 @@ struct SoftmaxArgs {
   const int32_t* perm;
   int32_t* status;
   int M, N;
-  int rows_per_block;    // single pass: rows of one block (1..32); a block's rows are contiguous in memory
+  int rows_per_block;    // single pass: rows of one block (1..96); a block's rows are contiguous in memory
   int reverse;           // phase 2: slot s works on the tile of slot T - 1 - s
   Sched sched;
 };
@@ -474,13 +474,13 @@ static int launch_rows(const CUtensorMap& tm, const CUtensorMap& tm_out, const S
 // Single pass: rows of one block; 0 when a row does not fit a buffer.  A block is kept to 48 KiB where the row length
 // allows: with three 64 KiB blocks in flight per SM the memory system is over-subscribed and delivers a tenth less
 // (rows of 4096: 5.75 TB/s with blocks of four rows, 6.47 with three; four buffers of 48 KiB are no better than three).
-// Long rows: floor(12288 / N) rows, at least one.  Short rows (a warp per row): a multiple of the eight consumer warps, 8 to 32.
+// Long rows: floor(12288 / N) rows, at least one.  Short rows (a warp per row): a multiple of the eight consumer warps, 8 to 96.
 int softmax_rows_per_block(int64_t N) {
   if (N * 4 > (int64_t)kSmStageBytes) return 0;
   const int64_t r = 12288 / N;
   if (N > kSmWarpRowLimit) return r < 1 ? 1 : (int)r;
   const int64_t r8 = r / kSmWarps * kSmWarps;
-  return (int)(r8 < kSmWarps ? kSmWarps : r8 > 32 ? 32 : r8);
+  return (int)(r8 < kSmWarps ? kSmWarps : r8 > 96 ? 96 : r8);
 }
 
 int launch_softmax(const void* in, void* out, int64_t M, int64_t N, int mode, const Sched& sched, const int32_t* perm_dev,

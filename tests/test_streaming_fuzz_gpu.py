@@ -80,7 +80,7 @@ def test_softmax_random_shapes_modes_and_orders(seed):
         if N > 16384 and mode == sp.SOFTMAX_SINGLE_PASS:
             mode = sp.SOFTMAX_TWO_PHASE                         # a single pass holds a whole row in one 64 KiB buffer
         if mode == sp.SOFTMAX_SINGLE_PASS:                          # blocks of whole rows: a grid of one column
-            rows = min(32, max(8, 12288 // N // 8 * 8)) if N <= 1792 else max(1, 12288 // N)   # the header's rule
+            rows = min(96, max(8, 12288 // N // 8 * 8)) if N <= 1792 else max(1, 12288 // N)   # the header's rule
             grid = (-(-M // rows), 1)
         else:
             grid = (-(-M // sp.SOFTMAX_TILE[0]), -(-N // sp.SOFTMAX_TILE[1]))
