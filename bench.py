@@ -218,8 +218,8 @@ def sustained_leg(fn, flops, stream, gpu_index, seconds=4.0):
 
 def workloads_block(sp, names, peaks, stream):
     """The other named workloads, each timed briefly in the same process: the fastest known (tile, order) for it beside
-    row-major on the same tile (alternating blocks of a quarter of a second, mean of two), and the workload's nominal tile when that is another
-    one.  For the launch-bound 512^3 also what a call costs on the host and how long one launch takes from call to
+    row-major on the same tile (alternating blocks of a quarter of a second, mean of two; best of four for the launch-bound 512^3), `torch.matmul`
+    in the same alternation as context where the output is bf16, and the workload's nominal tile when that is another one.  For the launch-bound 512^3 also what a call costs on the host and how long one launch takes from call to
     completion."""
     import torch
     out = {}
@@ -261,16 +261,33 @@ def workloads_block(sp, names, peaks, stream):
         # traffic turns into clock and time (in a burst of a few milliseconds every order runs at the full clock)
         n = int(max(10, min(20000, 250.0 / est)))
         ms = {k: [] for k, _, _ in arms}
-        for _ in range(2):
+        lib_ms = []                # torch.matmul on the same tensors in the same alternation (bf16 output only): context
+        if not out_f32:
+            for _ in range(3):
+                torch.matmul(dA, dB, out=dC)
+        launch_bound = flops < 1e9      # 512^3: host and launch jitter is one-sided, so more rounds and the best of them
+        for _ in range(4 if launch_bound else 2):
             for k, t_, s_ in arms:
                 ms[k].append(time_steps(sp, dA, dB, dC, *arm(t_, s_), n, stream) / n)
-        med = {k: sum(v) / len(v) for k, v in ms.items()}
+            if not out_f32:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                for _ in range(n):
+                    torch.matmul(dA, dB, out=dC)
+                e1.record(stream)
+                e1.synchronize()
+                lib_ms.append(e0.elapsed_time(e1) / n)
+        med = {k: (min(v) if launch_bound else sum(v) / len(v)) for k, v in ms.items()}
         rec = {"shape": [w.M, w.N, w.K], "out": w.out_dtype, "tile": tile, "scheme": spec, "launches_per_block": n,
                "ms": med["best"], "tflops": flops / med["best"] / 1e9,
                "frac_of_sustained_peak": flops / med["best"] / 1e9 / peaks["bf16_tflops_sustained"],
                "row_major_tflops": flops / med["row_major"] / 1e9, "speedup_over_row_major": med["row_major"] / med["best"]}
         if "nominal_tile" in med:
             rec["nominal_tile"] = {"tile": nominal_tile, "scheme": arms[2][2], "tflops": flops / med["nominal_tile"] / 1e9}
+        if lib_ms:
+            lib = sum(lib_ms) / len(lib_ms)
+            rec["cublas_context"] = {"tflops": flops / lib / 1e9, "ours_over_it": lib / med["best"],
+                                     "note": "torch.matmul in the same alternating blocks; context only, not a target"}
         if flops < 1e9:      # launch-bound: what a call costs
             scheme, p = arm(tile, spec)
             torch.cuda.synchronize()
