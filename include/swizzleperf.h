@@ -335,7 +335,8 @@ int sp_softmax(const void* in, void* out, int64_t M, int64_t N, int32_t mode, in
  * loop of the Python package does that).  Rule: among the supported tiles, the one with the least estimated time
  * waves x tile area / (CTAs per tile x relative efficiency of the tile shape), waves = ceil(T / units), units = what
  * sp_gemm_units reports on the current device, or, with no device present, 74 CTA pairs / 148 CTAs; row-major when A and B together are at most 64 MiB (they stay in L2) or the tile grid is at most
- * ten tiles wide, column-major when it is at most ten tiles tall, else bands of 8 tile columns (256x512 tile) or 8
+ * ten tiles wide, column-major when it is at most ten tiles tall (both with SP_FLAG_K_ALTERNATE and
+ * SP_FLAG_HINT_C_EVICT_FIRST when A and B together exceed 64 MiB), else bands of 8 tile columns (256x512 tile) or 8
  * tile rows (other tiles), walked serpentine-wise with SP_FLAG_K_ALTERNATE and SP_FLAG_HINT_C_EVICT_FIRST (the rounding
  * of C then depends on the order, within the usual tolerance); SP_FLAG_STREAM_K is set when the tiles fill at most half of the units and K is at least
  * 2048 (C then differs in rounding order from a launch without the flag).  Host code; no GPU needed.

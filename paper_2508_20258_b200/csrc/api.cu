@@ -803,10 +803,16 @@ int sp_recommend(int64_t M, int64_t N, int64_t K, int32_t out_dtype, int32_t b_l
   // (tall), plain row-major (column-major) already does that; else bands of eight.
   const double operands = 2.0 * ((double)M * (double)K + (double)K * (double)N);
   const int64_t Tm = (M + params->tile_m - 1) / params->tile_m, Tn = (N + params->tile_n - 1) / params->tile_n;
+  // A narrow grid whose operands do not fit in L2 still re-reads the long operand's panels round after round: walking K
+  // in alternating directions lets a round start on what the last one left (16384x2048x8192: 494 -> 407 MB of DRAM
+  // reads, +1 to +4 % in time), and C stores that give way first keep it there.
+  const uint32_t narrow_flags = operands > 64.0 * 1048576.0 ? (SP_FLAG_K_ALTERNATE | SP_FLAG_HINT_C_EVICT_FIRST) : 0u;
   if (operands <= 64.0 * 1048576.0 || Tn <= 10) {
     *scheme = SP_ROW_MAJOR;
+    params->flags |= narrow_flags;
   } else if (Tm <= 10) {
     *scheme = SP_COL_MAJOR;
+    params->flags |= narrow_flags;
   } else {
     *scheme = params->tile_n == 512 ? SP_GROUP_N : SP_GROUP_M;
     params->group = 8;

@@ -228,6 +228,8 @@ def test_recommendation_is_valid_and_matches_what_the_sweeps_found():
     bands = sp.FLAG_SERPENTINE | sp.FLAG_K_ALTERNATE | sp.FLAG_HINT_C_EVICT_FIRST
     assert sp.recommend(8192, 8192, 8192)[1].flags == bands and sp.recommend(16384, 16384, 4096)[1].flags == bands
     assert sp.recommend(512, 512, 512)[1].flags == 0 and sp.recommend(4096, 4096, 4096)[1].flags == 0
+    # a narrow grid whose operands exceed L2: row-major, K alternating, evict_first C stores
+    assert sp.recommend(16384, 2048, 8192)[1].flags == sp.FLAG_K_ALTERNATE | sp.FLAG_HINT_C_EVICT_FIRST
     rng = np.random.default_rng(0)
     for _ in range(200):                                  # always a supported tile and a bijective order
         M, N, K = (int(rng.integers(1, 40000)), int(rng.integers(1, 5000)) * 8, int(rng.integers(1, 3000)) * 8)
