@@ -211,9 +211,12 @@ def sustained_leg(fn, flops, stream, gpu_index, seconds=4.0):
     ms = e0.elapsed_time(e1)
     c = sampler.summary(t0, t1)
     inside = [x[1] for x in sampler.samples if t0 <= x[0] <= t1]
+    watts = c.get("power_w")       # board power, median over the stretch: at the power limit time is energy / power
     return {"launches": n, "seconds": ms / 1e3, "ms_per_launch": ms / n, "tflops": flops * n / ms / 1e9,
             "clocks": c, "sm_mhz_min": min(inside) if inside else None, "sm_mhz_max": max(inside) if inside else None,
-            "sm_cycles_per_launch": None if not c.get("sm_mhz") else ms / n * 1e3 * c["sm_mhz"]}
+            "sm_cycles_per_launch": None if not c.get("sm_mhz") else ms / n * 1e3 * c["sm_mhz"],
+            "joules_per_launch": None if not watts else watts * ms / n / 1e3,
+            "pj_per_flop": None if not watts else watts * ms / n / 1e3 / flops * 1e12}
 
 
 def workloads_block(sp, names, peaks, stream):
@@ -538,8 +541,9 @@ def run_ours(args) -> int:
             time.sleep(1.0)
             ref = torch.empty_like(dC)
             lib = sustained_leg(lambda: torch.matmul(dA, dB, out=ref), flops, stream, local_rank, args.sustained_seconds)
-            cublas["sustained"] = {k: lib[k] for k in ("tflops", "seconds", "sm_cycles_per_launch")}
+            cublas["sustained"] = {k: lib[k] for k in ("tflops", "seconds", "sm_cycles_per_launch", "joules_per_launch", "pj_per_flop")}
             cublas["sustained"]["sm_mhz"] = lib["clocks"]["sm_mhz"]
+            cublas["sustained"]["power_w"] = lib["clocks"].get("power_w")
             sustained["over_cublas_same_run"] = sustained["tflops"] / lib["tflops"]
             del ref
     assert sp.get_status() == 0

@@ -15,7 +15,7 @@ from typing import Dict, List, Optional
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons of one GPU in a background thread.
+    """Samples SM clock, throttle reasons and board power of one GPU in a background thread.
 
     Uses NVML when the Python binding is importable, else polls ``nvidia-smi``.  It only
     reads; it never changes a setting of the GPU.
@@ -27,7 +27,7 @@ class ClockSampler:
     def __init__(self, index: int = 0, period_s: float = 0.01):
         self.index = index
         self.period_s = period_s
-        self.samples: List[tuple] = []      # (t, sm_mhz, reasons_bitmask)
+        self.samples: List[tuple] = []      # (t, sm_mhz, reasons_bitmask, watts or None)
         self.max_mhz: Optional[float] = None
         self._stop = threading.Event()
         self._thread: Optional[threading.Thread] = None
@@ -51,20 +51,28 @@ class ClockSampler:
             try:
                 mhz = float(n.nvmlDeviceGetClockInfo(self._handle, n.NVML_CLOCK_SM))
                 reasons = int(n.nvmlDeviceGetCurrentClocksEventReasons(self._handle))
-                self.samples.append((time.perf_counter(), mhz, reasons))
+                try:
+                    watts = n.nvmlDeviceGetPowerUsage(self._handle) / 1000.0
+                except Exception:
+                    watts = None
+                self.samples.append((time.perf_counter(), mhz, reasons, watts))
             except Exception:
                 pass
             self._stop.wait(self.period_s)
 
     def _loop_smi(self) -> None:
-        q = "clocks.sm,clocks.max.sm,clocks_event_reasons.active"
+        q = "clocks.sm,clocks.max.sm,clocks_event_reasons.active,power.draw"
         while not self._stop.is_set():
             try:
                 out = subprocess.run(["nvidia-smi", f"--id={self.index}", f"--query-gpu={q}",
                                       "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=5).stdout
                 a = [v.strip() for v in out.strip().split(",")]
                 self.max_mhz = float(a[1])
-                self.samples.append((time.perf_counter(), float(a[0]), int(a[2], 16)))
+                try:
+                    watts = float(a[3])
+                except (IndexError, ValueError):
+                    watts = None
+                self.samples.append((time.perf_counter(), float(a[0]), int(a[2], 16), watts))
             except Exception:
                 pass
             self._stop.wait(max(self.period_s, 0.05))
@@ -92,8 +100,9 @@ class ClockSampler:
         for s in inside:
             mask |= s[2]
         reasons = [k for k, b in {**self.BAD, **self.NOTED}.items() if mask & b]
+        watts = [s[3] for s in inside if s[3] is not None]
         return {"sm_mhz": statistics.median(s[1] for s in inside), "sm_max_mhz": self.max_mhz, "reasons": reasons,
-                "samples": len(inside), "window": window}
+                "samples": len(inside), "window": window, "power_w": statistics.median(watts) if watts else None}
 
 
 def aggregate(ms_local: float, units_local: float, world_size: int) -> Dict[str, float]:
