@@ -104,6 +104,19 @@ __device__ __forceinline__ float warp_sum(float v) {
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
   return v;
 }
+// The same over aligned groups of LPR lanes (LPR a power of two): every lane of a group gets its group's result.
+template <int LPR>
+__device__ __forceinline__ float group_max(float v) {
+#pragma unroll
+  for (int o = LPR / 2; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+template <int LPR>
+__device__ __forceinline__ float group_sum(float v) {
+#pragma unroll
+  for (int o = LPR / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
 // exp(a - b) for a <= b, through the hardware's 2^x: the difference is rounded once, the product with log2(e) once
 __device__ __forceinline__ float exp_diff(float a, float b) { return exp2f((a - b) * 1.4426950408889634f); }
 __device__ __forceinline__ float max4(const float4& v) { return fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w)); }
@@ -309,13 +322,17 @@ __global__ void __launch_bounds__(32 * (G * ROWS + 1), 1) softmax_block_kernel(c
 // ------------------------------------------------------------------ a warp per row: short rows (single pass), and the two phases
 // A lane owns 16-byte units lane, lane + 32, ... (KW of them) of a row or row segment; a warp works on ROWS rows at a time
 // (their loads and reductions interleave), rows warp, warp + W, ... of the tile (W consumer warps).
-template <int MODE, int KW, int ROWS, int W>
+template <int MODE, int KW, int ROWS, int W, int LPR>
 __global__ void __launch_bounds__(32 * (W + 1), 1) softmax_rows_kernel(const __grid_constant__ CUtensorMap tm_in, const __grid_constant__ CUtensorMap tm_out,
                                                                      const SoftmaxArgs args) {
   extern __shared__ uint8_t smem_raw[];
   const SmLayout l = sm_layout(smem_raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int N = args.N, Tn = args.sched.Tn;
+  // LPR lanes work on a row (32 / LPR rows per warp at a time): very short rows would leave most lanes of a warp idle
+  static_assert(LPR == 32 || MODE == kSmSinglePass, "the two-phase kernels put a whole warp on a row segment");
+  constexpr int RPW = 32 / LPR;
+  const int sl = lane & (LPR - 1), q = lane / LPR;
   sm_init(l, W);
   if (warp == W) { sm_produce<MODE>(args, l, &tm_in, &tm_out); return; }
   // 16-byte unit i of row r of a buffer: rows of N elements back to back (single pass), or two boxes of 32 rows x 1 KiB
@@ -335,13 +352,13 @@ __global__ void __launch_bounds__(32 * (W + 1), 1) softmax_rows_kernel(const __g
     const uint32_t buf = l.base + stage * kSmStageBytes;
     const int nvec = ncols >> 2;
     const int tn = col0 / kSmTileN;
-    for (int rb = warp; rb < nrows; rb += W * ROWS) {
+    for (int rb = warp * RPW; rb < nrows; rb += W * RPW * ROWS) {
       float4 v[ROWS][KW];
       float m[ROWS];
       float2 part[ROWS];                       // phase 2: this lane's share of the row's partials, folded as they come
 #pragma unroll
       for (int j = 0; j < ROWS; ++j) {
-        const int r = rb + j * W;
+        const int r = rb + j * (W * RPW) + q;
         m[j] = -INFINITY;
         part[j] = make_float2(-INFINITY, 0.f);
         if (r < nrows) {
@@ -358,7 +375,7 @@ __global__ void __launch_bounds__(32 * (W + 1), 1) softmax_rows_kernel(const __g
           }
 #pragma unroll
           for (int k = 0; k < KW; ++k) {
-            const int i = lane + 32 * k;
+            const int i = sl + LPR * k;
             if (i < nvec) {
               v[j][k] = sm_lds128(unit_addr(buf, r, i));
               m[j] = fmaxf(m[j], max4(v[j][k]));
@@ -374,19 +391,19 @@ __global__ void __launch_bounds__(32 * (W + 1), 1) softmax_rows_kernel(const __g
           // a lane without a chunk holds (-inf, 0): its exponential is 0 and so is its share of the sum
           inv[j] = 1.f / warp_sum(part[j].x == -INFINITY ? 0.f : part[j].y * exp_diff(part[j].x, big[j]));
         } else {
-          big[j] = warp_max(m[j]);
+          big[j] = group_max<LPR>(m[j]);
           inv[j] = 0.f;
         }
       }
 #pragma unroll
       for (int j = 0; j < ROWS; ++j) {
-        const int r = rb + j * W;
-        if (r >= nrows) continue;
+        const int r = rb + j * (W * RPW) + q;
+        const bool live = r < nrows;          // with LPR < 32 the lanes of a warp hold different rows: no lane may skip a shuffle
         if (MODE == kSmPhase2) {
 #pragma unroll
           for (int k = 0; k < KW; ++k) {
-            const int i = lane + 32 * k;
-            if (i < nvec) {
+            const int i = sl + LPR * k;
+            if (live && i < nvec) {
               float4 o = v[j][k];
               exp4_sum(o, big[j]);
               o.x *= inv[j]; o.y *= inv[j]; o.z *= inv[j]; o.w *= inv[j];
@@ -397,15 +414,16 @@ __global__ void __launch_bounds__(32 * (W + 1), 1) softmax_rows_kernel(const __g
           float sum = 0.f;
 #pragma unroll
           for (int k = 0; k < KW; ++k)
-            if (lane + 32 * k < nvec) sum += exp4_sum(v[j][k], big[j]);
-          sum = warp_sum(sum);
+            if (live && sl + LPR * k < nvec) sum += exp4_sum(v[j][k], big[j]);
+          sum = group_sum<LPR>(sum);
+          if (!live) continue;
           if (MODE == kSmPhase1) {
             if (lane == 0) args.partial[(size_t)(row0 + r) * Tn + tn] = make_float2(big[j], sum);
           } else {
             const float sc = 1.f / sum;
 #pragma unroll
             for (int k = 0; k < KW; ++k) {
-              const int i = lane + 32 * k;
+              const int i = sl + LPR * k;
               if (i < nvec) {
                 float4 o = v[j][k];
                 o.x *= sc; o.y *= sc; o.z *= sc; o.w *= sc;
@@ -465,10 +483,10 @@ static int launch_block_for(int units, const CUtensorMap& tm, const SoftmaxArgs&
     return launch_block_for<G, ROWS, LO + 1, HI>(units, tm, args, tiles, stream);
   }
 }
-template <int MODE, int KW, int ROWS, int W = kSmWarps>
+template <int MODE, int KW, int ROWS, int W = kSmWarps, int LPR = 32>
 static int launch_rows(const CUtensorMap& tm, const CUtensorMap& tm_out, const SoftmaxArgs& args, int64_t tiles, cudaStream_t stream) {
   static uint64_t configured = 0;
-  return launch_one(softmax_rows_kernel<MODE, KW, ROWS, W>, configured, tm, tm_out, args, tiles, stream, 32 * (W + 1));
+  return launch_one(softmax_rows_kernel<MODE, KW, ROWS, W, LPR>, configured, tm, tm_out, args, tiles, stream, 32 * (W + 1));
 }
 
 // Single pass: rows of one block; 0 when a row does not fit a buffer.  A block is kept to 48 KiB where the row length
@@ -508,6 +526,8 @@ int launch_softmax(const void* in, void* out, int64_t M, int64_t N, int mode, co
     if (N <= kSmWarpRowLimit) {
       // 16-byte units per lane and row (N / 128, rounded up to what is instantiated), and how many rows a warp works on
       // together: two where a block has at least sixteen rows (N <= 768), else its one row
+      if (N <= 64) return launch_rows<kSmSinglePass, 2, 2, kSmWarps, 8>(tm, tm_out, args, T, stream);
+      if (N <= 128) return launch_rows<kSmSinglePass, 2, 2, kSmWarps, 16>(tm, tm_out, args, T, stream);
       if (N <= 256) return launch_rows<kSmSinglePass, 2, 2>(tm, tm_out, args, T, stream);
       if (N <= 512) return launch_rows<kSmSinglePass, 4, 2>(tm, tm_out, args, T, stream);
       if (N <= 768) return launch_rows<kSmSinglePass, 6, 2>(tm, tm_out, args, T, stream);

@@ -36,7 +36,8 @@ def close(got, ref):
 
 # sizes span several 32 x 512 tiles with ragged edges both ways, one tile, one row, one 16-byte unit per row, rows of
 # 16384 (one row per single-pass block) and 2048 (six)
-@pytest.mark.parametrize("M,N", [(32, 512), (100, 1300), (257, 4100), (1, 4), (3, 16384), (70, 2048), (9, 8), (33, 520)])
+@pytest.mark.parametrize("M,N", [(32, 512), (100, 1300), (257, 4100), (1, 4), (3, 16384), (70, 2048), (9, 8), (33, 520),
+                                 (1003, 64), (77, 128), (50, 32), (333, 96), (201, 20)])   # the last five: 8 or 16 lanes per row, ragged last block
 @pytest.mark.parametrize("mode", MODES)
 def test_matches_the_definition(M, N, mode):
     rng = np.random.default_rng(M * 7 + N)
