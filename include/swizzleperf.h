@@ -302,10 +302,14 @@ int sp_stencil2d(const void* in, void* out, int64_t M, int64_t N, float c_center
  * the exponentials and their sum, with the chunks of a row spread over blocks; the remap the paper finds keeps a row's
  * chunks in one chiplet's L2 between the phases):
  *   mode SP_SOFTMAX_SINGLE_PASS        : blocks of whole rows pass through shared memory once; every byte crosses HBM
- *                                        once per direction.  N <= 16384 (a row must fit a 64 KiB buffer), else
- *                                        SP_ERR_UNSUPPORTED.  `scheme` / `params` order the row blocks, as for
+ *                                        once per direction.  A row of more than 16384 elements (one 64 KiB buffer) is
+ *                                        shared by the ceil(N / 16384) CTAs (2 to 8) of a thread-block cluster, which
+ *                                        exchange their partial maxima and sums through distributed shared memory (faster
+ *                                        than the two-phase form up to about 49152 elements per row, slower beyond: the
+ *                                        more CTAs wait for each other per row, the more their skew costs); N <= 131072,
+ *                                        else SP_ERR_UNSUPPORTED.  `scheme` / `params` order the row blocks, as for
  *                                        sp_tile_map(M, N, rows, N, ...) with, in integer arithmetic, rows =
- *                                        max(1, 12288 / N) for N > 1792 (blocks of at most 48 KiB, several warps on a
+ *                                        max(1, 12288 / N) for N > 1792 (blocks of at most 48 KiB, or one row; several warps on a
  *                                        row) and rows = min(96, max(8, 12288 / N / 8 * 8)) for N <= 1792 (a warp per row).
  *   mode SP_SOFTMAX_TWO_PHASE          : the matrix is cut into SP_SOFTMAX_TILE_M x SP_SOFTMAX_TILE_N tiles, ordered exactly as
  *                                        for sp_tile_map(M, N, 32, 512, ...).  A first launch leaves per tile and row

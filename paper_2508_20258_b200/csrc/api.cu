@@ -740,7 +740,7 @@ int sp_softmax(const void* in, void* out, int64_t M, int64_t N, int32_t mode, in
   if (mode == SP_SOFTMAX_SINGLE_PASS) {
     tile_m = softmax_rows_per_block(N);
     tile_n = N;
-    if (tile_m < 1) { set_error("single-pass softmax needs a row to fit a 64 KiB buffer (N <= 16384); use a two-phase mode"); return SP_ERR_UNSUPPORTED; }
+    if (tile_m < 1) { set_error("single-pass softmax takes rows of up to 131072 elements (eight 64 KiB buffers of a cluster); use a two-phase mode"); return SP_ERR_UNSUPPORTED; }
   }
   Sched sched;
   int rc = resolve_sched(M, N, tile_m, (int32_t)tile_n, scheme, params, &sched);

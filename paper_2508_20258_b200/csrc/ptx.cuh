@@ -22,6 +22,12 @@ __device__ __forceinline__ uint32_t cluster_ctarank() {
   return r;
 }
 
+__device__ __forceinline__ uint32_t cluster_nctarank() {   // CTAs per cluster; 1 for a launch without clusters
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+  return r;
+}
+
 // True in exactly one lane of a fully converged warp.
 __device__ __forceinline__ bool elect_one() {
   uint32_t pred;

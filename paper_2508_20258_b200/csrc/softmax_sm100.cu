@@ -15,7 +15,9 @@
 //                      values are all taken there, the results written back to the same buffer and sent out from it by
 //                      one bulk copy.  Every byte crosses HBM once in each direction; the order of the row blocks has
 //                      nothing left to improve.  Rows of up to 1792 elements are handled a warp per row (no meeting of
-//                      warps at all), longer ones by two to twelve warps per row (two meetings per block).
+//                      warps at all), longer ones by two to twelve warps per row (two meetings per block), rows of more
+//                      than 16384 elements by the two to eight CTAs of a thread-block cluster, which exchange their partial
+//                      results through distributed shared memory.
 //
 // All kernels: persistent CTAs (one per SM), one producer warp that brings tiles into a ring of three 64 KiB buffers (a
 // block of whole rows is contiguous in memory: one bulk copy; a 32 x 512 tile: two TMA boxes of 32 rows x 1 KiB;
@@ -43,7 +45,7 @@ constexpr int kSmThreads = 32 * (kSmWarps + 1);
 constexpr int kSmBlockWarpsMax = 16;
 constexpr int kSmMaxRows = 8;                            // single pass, long rows: room for the partials of a block (it has at most six rows)
 constexpr int kSmWarpRowLimit = 1792;                    // single pass: rows up to this length are handled a warp per row
-constexpr uint32_t kSmSmem = kSmStages * kSmStageBytes + 1024 /* alignment */ + 64 /* barriers */ + (2 * kSmMaxRows * kSmBlockWarpsMax + 4) * 4;
+constexpr uint32_t kSmSmem = kSmStages * kSmStageBytes + 1024 /* alignment */ + 64 /* barriers */ + (2 * kSmMaxRows * kSmBlockWarpsMax + 4) * 4 + 4 * 8 + 4 * 8 * 8;
 static_assert(kSmTileM * kSmTileN * 4 == kSmStageBytes, "a two-phase tile fills one buffer");
 constexpr int kSmPhaseWarps = 16;                       // two-phase kernels: consumer warps
 static_assert(kSmTileM % kSmPhaseWarps == 0, "the rows of a two-phase tile are shared out evenly");
@@ -57,11 +59,12 @@ struct SoftmaxArgs {
   int M, N;
   int rows_per_block;    // single pass: rows of one block (1..96); a block's rows are contiguous in memory
   int reverse;           // phase 2: slot s works on the tile of slot T - 1 - s
+  int chunk;             // rows spread over a cluster: elements of a row per CTA (a multiple of 4)
   Sched sched;
 };
 
 enum : int { kRoleSoftmaxLoad = 7, kRoleSoftmaxCompute = 8 };
-enum : int { kSmSinglePass = 0, kSmPhase1 = 1, kSmPhase2 = 2 };
+enum : int { kSmSinglePass = 0, kSmPhase1 = 1, kSmPhase2 = 2, kSmCluster = 3 };
 
 __device__ __forceinline__ float4 sm_lds128(uint32_t addr) {
   float4 v;
@@ -127,6 +130,7 @@ __device__ __forceinline__ float exp4_sum(float4& v, float big) {   // v <- exp(
 
 struct SmLayout {
   uint32_t base, bar_full, bar_empty, red, fail_flag;
+  uint32_t xbar, xval;   // rows spread over a cluster: four exchange barriers, [4][8] pairs of floats (see softmax_cluster_kernel)
 };
 __device__ __forceinline__ SmLayout sm_layout(const uint8_t* smem_raw) {
   SmLayout l;
@@ -135,6 +139,8 @@ __device__ __forceinline__ SmLayout sm_layout(const uint8_t* smem_raw) {
   l.bar_empty = l.bar_full + 8 * kSmStages;
   l.red = l.bar_empty + 8 * kSmStages + 16;              // [2][kSmMaxRows][consumer warps] floats (long rows, single pass)
   l.fail_flag = l.red + 2 * kSmMaxRows * kSmBlockWarpsMax * 4;
+  l.xbar = l.fail_flag + 8;
+  l.xval = l.xbar + 4 * 8;
   return l;
 }
 
@@ -143,6 +149,8 @@ template <int MODE>
 __device__ __forceinline__ void sm_geometry(const SoftmaxArgs& a, int t, int& row0, int& nrows, int& col0, int& ncols) {
   if (MODE == kSmSinglePass) {
     row0 = t * a.rows_per_block; nrows = min(a.rows_per_block, a.M - row0); col0 = 0; ncols = a.N;
+  } else if (MODE == kSmCluster) {       // one row per slot; this CTA's share of it
+    row0 = t; nrows = 1; col0 = (int)cluster_ctarank() * a.chunk; ncols = max(0, min(a.chunk, a.N - col0));
   } else {
     const int Tn = a.sched.Tn, tm = t / Tn, tn = t - tm * Tn;
     row0 = tm * kSmTileM; nrows = min(kSmTileM, a.M - row0); col0 = tn * kSmTileN; ncols = min(kSmTileN, a.N - col0);
@@ -186,8 +194,8 @@ __device__ __forceinline__ void sm_produce(const SoftmaxArgs& args, const SmLayo
     sm_geometry<MODE>(args, sm_tile_of<MODE>(args, s_prev), row0, nrows, col0, ncols);
     if (lane == 0) {
       const uint32_t src = l.base + st * kSmStageBytes;
-      if (MODE == kSmSinglePass) {
-        bulk_store(args.out + (size_t)row0 * args.N, src, (uint32_t)nrows * (uint32_t)ncols * 4u);
+      if (MODE == kSmSinglePass || MODE == kSmCluster) {
+        if (ncols > 0) bulk_store(args.out + (size_t)row0 * args.N + col0, src, (uint32_t)nrows * (uint32_t)ncols * 4u);
       } else {
         tma_store_2d(tm_out, src, col0, row0);
         if (ncols > kSmBoxCols) tma_store_2d(tm_out, src + kSmBoxBytes, col0 + kSmBoxCols, row0);
@@ -197,20 +205,23 @@ __device__ __forceinline__ void sm_produce(const SoftmaxArgs& args, const SmLayo
     }
     __syncwarp();
   };
+  // slots of this CTA: its own index and stride, or its cluster's when a row is spread over a cluster
+  const int first = MODE == kSmCluster ? (int)(blockIdx.x / cluster_nctarank()) : (int)blockIdx.x;
+  const int step = MODE == kSmCluster ? (int)(gridDim.x / cluster_nctarank()) : (int)gridDim.x;
   int n_loaded = 0;
-  for (int s = blockIdx.x; s < args.sched.T && ok; s += gridDim.x, ++n_loaded) {
+  for (int s = first; s < args.sched.T && ok; s += step, ++n_loaded) {
     ok = mbar_wait(l.bar_empty + 8 * stage, phase ^ 1u, args.status, (kRoleSoftmaxLoad << 8) | 1);
     ok = __all_sync(0xffffffffu, ok);
     if (!ok) break;
-    if (STORE && n_loaded >= kSmStages) store_block(s - kSmStages * (int)gridDim.x, stage);
+    if (STORE && n_loaded >= kSmStages) store_block(s - kSmStages * step, stage);
     int row0, nrows, col0, ncols;
     sm_geometry<MODE>(args, sm_tile_of<MODE>(args, s), row0, nrows, col0, ncols);
     const uint32_t full = l.bar_full + 8 * stage, dst = l.base + stage * kSmStageBytes;
     if (elect_one()) {
-      if (MODE == kSmSinglePass) {
+      if (MODE == kSmSinglePass || MODE == kSmCluster) {
         const uint32_t bytes = (uint32_t)nrows * (uint32_t)ncols * 4u;
-        mbar_arrive_expect_tx(full, bytes);
-        bulk_load(dst, args.in + (size_t)row0 * args.N, bytes, full);
+        mbar_arrive_expect_tx(full, bytes);         // (a share of no columns: the phase completes by the arrival alone)
+        if (bytes) bulk_load(dst, args.in + (size_t)row0 * args.N + col0, bytes, full);
       } else {
         const int boxes = ncols > kSmBoxCols ? 2 : 1;
         mbar_arrive_expect_tx(full, boxes * kSmBoxBytes);
@@ -226,7 +237,7 @@ __device__ __forceinline__ void sm_produce(const SoftmaxArgs& args, const SmLayo
     ok = __all_sync(0xffffffffu, ok);
     // the last blocks: block n_loaded - kSmStages + i went through this stage, if there was one
     const int j = n_loaded - kSmStages + i;
-    if (STORE && ok && j >= 0) store_block((int)blockIdx.x + j * (int)gridDim.x, stage);
+    if (STORE && ok && j >= 0) store_block(first + j * step, stage);
     if (++stage == kSmStages) { stage = 0; phase ^= 1u; }
   }
   if (STORE && lane == 0) bulk_wait_all();      // ... nor away from it
@@ -317,6 +328,156 @@ __global__ void __launch_bounds__(32 * (G * ROWS + 1), 1) softmax_block_kernel(c
     if (lane == 0) mbar_arrive_release(l.bar_empty + 8 * stage);
     if (++stage == kSmStages) { stage = 0; phase ^= 1u; }
   }
+}
+
+// ------------------------------------------------------------------ single pass, rows longer than a buffer: a cluster per row
+// A row of up to CS x 16384 elements is spread over the CS CTAs of a thread-block cluster: CTA k brings elements
+// [k * chunk, (k + 1) * chunk) of the row into its own ring.  One sweep and one exchange per row:
+//   sweep    -- a thread reads its units of the share (G warps, UK units per lane), takes their maximum m_t, writes
+//               exp(x - m_t) back in place and keeps (m_t, s_t = sum of those); pairs combine as (m, s) + (m', s') =
+//               (M = max(m, m'), s exp(m - M) + s' exp(m' - M)): by shuffles within a warp, through shared memory across
+//               the warps (one meeting of the consumer warps per row), and
+//   exchange -- across the CTAs through distributed shared memory: one thread writes its CTA's pair into slot k of every
+//               CTA of the cluster and arrives, with release at cluster scope, on that CTA's exchange barrier;
+//   scaling  -- a thread waits on its own CTA's barrier (bounded, acquire at cluster scope), combines the CS pairs into
+//               (M, S), and multiplies its units by exp(m_t - M) / S; the buffer then goes to the producer warp, which
+//               sends it out.
+// The scaling of a row is done after the sweep of the next one, so the exchange has a sweep's time to complete.  A long
+// row crosses HBM once in each direction, where the two-phase form reads it twice.
+// Exchange slots and barriers go round four sets: a CTA can publish row j + 3 while a peer still reads the pairs of row j
+// (it needs nothing from that peer until it scales row j + 2), but row j + 4 only after the peer has published row
+// j + 2, which the peer does after it has scaled row j.  No hardware cluster barrier inside the loop: every wait is
+// bounded, so a CTA whose wait gave up leaves the loop, its peers' waits run out in turn, and all of them meet at the
+// cluster barrier before the exit (shared memory of a CTA that has exited must not be written).
+__device__ __forceinline__ void pair_combine(float& m, float& s, float m2, float s2) {
+  const float M = fmaxf(m, m2);
+  // a pair (-inf, 0) stands for "nothing": its share of the sum is 0, not exp(-inf + inf)
+  s = (m == -INFINITY ? 0.f : s * exp_diff(m, M)) + (m2 == -INFINITY ? 0.f : s2 * exp_diff(m2, M));
+  m = M;
+}
+template <int UK, int G, int CS>
+__global__ void __launch_bounds__(32 * (G + 1), 1) softmax_cluster_kernel(const __grid_constant__ CUtensorMap tm_in, const __grid_constant__ CUtensorMap tm_out,
+                                                                          const SoftmaxArgs args) {
+  constexpr int W = G;
+  extern __shared__ uint8_t smem_raw[];
+  const SmLayout l = sm_layout(smem_raw);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t rank = cluster_ctarank();
+  sm_init(l, W);
+  if (tid == 0) {
+    for (int i = 0; i < 4; ++i) mbar_init(l.xbar + 8 * i, CS);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // every CTA's barriers exist before any peer arrives on them
+  asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+
+  if (warp == W) {
+    sm_produce<kSmCluster>(args, l, &tm_in, &tm_out);
+  } else {
+    const int first = (int)(blockIdx.x / CS), step = (int)(gridDim.x / CS);
+    const int T = args.sched.T;
+    int stage = 0;
+    uint32_t phase = 0;
+    // the row swept in the previous iteration, waiting to be scaled
+    bool pending = false;
+    int p_stage = 0, p_nvec = 0, p_it = 0;
+    float p_mt = 0.f;
+    int it = 0;
+    for (int s = first;; s += step, ++it) {
+      const bool have = s < T;
+      if (!have && !pending) break;
+      int c_nvec = 0;
+      float mt = -INFINITY;
+      if (have) {
+        bool ok = mbar_wait(l.bar_full + 8 * stage, phase, args.status, (kRoleSoftmaxCompute << 8) | 1);
+        ok = __all_sync(0xffffffffu, ok);
+        // The warps meet below, so none may leave on its own: a warp whose wait gave up raises a flag, goes through the
+        // meeting empty-handed, and all of them leave together right after it.
+        if (!ok && lane == 0) sm_sts32(l.fail_flag, 1.f);
+        int row0, nrows, col0, ncols;
+        sm_geometry<kSmCluster>(args, sm_tile_of<kSmCluster>(args, s), row0, nrows, col0, ncols);
+        c_nvec = ok ? ncols >> 2 : 0;
+        const uint32_t base = l.base + stage * kSmStageBytes;
+        float4 v[UK];
+#pragma unroll
+        for (int k = 0; k < UK; ++k) {
+          const int i = warp * 32 + lane + 32 * G * k;
+          if (i < c_nvec) {
+            v[k] = sm_lds128(base + (uint32_t)i * 16u);
+            mt = fmaxf(mt, max4(v[k]));
+          }
+        }
+        float st = 0.f;
+#pragma unroll
+        for (int k = 0; k < UK; ++k) {
+          const int i = warp * 32 + lane + 32 * G * k;
+          if (i < c_nvec) {
+            st += exp4_sum(v[k], mt);
+            sm_sts128(base + (uint32_t)i * 16u, v[k]);      // exp(x - m_t) replaces x; scaled once (M, S) of the row are known
+          }
+        }
+        float m = mt;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const float m2 = __shfl_xor_sync(0xffffffffu, m, o), s2 = __shfl_xor_sync(0xffffffffu, st, o);
+          pair_combine(m, st, m2, s2);
+        }
+        const uint32_t red = l.red + (uint32_t)((it & 1) * 2 * kSmBlockWarpsMax) * 4u;     // pairs of the warps, two sets
+        if (lane == 0) { sm_sts32(red + (uint32_t)(2 * warp) * 4u, m); sm_sts32(red + (uint32_t)(2 * warp + 1) * 4u, st); }
+        consumer_sync<W>();
+        if (sm_lds32(l.fail_flag) != 0.f) break;
+        if (tid == 0) {
+          float cm = -INFINITY, cs = 0.f;
+#pragma unroll
+          for (int g = 0; g < G; ++g) pair_combine(cm, cs, sm_lds32(red + (uint32_t)(2 * g) * 4u), sm_lds32(red + (uint32_t)(2 * g + 1) * 4u));
+          const uint32_t q = (uint32_t)it & 3u;
+          const uint32_t slot = l.xval + (q * 8u + rank) * 8u, bar = l.xbar + q * 8u;
+#pragma unroll
+          for (uint32_t c = 0; c < (uint32_t)CS; ++c) {
+            asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(mapa(slot, c)), "f"(cm), "f"(cs) : "memory");
+            mbar_arrive_cluster(mapa(bar, c));
+          }
+        }
+      }
+      if (pending) {
+        const uint32_t q = (uint32_t)p_it & 3u, xphase = (uint32_t)(p_it >> 2) & 1u;
+        bool okx = mbar_wait_cluster_acquire(l.xbar + q * 8u, xphase, args.status, (kRoleSoftmaxCompute << 8) | 2);
+        okx = __all_sync(0xffffffffu, okx);
+        // (a warp whose wait gave up must not leave on its own either, or the others would wait for it at the next
+        // row's meeting: it raises the flag and goes there with them; the status word is set by then, so that row's
+        // wait for data returns at once)
+        if (!okx && lane == 0) sm_sts32(l.fail_flag, 1.f);
+        if (okx) {
+          float M = -INFINITY, S = 0.f;
+#pragma unroll
+          for (int c = 0; c < CS; ++c)
+            pair_combine(M, S, sm_lds32(l.xval + (q * 8u + (uint32_t)c) * 8u), sm_lds32(l.xval + (q * 8u + (uint32_t)c) * 8u + 4u));
+          const float f = p_mt == -INFINITY ? 0.f : exp_diff(p_mt, M) / S;
+          const uint32_t base = l.base + p_stage * kSmStageBytes;
+#pragma unroll
+          for (int k = 0; k < UK; ++k) {
+            const int i = warp * 32 + lane + 32 * G * k;
+            if (i < p_nvec) {
+              float4 o = sm_lds128(base + (uint32_t)i * 16u);
+              o.x *= f; o.y *= f; o.z *= f; o.w *= f;
+              sm_sts128(base + (uint32_t)i * 16u, o);
+            }
+          }
+          // the results are in the buffer: make them visible to the copy engine, then hand the buffer to the producer warp
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_release(l.bar_empty + 8 * p_stage);
+        }
+      }
+      pending = have;
+      p_stage = stage; p_nvec = c_nvec; p_it = it; p_mt = mt;
+      if (have && ++stage == kSmStages) { stage = 0; phase ^= 1u; }
+    }
+  }
+  // no CTA leaves while a peer may still write to its shared memory or arrive on its barriers
+  asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
 }
 
 // ------------------------------------------------------------------ a warp per row: short rows (single pass), and the two phases
@@ -483,6 +644,62 @@ static int launch_block_for(int units, const CUtensorMap& tm, const SoftmaxArgs&
     return launch_block_for<G, ROWS, LO + 1, HI>(units, tm, args, tiles, stream);
   }
 }
+// A row per cluster of CS CTAs: as many clusters as can be resident at once (asked of the occupancy calculator), at most
+// one per row.
+template <int UK, int G, int CS>
+static int launch_cluster(const CUtensorMap& tm, const SoftmaxArgs& args, int64_t rows, cudaStream_t stream) {
+  static uint64_t configured = 0;
+  static int clusters[64] = {};
+  auto kern = softmax_cluster_kernel<UK, G, CS>;
+  cudaError_t e;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { set_error("cannot query the device"); return SP_ERR_CUDA; }
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof cfg);
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = CS; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.blockDim = dim3(32 * (G + 1), 1, 1);
+  cfg.dynamicSmemBytes = kSmSmem;
+  cfg.stream = stream;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  if (first_use_on_this_device(configured)) {
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmSmem);
+    if (e != cudaSuccess) { configured = 0; set_error("cudaFuncSetAttribute failed: %s", cudaGetErrorString(e)); return SP_ERR_CUDA; }
+    int sms = 0, n = 0;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    cfg.gridDim = dim3((unsigned)(sms / CS * CS), 1, 1);
+    e = cudaOccupancyMaxActiveClusters(&n, kern, &cfg);
+    if (e != cudaSuccess || n < 1) {
+      configured = 0; cudaGetLastError();
+      set_error("no cluster of %d CTAs can be resident with this kernel (%s)", CS, e == cudaSuccess ? "0 active clusters" : cudaGetErrorString(e));
+      return SP_ERR_UNSUPPORTED;
+    }
+    clusters[dev & 63] = n;
+  }
+  const int64_t n_clusters = rows < clusters[dev & 63] ? rows : clusters[dev & 63];
+  cfg.gridDim = dim3((unsigned)(n_clusters * CS), 1, 1);
+  e = cudaLaunchKernelEx(&cfg, kern, tm, tm, args);
+  if (e != cudaSuccess) { set_error("softmax cluster launch failed: %s", cudaGetErrorString(e)); return SP_ERR_CUDA; }
+  return SP_OK;
+}
+template <int G, int CS, int LO, int HI>
+static int launch_cluster_for(int units, const CUtensorMap& tm, const SoftmaxArgs& args, int64_t rows, cudaStream_t stream) {
+  if constexpr (LO > HI) {
+    set_error("softmax: no cluster kernel for %d units per share with %d warps", units, G);
+    return SP_ERR_UNSUPPORTED;
+  } else {
+    if ((units + 32 * G - 1) / (32 * G) <= LO) return launch_cluster<LO, G, CS>(tm, args, rows, stream);
+    return launch_cluster_for<G, CS, LO + 1, HI>(units, tm, args, rows, stream);
+  }
+}
+template <int CS>
+static int launch_cluster_share(int units, const CUtensorMap& tm, const SoftmaxArgs& args, int64_t rows, cudaStream_t stream) {
+  // a share of 8196 to 16384 elements: the same choice of warps as for a whole row of that length
+  return units > 3072 ? launch_cluster_for<8, CS, 13, 16>(units, tm, args, rows, stream)
+                      : launch_cluster_for<12, CS, 6, 8>(units, tm, args, rows, stream);
+}
+
 template <int MODE, int KW, int ROWS, int W = kSmWarps, int LPR = 32>
 static int launch_rows(const CUtensorMap& tm, const CUtensorMap& tm_out, const SoftmaxArgs& args, int64_t tiles, cudaStream_t stream) {
   static uint64_t configured = 0;
@@ -494,7 +711,7 @@ static int launch_rows(const CUtensorMap& tm, const CUtensorMap& tm_out, const S
 // (rows of 4096: 5.75 TB/s with blocks of four rows, 6.47 with three; four buffers of 48 KiB are no better than three).
 // Long rows: floor(12288 / N) rows, at least one.  Short rows (a warp per row): a multiple of the eight consumer warps, 8 to 96.
 int softmax_rows_per_block(int64_t N) {
-  if (N * 4 > (int64_t)kSmStageBytes) return 0;
+  if (N * 4 > (int64_t)kSmStageBytes) return N <= 8 * (int64_t)(kSmStageBytes / 4) ? 1 : 0;   // a cluster of up to eight CTAs per row
   const int64_t r = 12288 / N;
   if (N > kSmWarpRowLimit) return r < 1 ? 1 : (int)r;
   const int64_t r8 = r / kSmWarps * kSmWarps;
@@ -512,6 +729,7 @@ int launch_softmax(const void* in, void* out, int64_t M, int64_t N, int mode, co
   args.M = (int)M; args.N = (int)N;
   args.rows_per_block = mode == SP_SOFTMAX_SINGLE_PASS ? softmax_rows_per_block(N) : 0;
   args.reverse = mode == SP_SOFTMAX_TWO_PHASE_REVERSED ? 1 : 0;
+  args.chunk = 0;
   args.sched = sched;
   const int64_t T = sched.T;
   CUtensorMap tm, tm_out;      // used by the two-phase kernels only; the single-pass kernels take them and ignore them
@@ -521,6 +739,23 @@ int launch_softmax(const void* in, void* out, int64_t M, int64_t N, int mode, co
     int rc = make_map_plain(&tm, in, M, N, kSmTileM, kSmBoxCols);
     if (rc == SP_OK) rc = make_map_plain(&tm_out, out, M, N, kSmTileM, kSmBoxCols);
     if (rc != SP_OK) return rc;
+  }
+  if (mode == SP_SOFTMAX_SINGLE_PASS && N * 4 > (int64_t)kSmStageBytes) {
+    // the row does not fit one CTA's buffer: the fewest CTAs whose buffers hold it share it as a cluster (2 to 8; a cluster
+    // need not be a power of two), in equal shares of a multiple of 4 elements: the larger the shares, the fewer exchanges
+    // per byte, and the more SMs the clusters cover (3 x 49, 5 x 29, 7 x 21 of 148)
+    const int cs = (int)((N + 16383) / 16384);
+    args.chunk = (int)(((N + cs - 1) / cs + 3) / 4 * 4);
+    const int units = args.chunk / 4;
+    switch (cs) {
+      case 2: return launch_cluster_share<2>(units, tm, args, M, stream);
+      case 3: return launch_cluster_share<3>(units, tm, args, M, stream);
+      case 4: return launch_cluster_share<4>(units, tm, args, M, stream);
+      case 5: return launch_cluster_share<5>(units, tm, args, M, stream);
+      case 6: return launch_cluster_share<6>(units, tm, args, M, stream);
+      case 7: return launch_cluster_share<7>(units, tm, args, M, stream);
+      default: return launch_cluster_share<8>(units, tm, args, M, stream);
+    }
   }
   if (mode == SP_SOFTMAX_SINGLE_PASS) {
     if (N <= kSmWarpRowLimit) {

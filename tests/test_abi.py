@@ -95,6 +95,6 @@ def test_softmax_rejects_bad_arguments_before_touching_a_device():
     assert L.sp_softmax(a, a, 64, 128, 1, sp.ROW_MAJOR, None, None) == sp.ERR_INVALID_ARG
     assert L.sp_softmax(a, b, 64, 128, 7, sp.ROW_MAJOR, None, None) == sp.ERR_INVALID_ARG
     assert L.sp_softmax(a, b, 0, 128, 0, sp.ROW_MAJOR, None, None) == sp.ERR_INVALID_ARG
-    assert L.sp_softmax(a, b, 64, 16388, 0, sp.ROW_MAJOR, None, None) == sp.ERR_UNSUPPORTED     # a row must fit a buffer
+    assert L.sp_softmax(a, b, 64, 131076, 0, sp.ROW_MAJOR, None, None) == sp.ERR_UNSUPPORTED    # a row must fit the eight buffers of a cluster
     bad = sp.make_params(num_xcds=4, xcd_balanced=0)      # 5 x 2 tiles of 32 x 512: the printed formula leaves [0, 10)
     assert L.sp_softmax(a, b, 160, 1024, 1, sp.XCD, ctypes.byref(bad), None) == sp.ERR_NOT_BIJECTIVE

@@ -97,7 +97,7 @@ def test_rejections_launch_nothing():
     assert L.sp_softmax(x.data_ptr(), out.data_ptr(), 8, 16, 3, sp.ROW_MAJOR, ctypes.byref(p), None) == sp.ERR_INVALID_ARG
     assert L.sp_softmax(x.data_ptr(), out.data_ptr(), 8, 18, 0, sp.ROW_MAJOR, ctypes.byref(p), None) == sp.ERR_ALIGNMENT
     assert L.sp_softmax(x.data_ptr() + 4, out.data_ptr(), 8, 12, 0, sp.ROW_MAJOR, ctypes.byref(p), None) == sp.ERR_ALIGNMENT
-    assert L.sp_softmax(x.data_ptr(), out.data_ptr(), 1, 16388, 0, sp.ROW_MAJOR, ctypes.byref(p), None) == sp.ERR_UNSUPPORTED
+    assert L.sp_softmax(x.data_ptr(), out.data_ptr(), 1, 131076, 0, sp.ROW_MAJOR, ctypes.byref(p), None) == sp.ERR_UNSUPPORTED
     assert L.sp_softmax(None, out.data_ptr(), 8, 16, 0, sp.ROW_MAJOR, ctypes.byref(p), None) == sp.ERR_INVALID_ARG
     torch.cuda.synchronize()
     assert bool((out == 7.0).all())
@@ -110,6 +110,29 @@ def test_rows_longer_than_a_buffer_take_the_two_phase_form():
     ref = SM.softmax(x)
     for mode in MODES[1:]:
         assert close(run(x, mode, sp.GROUP_N, group=7), ref)
+
+
+# rows spread over a cluster of 2, 4 or 8 CTAs: the shortest and longest row of each cluster size, shares with a ragged last
+# CTA, more rows than resident clusters, fewer rows than that, one row
+@pytest.mark.parametrize("M,N", [(5, 16388), (300, 32768), (7, 32772), (3, 50000), (200, 65536), (2, 65540), (9, 100000),
+                                 (150, 131072), (1, 131072), (40, 16400), (11, 98308)])
+def test_single_pass_with_a_cluster_per_row(M, N):
+    rng = np.random.default_rng(M * 13 + N)
+    x = (rng.standard_normal((M, N)) * 3.0).astype(np.float32)
+    x[M // 2, (2 * N) // 3] += 35.0                     # a dominant entry in one CTA's share: every share needs its maximum
+    ref = SM.softmax(x)
+    for scheme, kw in [(sp.ROW_MAJOR, {}), (sp.GROUP_M, dict(group=3)), (sp.HILBERT, {})]:
+        got = run(x, sp.SOFTMAX_SINGLE_PASS, scheme, **kw)
+        assert close(got, ref), (M, N, scheme)
+        assert np.abs(got.astype(np.float64).sum(axis=1) - 1.0).max() <= 1e-5
+
+
+def test_single_pass_refuses_rows_beyond_eight_buffers():
+    x = torch.zeros((2, 131076), dtype=torch.float32, device="cuda")
+    out = torch.empty_like(x)
+    with pytest.raises(sp.SpError) as e:
+        sp.softmax(x, out, sp.SOFTMAX_SINGLE_PASS, sp.ROW_MAJOR, sp.make_params())
+    assert e.value.status == sp.ERR_UNSUPPORTED
 
 
 def test_single_pass_at_every_row_length_of_the_long_row_kernels():

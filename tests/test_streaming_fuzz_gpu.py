@@ -77,8 +77,6 @@ def test_softmax_random_shapes_modes_and_orders(seed):
         x = (rng.standard_normal((M, N)) * float(rng.uniform(0.5, 6.0))).astype(np.float32)
         x[int(rng.integers(M)), int(rng.integers(N))] += 50.0
         mode = [sp.SOFTMAX_SINGLE_PASS, sp.SOFTMAX_TWO_PHASE, sp.SOFTMAX_TWO_PHASE_REVERSED][rng.integers(3)]
-        if N > 16384 and mode == sp.SOFTMAX_SINGLE_PASS:
-            mode = sp.SOFTMAX_TWO_PHASE                         # a single pass holds a whole row in one 64 KiB buffer
         if mode == sp.SOFTMAX_SINGLE_PASS:                          # blocks of whole rows: a grid of one column
             rows = min(96, max(8, 12288 // N // 8 * 8)) if N <= 1792 else max(1, 12288 // N)   # the header's rule
             grid = (-(-M // rows), 1)
