@@ -303,7 +303,7 @@ int sp_stencil2d(const void* in, void* out, int64_t M, int64_t N, float c_center
  * chunks in one chiplet's L2 between the phases):
  *   mode SP_SOFTMAX_SINGLE_PASS        : blocks of whole rows pass through shared memory once; every byte crosses HBM
  *                                        once per direction.  A row of more than 16384 elements (one 64 KiB buffer) is
- *                                        shared by the ceil(N / 16384) CTAs (2 to 8) of a thread-block cluster, which
+ *                                        shared by the ceil(N / 16384) CTAs (2 to 8; 8 instead of 7) of a thread-block cluster, which
  *                                        exchange their partial maxima and sums through distributed shared memory (faster
  *                                        than the two-phase form up to about 49152 elements per row, slower beyond: the
  *                                        more CTAs wait for each other per row, the more their skew costs); N <= 131072,

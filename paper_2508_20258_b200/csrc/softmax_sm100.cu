@@ -743,8 +743,10 @@ int launch_softmax(const void* in, void* out, int64_t M, int64_t N, int mode, co
   if (mode == SP_SOFTMAX_SINGLE_PASS && N * 4 > (int64_t)kSmStageBytes) {
     // the row does not fit one CTA's buffer: the fewest CTAs whose buffers hold it share it as a cluster (2 to 8; a cluster
     // need not be a power of two), in equal shares of a multiple of 4 elements: the larger the shares, the fewer exchanges
-    // per byte, and the more SMs the clusters cover (3 x 49, 5 x 29, 7 x 21 of 148)
-    const int cs = (int)((N + 16383) / 16384);
+    // per byte (resident on B200: 148 CTAs in clusters of two, 135 of three, 132 of four and six, 130 of five, 120 of eight)
+    // (clusters of seven cover 105 of 148 SMs, of eight 120: seven are never used)
+    int cs = (int)((N + 16383) / 16384);
+    if (cs == 7) cs = 8;
     args.chunk = (int)(((N + cs - 1) / cs + 3) / 4 * 4);
     const int units = args.chunk / 4;
     switch (cs) {
@@ -753,7 +755,6 @@ int launch_softmax(const void* in, void* out, int64_t M, int64_t N, int mode, co
       case 4: return launch_cluster_share<4>(units, tm, args, M, stream);
       case 5: return launch_cluster_share<5>(units, tm, args, M, stream);
       case 6: return launch_cluster_share<6>(units, tm, args, M, stream);
-      case 7: return launch_cluster_share<7>(units, tm, args, M, stream);
       default: return launch_cluster_share<8>(units, tm, args, M, stream);
     }
   }
