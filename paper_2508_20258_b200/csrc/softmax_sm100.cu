@@ -695,9 +695,8 @@ static int launch_cluster_for(int units, const CUtensorMap& tm, const SoftmaxArg
 }
 template <int CS>
 static int launch_cluster_share(int units, const CUtensorMap& tm, const SoftmaxArgs& args, int64_t rows, cudaStream_t stream) {
-  // a share of 8196 to 16384 elements: the same choice of warps as for a whole row of that length
-  return units > 3072 ? launch_cluster_for<8, CS, 13, 16>(units, tm, args, rows, stream)
-                      : launch_cluster_for<12, CS, 6, 8>(units, tm, args, rows, stream);
+  // a share of 8196 to 16384 elements: twelve consumer warps (eight: 3-6 % slower, fifteen: the same)
+  return launch_cluster_for<12, CS, 6, 11>(units, tm, args, rows, stream);
 }
 
 template <int MODE, int KW, int ROWS, int W = kSmWarps, int LPR = 32>
