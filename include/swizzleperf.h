@@ -305,7 +305,7 @@ int sp_stencil2d(const void* in, void* out, int64_t M, int64_t N, float c_center
  *                                        once per direction.  A row of more than 16384 elements (one 64 KiB buffer) is
  *                                        shared by the ceil(N / 16384) CTAs (2 to 8; 8 instead of 7) of a thread-block cluster, which
  *                                        exchange their partial maxima and sums through distributed shared memory (faster
- *                                        than the two-phase form up to about 49152 elements per row, slower beyond: the
+ *                                        than the two-phase form up to about 65536 elements per row, slower beyond: the
  *                                        more CTAs wait for each other per row, the more their skew costs); N <= 131072,
  *                                        else SP_ERR_UNSUPPORTED.  `scheme` / `params` order the row blocks, as for
  *                                        sp_tile_map(M, N, rows, N, ...) with, in integer arithmetic, rows =
