@@ -307,6 +307,23 @@ def workloads_block(sp, names, peaks, stream):
                 lat.append((time.perf_counter() - t0) * 1e6)
             rec["call_to_completion_us"] = min(lat)
             rec["device_us_per_launch_back_to_back"] = med["best"] * 1e3
+            # the same launches replayed from a CUDA graph (200 per graph): what a launch-bound loop should use
+            side, graph, per_graph = torch.cuda.Stream(), torch.cuda.CUDAGraph(), 200
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(graph, stream=side):
+                    for _ in range(per_graph):
+                        sp.gemm(dA, dB, dC, scheme, p, side)
+            for _ in range(3):
+                graph.replay()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(50):
+                graph.replay()
+            e1.record()
+            e1.synchronize()
+            rec["device_us_per_launch_from_a_cuda_graph"] = e0.elapsed_time(e1) / (50 * per_graph) * 1e3
+            del graph
         assert sp.get_status() == 0
         out[name] = rec
         del dA, dB, dC
