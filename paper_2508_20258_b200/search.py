@@ -23,6 +23,7 @@ import os
 import shutil
 import subprocess
 import sys
+import time
 import tempfile
 from dataclasses import asdict, dataclass, field
 from typing import Callable, Dict, List, Optional, Sequence, Tuple
@@ -81,6 +82,12 @@ def default_candidates(units: int) -> List[Tuple[str, int, Dict]]:
     c.append(("group_n:8:s+a", sp.GROUP_N, dict(group=8, flags=ka)))
     c.append(("die_split:m:group_m:8:p:s+a", sp.DIE_SPLIT,
               dict(split_axis=0, inner_scheme=sp.GROUP_M, inner_group=8, flags=ka | sp.FLAG_DIE_PINNED)))
+    # ... and with C stores that give way first in L2 (what the library's own suggestion and the benchmark's defaults use)
+    kah = ka | sp.FLAG_HINT_C_EVICT_FIRST
+    c.append(("group_n:8:s+a+hc", sp.GROUP_N, dict(group=8, flags=kah)))
+    c.append(("die_split:m:group_m:8:p:s+a+hc", sp.DIE_SPLIT,
+              dict(split_axis=0, inner_scheme=sp.GROUP_M, inner_group=8, flags=kah | sp.FLAG_DIE_PINNED)))
+    c.append(("row_major+a+hc", sp.ROW_MAJOR, dict(flags=sp.FLAG_K_ALTERNATE | sp.FLAG_HINT_C_EVICT_FIRST)))
     c.append(("group_m:8+clc", sp.GROUP_M, dict(group=8, flags=sp.FLAG_CLC)))
     return c
 
@@ -165,12 +172,31 @@ def _search_tile(A, B, C, tile, candidates, launches, out_dtype, b_layout, verbo
                 att.status = "wrong"
                 continue
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        if not state.get("settled"):
+            # The chip boosts while it is cool and settles at its power limit within a few hundred milliseconds of load:
+            # the first candidate must not be timed in the boost the later ones never see.  One second of its launches
+            # first; every candidate is then timed over at least 0.15 s.
+            state["settled"] = True
+            t_end = time.perf_counter() + 1.0
+            while time.perf_counter() < t_end:
+                for _ in range(launches):
+                    sp.gemm(A, B, C, scheme, p)
+                torch.cuda.synchronize()
         e0.record()
         for _ in range(launches):
             sp.gemm(A, B, C, scheme, p)
         e1.record()
         e1.synchronize()
-        att.ms = e0.elapsed_time(e1) / launches
+        n_timed = launches
+        one = e0.elapsed_time(e1) / launches
+        if one * launches < 150.0:                      # extend to 0.15 s; the short run above then served as warm-up
+            n_timed = int(min(200000, max(launches, 150.0 / max(one, 1e-4))))
+            e0.record()
+            for _ in range(n_timed):
+                sp.gemm(A, B, C, scheme, p)
+            e1.record()
+            e1.synchronize()
+        att.ms = e0.elapsed_time(e1) / n_timed
         att.tflops = flops / att.ms / 1e9
         state["base_ms"] = state["base_ms"] or att.ms
         att.speedup = state["base_ms"] / att.ms
