@@ -268,6 +268,8 @@ def workloads_block(sp, names, peaks, stream):
         if not out_f32:
             for _ in range(3):
                 torch.matmul(dA, dB, out=dC)
+        # one untimed block first: the first timed block must not run in the boost the later ones never see
+        time_steps(sp, dA, dB, dC, *arm(tile, spec), n, stream)
         launch_bound = flops < 1e9      # 512^3: host and launch jitter is one-sided, so more rounds and the best of them
         for _ in range(4 if launch_bound else 2):
             for k, t_, s_ in arms:
