@@ -47,14 +47,17 @@ class ClockSampler:
 
     def _loop_nvml(self) -> None:
         n = self._nvml
+        watts, i = None, 0
         while not self._stop.is_set():
             try:
                 mhz = float(n.nvmlDeviceGetClockInfo(self._handle, n.NVML_CLOCK_SM))
                 reasons = int(n.nvmlDeviceGetCurrentClocksEventReasons(self._handle))
-                try:
-                    watts = n.nvmlDeviceGetPowerUsage(self._handle) / 1000.0
-                except Exception:
-                    watts = None
+                if i % 8 == 0:      # the power query takes as long as a sampling period: every eighth sample carries a fresh one
+                    try:
+                        watts = n.nvmlDeviceGetPowerUsage(self._handle) / 1000.0
+                    except Exception:
+                        watts = None
+                i += 1
                 self.samples.append((time.perf_counter(), mhz, reasons, watts))
             except Exception:
                 pass
