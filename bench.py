@@ -126,7 +126,8 @@ FALLBACK_SCHEME_BY_TILE = {("cfg3", "256x512"): "group_m:16:s+a+hc", ("cfg5", "2
 # 8192^3 is timed with two 256x256 2-CTA MMA tiles per scheduler tile (they share the A panel: a quarter less operand
 # traffic from L2); the plain 256x256 scheduler tile is timed beside it and reported in the same line.
 DEFAULT_TILE = {"cfg3": "256x512", "cfg2": "256x512",   # 4096^3: A and B fit in L2, the order hardly matters, the wider tile does
-                "cfg5": "256x512"}
+                "cfg5": "256x512",
+                "cfg1": "256x128"}   # 512^3: 8 CTA pairs, a quarter fewer operand bytes per SM than 16 CTAs of 128x128 (7.34 against 7.67 us)
 DEFAULT_SCHEME_BY_TILE = {("cfg3", "256x512"): "die_split:m:group_m:8:p:s+a+hc", ("cfg5", "256x512"): "die_split:m:group_m:8:p:s+a+hc",
                           ("cfg2", "256x512"): "row_major"}
 
