@@ -40,6 +40,15 @@ class ClockSampler:
             self._nvml = pynvml
             self._handle = pynvml.nvmlDeviceGetHandleByIndex(self.index)
             self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self._handle, pynvml.NVML_CLOCK_SM))
+            # the first call of each query takes milliseconds (later ones microseconds): make them here, not inside the
+            # region that is about to be sampled
+            for _ in range(2):
+                pynvml.nvmlDeviceGetClockInfo(self._handle, pynvml.NVML_CLOCK_SM)
+                pynvml.nvmlDeviceGetCurrentClocksEventReasons(self._handle)
+                try:
+                    pynvml.nvmlDeviceGetPowerUsage(self._handle)
+                except Exception:
+                    pass
             return True
         except Exception:
             self._nvml = None
@@ -47,12 +56,16 @@ class ClockSampler:
 
     def _loop_nvml(self) -> None:
         n = self._nvml
-        watts, i = None, 0
+        watts, reasons, i = None, 0, 0
         while not self._stop.is_set():
             try:
+                # every query costs a good part of a sampling period (more on some hosts): the clock is read every time,
+                # the reasons every second time (a sample carries the last mask read, and the union over a window is
+                # what is reported), the power every sixteenth
                 mhz = float(n.nvmlDeviceGetClockInfo(self._handle, n.NVML_CLOCK_SM))
-                reasons = int(n.nvmlDeviceGetCurrentClocksEventReasons(self._handle))
-                if i % 8 == 0:      # the power query takes as long as a sampling period: every eighth sample carries a fresh one
+                if i % 2 == 0:
+                    reasons = int(n.nvmlDeviceGetCurrentClocksEventReasons(self._handle))
+                if i % 16 == 1:
                     try:
                         watts = n.nvmlDeviceGetPowerUsage(self._handle) / 1000.0
                     except Exception:
@@ -81,6 +94,11 @@ class ClockSampler:
             self._stop.wait(max(self.period_s, 0.05))
 
     def start(self) -> "ClockSampler":
+        # the sampling thread re-acquires the interpreter lock after every query; with the default 5 ms switch interval a
+        # busy main thread would hold it off for most of a short timed region
+        import sys
+        if sys.getswitchinterval() > 0.0005:
+            sys.setswitchinterval(0.0005)
         target = self._loop_nvml if self._init_nvml() else self._loop_smi
         self._thread = threading.Thread(target=target, daemon=True)
         self._thread.start()
@@ -94,9 +112,11 @@ class ClockSampler:
     def summary(self, t0: float, t1: float) -> Dict:
         inside = [s for s in self.samples if t0 <= s[0] <= t1]
         window = "timed region"
-        if len(inside) < 3:
-            inside = [s for s in self.samples if t0 - 0.05 <= s[0] <= t1 + 0.05]
-            window = "timed region +-50 ms (too short for 3 samples)"
+        for pad in (0.05, 0.2):      # a region of a few milliseconds may hold fewer than three samples: say how far the window was widened
+            if len(inside) >= 3:
+                break
+            inside = [s for s in self.samples if t0 - pad <= s[0] <= t1 + pad]
+            window = f"timed region +-{int(pad * 1000)} ms (too short for 3 samples)"
         if not inside:
             return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0, "window": window}
         mask = 0
